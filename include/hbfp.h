@@ -1,0 +1,208 @@
+/* hbfp.h - C ABI of the HBFP dot-product path for NVIDIA B200 (sm_100a).
+ *
+ * Hybrid block floating point (Drumond, Lin, Jaggi, Falsafi: "Training DNNs with Hybrid
+ * Block Floating Point") performs every dot product of DNN training in block floating
+ * point (BFP) and everything else in floating point. This library is that dot-product
+ * path: FP32 -> BFP conversion and the BFP matrix products of a training step, as CUDA
+ * kernels. All matrix pointers are DEVICE pointers unless a comment says "host"; all
+ * matrices are row-major; every call is asynchronous on the caller's stream (a
+ * cudaStream_t passed as void*, NULL = the legacy default stream), allocates nothing and
+ * never synchronises unless stated. Functions return an hbfp_status code; on error the
+ * outputs are unspecified but nothing is written out of bounds.
+ *
+ * ---- Number format (Eq. 1; Sec. 4.1; Sec. 5.3) -------------------------------------
+ * A block of values shares one exponent; element i of the block is  q_i * 2^s  with an
+ * integer mantissa q_i of m bits (sign + m-1 magnitude bits, |q_i| <= 2^(m-1)-1).
+ *   amax = max |x_i| over the block;   e = floor(log2 amax) + 1   (exp_mode 0; equals
+ *   ceil(log2 amax) except at exact powers of two, where it avoids saturating the maximum);
+ *   s = max(e - (m-1), -63);  all-zero block: s = -63.
+ *   rounding 0: q = clamp(round-half-even(x * 2^-s));
+ *   rounding 1: stochastic, 16 random bits r per element:
+ *               Y = floor(fl32(x * 2^(16-s))),  q = clamp(floor((Y + r) / 65536)).
+ * The random bits come from Philox4x32-10 with key = (seed lo, seed hi) and counter =
+ * (g lo, g hi, stream_id, 0), g = L >> 3, where L = i*d1 + j is the row-major index of
+ * the element in the FP32 matrix AS PASSED (before any trans flag; independent of
+ * blocking and layout). Of the four output words, element L takes 16-bit half (L & 1) of
+ * word (L & 7) >> 1. The same (seed, stream_id, L) always gives the same draw.
+ * Blocks are 1-D runs of `block` consecutive elements along the contraction axis of the
+ * GEMM the operand feeds (block = 0: the whole axis, i.e. one exponent per row of A / per
+ * column of B, Sec. 4), or, for weights, 2-D tile x tile squares of the stored matrix that
+ * are shared by W and its transpose (Sec. 4.2 "Tiling"). Ragged last blocks share their
+ * exponent among the elements that exist. Inputs must be finite.
+ *
+ * ---- Packed operand layout -----------------------------------------------------------
+ * A quantised GEMM operand with `rows` non-contraction lines and contraction length k:
+ *   b   = block (or k when block == 0),  nkb = ceil(k / b)
+ *   bp  = padded block: 32, 64 or 128 for b <= 32, 64, 128; else b rounded up to 128
+ *   kst = nkb*bp rounded up to a multiple of 128 (bytes per row)
+ *   mantissas: `planes` planes of int8 [rows][kst]; block kb of a row occupies bytes
+ *              [kb*bp, kb*bp + b), everything else in the row is zero. m <= 8: one plane
+ *              holding q. 8 < m <= 12: plane 0 holds hi = q >> 4 (arithmetic), plane 1
+ *              holds lo = q & 15, so q = 16*hi + lo exactly; planes are plane_stride bytes
+ *              apart (rows*kst rounded up to 1024).
+ *   exponents: int8 [nkb][rs], rs = rows rounded up to 16; entry [kb][r] is s of block kb
+ *              of line r (bytes r >= rows are zero).
+ * hbfp_packed_layout() returns these numbers; mantissa and exponent buffers must be
+ * 256-byte and 128-byte aligned respectively (cudaMalloc/torch allocations are).
+ */
+#ifndef HBFP_H_
+#define HBFP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define HBFP_API
+#else
+#define HBFP_API __attribute__((visibility("default")))
+#endif
+
+typedef enum hbfp_status {
+    HBFP_OK = 0,
+    HBFP_ERR_INVALID_ARG = 1, /* null pointer, negative size, ld too small, bad enum value   */
+    HBFP_ERR_UNSUPPORTED = 2, /* a valid request this build has no kernel for                */
+    HBFP_ERR_ALIGNMENT = 3,   /* a packed buffer or C is not aligned as documented           */
+    HBFP_ERR_WORKSPACE = 4,   /* workspace pointer null or smaller than the query returned   */
+    HBFP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor map, ...)  */
+    HBFP_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (see hbfp_device_status) */
+} hbfp_status;
+
+#define HBFP_ROUND_NEAREST_EVEN 0
+#define HBFP_ROUND_STOCHASTIC 1
+
+/* Format of one quantised operand. Set struct_size = sizeof(hbfp_format). */
+typedef struct hbfp_format {
+    uint32_t struct_size;
+    int32_t mant_bits; /* m: 3..12 (sign included). 8 and 12 are the paper's design points     */
+    int32_t block;     /* b: 1-D block length along the contraction axis; 0 = whole axis        */
+    int32_t tile;      /* 0 = 1-D blocks; t > 0 = t x t tiles of the stored matrix (block == t)  */
+    int32_t rounding;  /* HBFP_ROUND_NEAREST_EVEN or HBFP_ROUND_STOCHASTIC                       */
+    int32_t exp_mode;  /* 0 = floor(log2 amax)+1 (default); 1 = literal ceil(log2 amax)          */
+    uint32_t stream_id; /* third Philox counter word: distinct tensors use distinct ids          */
+    uint32_t reserved;  /* must be 0                                                              */
+    uint64_t seed;      /* Philox key                                                             */
+} hbfp_format;
+
+/* Geometry of a packed operand (all host-side numbers). */
+typedef struct hbfp_layout {
+    int64_t rows, k;       /* as passed                                     */
+    int64_t b, bp, nkb;    /* block, padded block, number of blocks         */
+    int64_t kst;           /* bytes per mantissa row                        */
+    int64_t planes;        /* 1 or 2                                        */
+    int64_t plane_stride;  /* bytes between mantissa planes                 */
+    int64_t rs;            /* bytes per exponent row                        */
+    int64_t mant_bytes;    /* planes * plane_stride                         */
+    int64_t exp_bytes;     /* nkb * rs rounded up to 128                    */
+} hbfp_layout;
+
+/* Static, never-freed description of a status code (host). */
+HBFP_API const char* hbfp_status_string(int status);
+
+/* Host-only: layout and buffer sizes of a packed operand with `rows` lines of contraction
+ * length `k` in format `fmt` (Eq. 1 storage; see "Packed operand layout"). */
+HBFP_API int hbfp_packed_layout(int64_t rows, int64_t k, const hbfp_format* fmt, hbfp_layout* out);
+HBFP_API int hbfp_packed_sizes(int64_t rows, int64_t k, const hbfp_format* fmt, size_t* mant_bytes,
+                               size_t* exp_bytes);
+
+/* FP32 -> BFP conversion (Sec. 4.1 "convert tensors to BFP before every dot product, using
+ * the exponent of the largest tensor value"; Sec. 5.3 FP-to-BFP unit).
+ * x: FP32 [d0][d1], row stride ld >= d1 (elements). Blocks run along contract_axis (1 = along
+ * rows of x, 0 = down its columns). Output: packed operand with rows = the other extent and
+ * k = the extent of contract_axis (so contract_axis 0 writes the transposed, contraction-major
+ * layout). With fmt->tile > 0 the exponents are those of tile x tile squares of x and each
+ * entry [kb][r] repeats its tile's exponent. mant / exps: buffers of the sizes
+ * hbfp_packed_sizes(rows, k) returns; fully overwritten. Any d0, d1 >= 0, any ld; the fastest
+ * path needs x 16-byte aligned, ld % 4 == 0 and d1 % 8 == 0. */
+HBFP_API int hbfp_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int contract_axis,
+                           const hbfp_format* fmt, void* mant, int8_t* exps, void* stream);
+
+/* Weight conversion with shared tiles (Sec. 4.2 "Tiling"): one pass over w [d0][d1] that
+ * writes BOTH packed views of the same mantissas - `*_c0` for GEMMs contracting over d0
+ * (rows = d1, k = d0: forward Y = X W) and `*_c1` for GEMMs contracting over d1 (rows = d0,
+ * k = d1: backward-data dX = dY W^T) - plus the tile exponent grid tile_exps
+ * [ceil(d0/t)][ceil(d1/t)] (int8, may be NULL). Requires fmt->tile == fmt->block > 0,
+ * tile <= 128. The backward pass therefore needs no re-quantisation. */
+HBFP_API int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld,
+                                 const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0,
+                                 void* mant_c1, int8_t* exps_c1, int8_t* tile_exps, void* stream);
+
+/* Packed -> canonical arrays for inspection: q [rows][k] int16 mantissas and s [rows][nkb]
+ * int8 exponents (either may be NULL). */
+HBFP_API int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k,
+                         const hbfp_format* fmt, int16_t* q, int8_t* s, void* stream);
+
+/* Packed -> FP32 values q * 2^s (Eq. 1), out [rows][k] with row stride ld. */
+HBFP_API int hbfp_dequantize(const void* mant, const int8_t* exps, int64_t rows, int64_t k,
+                             const hbfp_format* fmt, float* out, int64_t ld, void* stream);
+
+/* One GEMM operand: either an FP32 matrix that the call quantises, or a packed operand
+ * produced earlier (weights live in BFP and are reused, Sec. 4.1). Set struct_size. */
+#define HBFP_OPERAND_FP32 0
+#define HBFP_OPERAND_PACKED 1
+typedef struct hbfp_operand {
+    uint32_t struct_size;
+    int32_t kind;       /* HBFP_OPERAND_FP32 or HBFP_OPERAND_PACKED                                 */
+    const void* data;   /* FP32: the matrix. PACKED: mantissas                                       */
+    const int8_t* exps; /* PACKED only                                                               */
+    int64_t ld;         /* FP32 only: row stride in elements                                         */
+    int32_t trans;      /* FP32 only. A: 0 = stored [M][K], 1 = [K][M]. B: 0 = [K][N], 1 = [N][K]    */
+    int32_t reserved;
+    hbfp_format fmt;    /* FP32: format to quantise to. PACKED: format it was quantised with         */
+} hbfp_operand;
+
+#define HBFP_GEMM_AUTO 0u        /* tensor-core kernel when it supports the case, else SIMT */
+#define HBFP_GEMM_FORCE_SIMT 1u  /* plain dp4a kernel (reference path, any format)           */
+#define HBFP_GEMM_FORCE_TENSOR 2u /* tcgen05 kernel or HBFP_ERR_UNSUPPORTED                  */
+
+/* Host-only: bytes of workspace hbfp_gemm / hbfp_gemm_q need for this problem (packed copies
+ * of FP32 operands, split-K partial tiles). Depends only on its arguments. */
+HBFP_API int hbfp_gemm_workspace(int transA, int transB, int64_t M, int64_t N, int64_t K,
+                                 const hbfp_format* fmtA, const hbfp_format* fmtB, size_t* bytes);
+HBFP_API int hbfp_gemm_q_workspace(int64_t M, int64_t N, int64_t K, const hbfp_operand* a,
+                                   const hbfp_operand* b, size_t* bytes);
+
+/* BFP matrix product C = op(A) op(B) (Eq. 2 per block; blocks accumulated in FP32, Sec. 4):
+ *   P[i][j][kb] = sum_{k in block kb} qA[i][k] * qB[k][j]        exact integers (int32)
+ *   C[i][j]     = sum_kb  float(P[i][j][kb]) * 2^(sA[i][kb] + sB[kb][j])   in FP32
+ * A: FP32 [M][K] (transA = 0) or [K][M] (transA = 1), row stride lda; B: FP32 [K][N] (transB =
+ * 0) or [N][K] (transB = 1), row stride ldb; C: FP32 [M][N], row stride ldc, overwritten.
+ * Both operands are first quantised along the contraction axis (fmtA, fmtB; their blocks must
+ * coincide) into `workspace` (>= hbfp_gemm_workspace bytes, 256-byte aligned).
+ * forward Y = X W is (0,0); backward-data dX = dY W^T is (0,1); backward-weight dW = X^T dY is
+ * (1,0). Without split-K the blocks are accumulated in ascending order with one FP32 rounding
+ * each; with split-K (chosen for small C and long K) each split does so and the splits are
+ * summed in ascending order. The exact range of the scaled FP32 accumulation needs
+ * sA + sB in [-126, 127], sA <= 110 (|A| < 2^117) for 8-bit mantissas. */
+HBFP_API int hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K, const float* A,
+                       int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                       const hbfp_format* fmtA, const hbfp_format* fmtB, void* workspace,
+                       size_t workspace_bytes, uint32_t flags, void* stream);
+
+/* Same product with each operand either FP32 (quantised by the call) or already packed: the
+ * steady state of training, where W is quantised once per step into shared tiles and used by
+ * forward and backward-data (Sec. 4.1, Sec. 4.2). A packed A has rows = M, k = K; a packed B
+ * has rows = N, k = K. */
+HBFP_API int hbfp_gemm_q(int64_t M, int64_t N, int64_t K, const hbfp_operand* a,
+                         const hbfp_operand* b, float* C, int64_t ldc, void* workspace,
+                         size_t workspace_bytes, uint32_t flags, void* stream);
+
+/* Inspection hook: the exact per-block integer sums P [M][N][nkb] (int32) of two packed
+ * operands (Eq. 2's fixed-point dot product), for small shapes. `impl` selects the kernel that
+ * produces them: HBFP_GEMM_FORCE_SIMT or HBFP_GEMM_FORCE_TENSOR. */
+HBFP_API int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbfp_operand* a,
+                                      const hbfp_operand* b, int32_t* P, uint32_t impl,
+                                      void* stream);
+
+/* Synchronises `stream`, then returns and clears the device-side status word of the current
+ * device in *status (host int): 0, or a code recorded by a kernel whose bounded wait on a
+ * barrier expired (the kernel then abandons its work and exits; HBFP_ERR_TIMEOUT is returned). */
+HBFP_API int hbfp_device_status(void* stream, int32_t* status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HBFP_H_ */

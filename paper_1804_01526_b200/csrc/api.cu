@@ -1,0 +1,272 @@
+// extern "C" entry points of the HBFP library: argument checks, workspace carving, dispatch.
+#include "common.cuh"
+
+#include <string.h>
+
+namespace hbfp {
+
+__device__ int32_t g_device_status;
+
+int32_t* device_status_word() {
+    int32_t* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status) != cudaSuccess) return nullptr;
+    return p;
+}
+
+int read_clear_device_status(cudaStream_t st, int32_t* out) {
+    HBFP_CUDA_OK(cudaStreamSynchronize(st));
+    int32_t v = 0, zero = 0;
+    HBFP_CUDA_OK(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)));
+    HBFP_CUDA_OK(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)));
+    *out = v;
+    return v == 0 ? HBFP_OK : HBFP_ERR_TIMEOUT;
+}
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct GemmPlan {
+    Layout la, lb;
+    size_t off_am, off_ae, off_bm, off_be, off_partial, total;
+    TensorPlan tp;
+};
+
+int check_operand(const hbfp_operand* o) {
+    if (!o || o->struct_size != sizeof(hbfp_operand)) return HBFP_ERR_INVALID_ARG;
+    if (o->kind != HBFP_OPERAND_FP32 && o->kind != HBFP_OPERAND_PACKED) return HBFP_ERR_INVALID_ARG;
+    return HBFP_OK;
+}
+
+int make_plan(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp_operand* b, GemmPlan* g) {
+    if (M < 0 || N < 0 || K < 0) return HBFP_ERR_INVALID_ARG;
+    int rc = check_operand(a);
+    if (rc) return rc;
+    rc = check_operand(b);
+    if (rc) return rc;
+    rc = make_layout(M, K, &a->fmt, &g->la);
+    if (rc) return rc;
+    rc = make_layout(N, K, &b->fmt, &g->lb);
+    if (rc) return rc;
+    if (g->la.b != g->lb.b) return HBFP_ERR_INVALID_ARG;   // the blocks of the two operands must coincide
+    size_t off = 0;
+    g->off_am = off; if (a->kind == HBFP_OPERAND_FP32) off += align_up((size_t)g->la.mant_bytes, 1024);
+    g->off_ae = off; if (a->kind == HBFP_OPERAND_FP32) off += align_up((size_t)g->la.exp_bytes, 1024);
+    g->off_bm = off; if (b->kind == HBFP_OPERAND_FP32) off += align_up((size_t)g->lb.mant_bytes, 1024);
+    g->off_be = off; if (b->kind == HBFP_OPERAND_FP32) off += align_up((size_t)g->lb.exp_bytes, 1024);
+    g->tp = plan_gemm_tensor(M, N, K, g->la, g->lb, a->fmt.mant_bits, b->fmt.mant_bits);
+    g->off_partial = off;
+    off += align_up(g->tp.partial_bytes, 1024);
+    g->total = off;
+    return HBFP_OK;
+}
+
+void fill_operand(hbfp_operand* o, const float* data, int64_t ld, int trans, const hbfp_format* f) {
+    memset(o, 0, sizeof(*o));
+    o->struct_size = sizeof(*o);
+    o->kind = HBFP_OPERAND_FP32;
+    o->data = data;
+    o->ld = ld;
+    o->trans = trans;
+    if (f) o->fmt = *f;
+}
+
+// Quantises an FP32 operand into the workspace (or takes a packed one as is).
+int resolve_operand(const hbfp_operand* o, bool is_a, int64_t rows, int64_t K, const Layout& L,
+                    char* ws, size_t off_m, size_t off_e, Packed* out, cudaStream_t st) {
+    out->L = L;
+    out->mant_bits = o->fmt.mant_bits;
+    if (o->kind == HBFP_OPERAND_PACKED) {
+        if (!o->data || !o->exps) return HBFP_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(o->data) & 255) || (reinterpret_cast<uintptr_t>(o->exps) & 127))
+            return HBFP_ERR_ALIGNMENT;
+        out->mant = static_cast<const int8_t*>(o->data);
+        out->exps = o->exps;
+        return HBFP_OK;
+    }
+    if (!o->data && rows * K > 0) return HBFP_ERR_INVALID_ARG;
+    int8_t* m = reinterpret_cast<int8_t*>(ws + off_m);
+    int8_t* e = reinterpret_cast<int8_t*>(ws + off_e);
+    out->mant = m;
+    out->exps = e;
+    const float* x = static_cast<const float*>(o->data);
+    // A: trans 0 = stored [rows][K] (blocks along rows); trans 1 = stored [K][rows].
+    // B: trans 0 = stored [K][rows] (blocks down columns); trans 1 = stored [rows][K].
+    const bool k_contiguous = is_a ? (o->trans == 0) : (o->trans != 0);
+    if (k_contiguous) {
+        if (o->ld < K) return HBFP_ERR_INVALID_ARG;
+        return launch_quantize(x, rows, K, o->ld, 1, &o->fmt, m, e, st);
+    }
+    if (o->ld < rows) return HBFP_ERR_INVALID_ARG;
+    return launch_quantize(x, K, rows, o->ld, 0, &o->fmt, m, e, st);
+}
+
+int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp_operand* b, float* C,
+              int64_t ldc, void* workspace, size_t ws_bytes, uint32_t flags, int32_t* P, cudaStream_t st) {
+    GemmPlan g;
+    int rc = make_plan(M, N, K, a, b, &g);
+    if (rc) return rc;
+    if (flags > HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_INVALID_ARG;
+    if (P) {   // the inspection hook never splits K and needs no scratch
+        g.total -= align_up(g.tp.partial_bytes, 1024);
+        g.tp.partial_bytes = 0;
+        g.tp.splits = 1;
+        g.tp.kb_per_split = g.la.nkb;
+    }
+    if (M == 0 || N == 0) return HBFP_OK;
+    if ((!C && !P) || ldc < N) return HBFP_ERR_INVALID_ARG;
+    if (g.total > 0) {
+        if (!workspace || ws_bytes < g.total) return HBFP_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(workspace) & 255) return HBFP_ERR_ALIGNMENT;
+    }
+    char* ws = static_cast<char*>(workspace);
+    Packed pa, pb;
+    rc = resolve_operand(a, true, M, K, g.la, ws, g.off_am, g.off_ae, &pa, st);
+    if (rc) return rc;
+    rc = resolve_operand(b, false, N, K, g.lb, ws, g.off_bm, g.off_be, &pb, st);
+    if (rc) return rc;
+    const bool want_tensor = flags != HBFP_GEMM_FORCE_SIMT && g.tp.supported &&
+                             (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc % 4) == 0;
+    if (want_tensor)
+        return launch_gemm_tensor(M, N, K, pa, pb, C, ldc, P, g.tp, ws ? ws + g.off_partial : nullptr, st);
+    if (flags == HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_UNSUPPORTED;
+    return launch_gemm_simt(M, N, K, pa, pb, C, ldc, P, st);
+}
+
+}  // namespace
+}  // namespace hbfp
+
+using namespace hbfp;
+
+extern "C" {
+
+const char* hbfp_status_string(int status) {
+    switch (status) {
+        case HBFP_OK: return "ok";
+        case HBFP_ERR_INVALID_ARG: return "invalid argument";
+        case HBFP_ERR_UNSUPPORTED: return "unsupported format or size";
+        case HBFP_ERR_ALIGNMENT: return "buffer not aligned as required";
+        case HBFP_ERR_WORKSPACE: return "workspace missing or too small";
+        case HBFP_ERR_CUDA: return "CUDA call failed";
+        case HBFP_ERR_TIMEOUT: return "bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+int hbfp_packed_layout(int64_t rows, int64_t k, const hbfp_format* fmt, hbfp_layout* out) {
+    if (!out) return HBFP_ERR_INVALID_ARG;
+    Layout L;
+    int rc = make_layout(rows, k, fmt, &L);
+    if (rc) return rc;
+    out->rows = L.rows; out->k = L.k; out->b = L.b; out->bp = L.bp; out->nkb = L.nkb; out->kst = L.kst;
+    out->planes = L.planes; out->plane_stride = L.plane_stride; out->rs = L.rs;
+    out->mant_bytes = L.mant_bytes; out->exp_bytes = L.exp_bytes;
+    return HBFP_OK;
+}
+
+int hbfp_packed_sizes(int64_t rows, int64_t k, const hbfp_format* fmt, size_t* mant_bytes, size_t* exp_bytes) {
+    Layout L;
+    int rc = make_layout(rows, k, fmt, &L);
+    if (rc) return rc;
+    if (mant_bytes) *mant_bytes = (size_t)L.mant_bytes;
+    if (exp_bytes) *exp_bytes = (size_t)L.exp_bytes;
+    return HBFP_OK;
+}
+
+int hbfp_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int contract_axis,
+                  const hbfp_format* fmt, void* mant, int8_t* exps, void* stream) {
+    if (d0 < 0 || d1 < 0 || ld < d1 || (contract_axis != 0 && contract_axis != 1)) return HBFP_ERR_INVALID_ARG;
+    if (!fmt) return HBFP_ERR_INVALID_ARG;
+    if ((!x && d0 * d1 > 0) || !mant || !exps) return HBFP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mant) & 255) || (reinterpret_cast<uintptr_t>(exps) & 127)) return HBFP_ERR_ALIGNMENT;
+    return launch_quantize(x, d0, d1, ld, contract_axis, fmt, static_cast<int8_t*>(mant), exps,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* fmt,
+                        void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, int8_t* tile_exps,
+                        void* stream) {
+    if (d0 < 0 || d1 < 0 || ld < d1 || !fmt) return HBFP_ERR_INVALID_ARG;
+    if ((!w && d0 * d1 > 0) || !mant_c0 || !exps_c0 || !mant_c1 || !exps_c1) return HBFP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mant_c0) & 255) || (reinterpret_cast<uintptr_t>(mant_c1) & 255) ||
+        (reinterpret_cast<uintptr_t>(exps_c0) & 127) || (reinterpret_cast<uintptr_t>(exps_c1) & 127))
+        return HBFP_ERR_ALIGNMENT;
+    return launch_quantize_tiles(w, d0, d1, ld, fmt, static_cast<int8_t*>(mant_c0), exps_c0,
+                                 static_cast<int8_t*>(mant_c1), exps_c1, tile_exps,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k, const hbfp_format* fmt,
+                int16_t* q, int8_t* s, void* stream) {
+    Packed p;
+    int rc = make_layout(rows, k, fmt, &p.L);
+    if (rc) return rc;
+    if (!mant || !exps) return HBFP_ERR_INVALID_ARG;
+    p.mant = static_cast<const int8_t*>(mant);
+    p.exps = exps;
+    p.mant_bits = fmt->mant_bits;
+    return launch_unpack(p, q, s, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_dequantize(const void* mant, const int8_t* exps, int64_t rows, int64_t k, const hbfp_format* fmt,
+                    float* out, int64_t ld, void* stream) {
+    Packed p;
+    int rc = make_layout(rows, k, fmt, &p.L);
+    if (rc) return rc;
+    if (!mant || !exps || !out || ld < k) return HBFP_ERR_INVALID_ARG;
+    p.mant = static_cast<const int8_t*>(mant);
+    p.exps = exps;
+    p.mant_bits = fmt->mant_bits;
+    return launch_dequantize(p, out, ld, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_gemm_q_workspace(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp_operand* b,
+                          size_t* bytes) {
+    if (!bytes) return HBFP_ERR_INVALID_ARG;
+    GemmPlan g;
+    int rc = make_plan(M, N, K, a, b, &g);
+    if (rc) return rc;
+    *bytes = g.total;
+    return HBFP_OK;
+}
+
+int hbfp_gemm_workspace(int transA, int transB, int64_t M, int64_t N, int64_t K, const hbfp_format* fmtA,
+                        const hbfp_format* fmtB, size_t* bytes) {
+    if (!fmtA || !fmtB) return HBFP_ERR_INVALID_ARG;
+    hbfp_operand a, b;
+    fill_operand(&a, nullptr, 0, transA, fmtA);
+    fill_operand(&b, nullptr, 0, transB, fmtB);
+    return hbfp_gemm_q_workspace(M, N, K, &a, &b, bytes);
+}
+
+int hbfp_gemm_q(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp_operand* b, float* C,
+                int64_t ldc, void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+    if (!C && M * N > 0) return HBFP_ERR_INVALID_ARG;
+    return gemm_impl(M, N, K, a, b, C, ldc, workspace, workspace_bytes, flags, nullptr,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K, const float* A, int64_t lda,
+              const float* B, int64_t ldb, float* C, int64_t ldc, const hbfp_format* fmtA,
+              const hbfp_format* fmtB, void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+    if (!fmtA || !fmtB) return HBFP_ERR_INVALID_ARG;
+    hbfp_operand a, b;
+    fill_operand(&a, A, lda, transA, fmtA);
+    fill_operand(&b, B, ldb, transB, fmtB);
+    return hbfp_gemm_q(M, N, K, &a, &b, C, ldc, workspace, workspace_bytes, flags, stream);
+}
+
+int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp_operand* b,
+                             int32_t* P, uint32_t impl, void* stream) {
+    if (!P || !a || !b) return HBFP_ERR_INVALID_ARG;
+    if (a->kind != HBFP_OPERAND_PACKED || b->kind != HBFP_OPERAND_PACKED) return HBFP_ERR_INVALID_ARG;
+    if (impl != HBFP_GEMM_FORCE_SIMT && impl != HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_INVALID_ARG;
+    return gemm_impl(M, N, K, a, b, nullptr, N, nullptr, 0, impl, P, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_device_status(void* stream, int32_t* status) {
+    if (!status) return HBFP_ERR_INVALID_ARG;
+    return read_clear_device_status(static_cast<cudaStream_t>(stream), status);
+}
+
+}  // extern "C"

@@ -1,0 +1,625 @@
+// Tensor-core BFP GEMM for sm_100a: TMA -> shared memory -> tcgen05.mma kind::i8 -> int32 in
+// tensor memory -> per-block rescale into FP32 registers (Eq. 2 per block, blocks accumulated in
+// floating point, Sec. 4).
+//
+// One persistent CTA per SM, 10 warps:
+//   warps 0-7  rescale: tcgen05.ld the int32 block sums, convert, scale by 2^(sA+sB), accumulate
+//              in FP32 registers (128 rows x N_TILE columns per tile), store C
+//   warp 8     TMA producer: mantissa tiles (128B-swizzled, K-major) and exponent slices
+//   warp 9     MMA issuer (one thread) and owner of the tensor-memory allocation
+// A stage is 128 bytes of K for every row of the A (128 rows) and B (N_TILE rows) tiles, i.e. four
+// K=32 MMA steps; a K-block of bp bytes is bp/32 consecutive steps accumulated into one fresh
+// int32 accumulator group in tensor memory. Groups form a ring, so the MMA of the next block
+// overlaps the rescale of the previous one. 12-bit mantissas (two int8 planes, q = 16 hi + lo) use
+// four MMAs per step into three accumulators (hi*hi, hi*lo + lo*hi, lo*lo) that the rescale warps
+// combine exactly in int32.
+//
+// Every wait on an mbarrier is bounded: when it expires the CTA records a code in the device
+// status word, raises a shared abort flag, drains its own copies and MMAs (bounded again),
+// releases tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace hbfp {
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int STAGE_K = 128;          // bytes of K per stage (= one 128B swizzle row)
+constexpr int RESCALE_WARPS = 8;
+constexpr int PRODUCER_WARP = 8;
+constexpr int MMA_WARP = 9;
+constexpr int THREADS = 320;
+constexpr int TMEM_COLS = 512;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
+
+template <int N_TILE, int PLANES>
+struct Cfg {
+    static constexpr int PARTS = PLANES == 1 ? 1 : 3;
+    static constexpr int GROUPS_RAW = TMEM_COLS / (N_TILE * PARTS);
+    static constexpr int GROUPS = GROUPS_RAW > 4 ? 4 : GROUPS_RAW;
+    static constexpr int A_BYTES = TILE_M * STAGE_K;              // per plane
+    static constexpr int B_BYTES = N_TILE * STAGE_K;              // per plane
+    static constexpr int MANT_STAGE = PLANES * (A_BYTES + B_BYTES);
+    static constexpr int EXP_A = 4 * TILE_M, EXP_B = 4 * N_TILE;
+    static constexpr int EXP_STAGE = EXP_A + EXP_B;
+    static constexpr int TABLE_BYTES = 2 * 4 * N_TILE * 4;        // [event parity][block in stage][column]
+    static constexpr int STAGES_RAW = (232448 - 2048 - TABLE_BYTES) / (MANT_STAGE + EXP_STAGE);
+    static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
+    static constexpr int SMEM = 1024 /*align slack*/ + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024 /*barriers*/;
+    static constexpr uint32_t TX_BYTES = MANT_STAGE + EXP_STAGE;
+    static_assert(GROUPS >= 2, "need two accumulator groups to overlap MMA and rescale");
+    static_assert(STAGES >= 3, "pipeline too shallow");
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait. Returns false when the wait was abandoned (abort flag raised by anyone, or the
+// cycle budget ran out, in which case this thread raises the flag and records `code`).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int32_t* status, int code, bool heed_abort) {
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (heed_abort && *abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, int code, bool heed_abort = true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status, code, heed_abort);
+}
+
+// Whole-warp variant: every lane waits and the verdict is made uniform, so that the warp never
+// diverges around the .sync.aligned tensor-memory instructions that follow.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               int32_t* status, int code) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], int8 x int8 -> int32, M = 128, N from idesc, K = 32.
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// 32 lanes x 32 consecutive columns of 32-bit words: thread t of the warp gets lane (base + t).
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major, 128B-swizzled tile: 8-row groups 1024 bytes
+// apart, descriptor version 1 (sm_100), start address advanced by 32 bytes per K=32 step.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: int32 accumulate, signed 8-bit A and B, both K-major, M = 128.
+template <int N_TILE>
+__device__ __forceinline__ constexpr uint32_t idesc_i8() {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------ work decomposition
+
+struct Problem {
+    int64_t M, N;
+    int64_t nkb;            // K-blocks
+    int bp;                 // padded block bytes: 32, 64, 128, or a multiple of 128
+    int tiles_m, tiles_n;
+    int splits;
+    int64_t kb_per_split;
+    int64_t rsA, rsB;       // exponent row strides (only for the dump path's bookkeeping)
+    float* C;
+    int64_t ldc;
+    float* partial;         // [splits][M][ldp] when splits > 1
+    int64_t ldp;
+    int32_t* P;             // optional dump of block sums [M][N][nkb]
+    int32_t* status;
+};
+
+struct Work {
+    int m0, n0, split;
+    int64_t step0, step1;   // K=32 steps [step0, step1), step0 % 4 == 0
+};
+
+__device__ __forceinline__ bool get_work(const Problem& p, int64_t w, Work* out) {
+    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+    if (w >= tiles * p.splits) return false;
+    const int split = (int)(w / tiles);
+    const int64_t t = w % tiles;
+    // groups of 16 tile rows share their B panels in L2 while a group sweeps across N
+    const int G = 16;
+    const int64_t per_group = (int64_t)G * p.tiles_n;
+    const int group = (int)(t / per_group);
+    const int first_m = group * G;
+    const int gsize = min(G, p.tiles_m - first_m);
+    const int64_t within = t % per_group;
+    out->m0 = (first_m + (int)(within % gsize)) * TILE_M;
+    out->n0 = (int)(within / gsize);
+    out->split = split;
+    const int spb = p.bp / 32;
+    const int64_t kb0 = (int64_t)split * p.kb_per_split;
+    const int64_t kb1 = min(p.nkb, kb0 + p.kb_per_split);
+    out->step0 = kb0 * spb;
+    out->step1 = kb1 * spb;
+    return true;
+}
+
+// ------------------------------------------------------------------------------ kernel
+
+template <int N_TILE, int PLANES>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
+               const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+               const __grid_constant__ CUtensorMap mapEA, const __grid_constant__ CUtensorMap mapEB,
+               const Problem p) {
+    using C = Cfg<N_TILE, PLANES>;
+    constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
+    constexpr int COLS_PER_WARP = N_TILE / 2;          // each half of the rescale warps owns half the columns
+
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    const uint32_t mant_base = base;                                        // STAGES x MANT_STAGE, 1024-aligned
+    const uint32_t exp_base = mant_base + STAGES * C::MANT_STAGE;           // STAGES x EXP_STAGE
+    const uint32_t table_off = STAGES * (C::MANT_STAGE + C::EXP_STAGE);
+    int* tables = reinterpret_cast<int*>(base_ptr + table_off);             // [2][4][N_TILE]
+    const uint32_t bar_off = table_off + C::TABLE_BYTES;
+    const uint32_t bars = base + bar_off;
+    const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
+    const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 8 * GROUPS;
+    const uint32_t done_bar = tempty_bar + 8 * GROUPS;
+    const uint32_t tbl_bar = done_bar + 8;                 // one per half of the rescale warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + 16 * STAGES + 16 * GROUPS + 24);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1 + RESCALE_WARPS);
+        }
+        for (int g = 0; g < GROUPS; ++g) {
+            mbar_init(tfull_bar + 8 * g, 1);
+            mbar_init(tempty_bar + 8 * g, RESCALE_WARPS);
+        }
+        mbar_init(done_bar, 1);
+        mbar_init(tbl_bar, RESCALE_WARPS / 2);
+        mbar_init(tbl_bar + 8, RESCALE_WARPS / 2);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == MMA_WARP) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int spb = p.bp / 32;                      // K=32 steps per block
+
+    if (warp == PRODUCER_WARP) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            Work w;
+            for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                const int n0 = w.n0 * N_TILE;
+                for (int64_t st0 = w.step0; st0 < w.step1; st0 += 4, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
+                    const uint32_t fb = full_bar + 8 * s;
+                    mbar_expect_tx(fb, C::TX_BYTES);
+                    const int kbyte = (int)(st0 * 32);
+                    const uint32_t ms = mant_base + s * C::MANT_STAGE;
+                    tma_load_2d(ms, &mapA0, kbyte, w.m0, fb);
+                    tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
+                    if (PLANES == 2) {
+                        tma_load_2d(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb);
+                        tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
+                    }
+                    const int kb = (int)((st0 * 32) / p.bp);        // first block touched by this stage
+                    const uint32_t es = exp_base + s * C::EXP_STAGE;
+                    tma_load_2d(es, &mapEA, w.m0, kb, fb);
+                    tma_load_2d(es + C::EXP_A, &mapEB, n0, kb, fb);
+                }
+            }
+            // Drain: every issued copy must have landed before the CTA may exit. In a normal run
+            // the consumers already waited for all of them, so these return at once.
+            const uint32_t issued = it;
+            for (uint32_t k = issued > (uint32_t)STAGES ? issued - STAGES : 0; k < issued; ++k)
+                mbar_wait(full_bar + 8 * (k % STAGES), (k / STAGES) & 1, abort_flag, p.status, 102, false);
+        }
+    } else if (warp == MMA_WARP) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_i8<N_TILE>();
+            uint32_t it = 0, blk = 0;
+            bool ok = true;
+            Work w;
+            for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                for (int64_t st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 201)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t ms = mant_base + s * C::MANT_STAGE;
+                    const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
+                    const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
+                    const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
+                    for (int j = 0; j < 4; ++j) {
+                        const int64_t step = st0 + j;
+                        if (step >= w.step1) break;
+                        const int pos = (int)(step % spb);
+                        const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
+                        if (pos == 0) {
+                            if (!mbar_wait(tempty_bar + 8 * g, gph ^ 1, abort_flag, p.status, 202)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+                        const uint32_t d = tmem_base + g * PARTS * N_TILE;
+                        const uint64_t ko = (uint64_t)(2 * j);          // 32 bytes per step, in 16-byte units
+                        const uint32_t acc = pos != 0;
+                        tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
+                        if (PLANES == 2) {
+                            tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
+                            tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc, 1u);
+                            tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_lo + ko, idesc, acc);
+                        }
+                        if (pos == spb - 1) {
+                            tc_commit(tfull_bar + 8 * g);
+                            ++blk;
+                        }
+                    }
+                    tc_commit(empty_bar + 8 * s);        // the stage is free once these MMAs have read it
+                }
+            }
+            tc_commit(done_bar);
+            mbar_wait(done_bar, 0, abort_flag, p.status, 203, false);
+        }
+    } else {
+        // ------------------------------------------------------------------ rescale warps
+        const int quarter = warp & 3, half = warp >> 2;
+        const int row = quarter * 32 + lane;                 // row of the tile = tensor-memory lane
+        const int col0 = half * COLS_PER_WARP;
+        const int tid_half = threadIdx.x & 127;
+        float acc[COLS_PER_WARP];
+        uint32_t it = 0, blk = 0, ev = 0;
+        bool ok = true;
+        Work w;
+        for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+            const int n0 = w.n0 * N_TILE;
+#pragma unroll
+            for (int c = 0; c < COLS_PER_WARP; ++c) acc[c] = 0.f;
+            int sa_bits[4] = {0, 0, 0, 0};
+            uint32_t tab_ev = 0;
+            for (int64_t st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
+                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                if (!mbar_wait_warp(full_bar + 8 * s, ph, abort_flag, p.status, 301)) { ok = false; break; }
+                // blocks that start in this stage: build their column tables and fetch this row's exponent
+                const int first_pos = (int)(st0 % spb);
+                const bool has_start = spb <= 4 || first_pos == 0;
+                if (has_start) {
+                    const int8_t* eA = reinterpret_cast<const int8_t*>(base_ptr + (exp_base - base) + s * C::EXP_STAGE);
+                    const int8_t* eB = eA + C::EXP_A;
+                    const int nb = spb >= 4 ? 1 : 4 / spb;           // blocks per stage
+                    tab_ev = ev & 1;
+                    for (int jb = 0; jb < nb; ++jb) {
+                        sa_bits[jb] = ((int)eA[jb * TILE_M + row] + 127) << 23;
+                        for (int c = tid_half; c < COLS_PER_WARP; c += 128)
+                            tables[(tab_ev * 4 + jb) * N_TILE + col0 + c] = (int)eB[jb * N_TILE + col0 + c] << 23;
+                    }
+                    // the four warps of this half publish their table entries to each other
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tbl_bar + 8 * half);
+                    if (!mbar_wait_warp(tbl_bar + 8 * half, ev & 1, abort_flag, p.status, 303)) { ok = false; break; }
+                    ++ev;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar + 8 * s);       // exponent slices of the stage are consumed
+                // blocks that end in this stage
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t step = st0 + j;
+                    if (step >= w.step1) break;
+                    if ((int)(step % spb) != spb - 1) continue;
+                    const int jb = spb >= 4 ? 0 : j / spb;
+                    const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
+                    if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * PARTS * N_TILE + col0;
+                    const int* tab = tables + (tab_ev * 4 + jb) * N_TILE + col0;
+                    const int sa = sa_bits[jb];
+                    const int64_t kb = step / spb;
+#pragma unroll
+                    for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
+                        int v[32];
+                        tc_ld32(taddr + ch * 32, v);
+                        if (PLANES == 2) {
+                            int mid[32], ll[32];
+                            tc_ld32(taddr + N_TILE + ch * 32, mid);
+                            tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
+                        } else {
+                            tc_wait_ld();
+                        }
+                        if (p.P != nullptr) {
+                            const int64_t gi = w.m0 + row;
+                            if (gi < p.M)
+#pragma unroll
+                                for (int c = 0; c < 32; ++c) {
+                                    const int64_t gj = n0 + col0 + ch * 32 + c;
+                                    if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = v[c];
+                                }
+                        }
+#pragma unroll
+                        for (int c4 = 0; c4 < 32; c4 += 4) {
+                            const int4 sb = *reinterpret_cast<const int4*>(tab + ch * 32 + c4);
+                            acc[ch * 32 + c4 + 0] = fmaf((float)v[c4 + 0], __int_as_float(sa + sb.x), acc[ch * 32 + c4 + 0]);
+                            acc[ch * 32 + c4 + 1] = fmaf((float)v[c4 + 1], __int_as_float(sa + sb.y), acc[ch * 32 + c4 + 1]);
+                            acc[ch * 32 + c4 + 2] = fmaf((float)v[c4 + 2], __int_as_float(sa + sb.z), acc[ch * 32 + c4 + 2]);
+                            acc[ch * 32 + c4 + 3] = fmaf((float)v[c4 + 3], __int_as_float(sa + sb.w), acc[ch * 32 + c4 + 3]);
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(tempty_bar + 8 * g);
+                    ++blk;
+                }
+            }
+            if (!ok) break;
+            // ---- store the tile (or this split's partial tile)
+            float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
+            const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
+            const int64_t gi = w.m0 + row;
+            if (dst != nullptr && gi < p.M) {
+                float* rowp = dst + gi * ldd + n0 + col0;
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP; c += 4) {
+                    const int64_t gj = n0 + col0 + c;
+                    if (gj + 3 < p.N) {
+                        *reinterpret_cast<float4*>(rowp + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+                    } else {
+                        for (int e = 0; e < 4; ++e)
+                            if (gj + e < p.N) rowp[c + e] = acc[c + e];
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == MMA_WARP) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// Sums the split-K partial tiles in ascending split order.
+__global__ void splitk_reduce(const float* __restrict__ partial, int splits, int64_t M, int64_t N, int64_t ldp,
+                              float* __restrict__ C, int64_t ldc) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= M * N) return;
+    const int64_t r = i / N, c = i % N;
+    float acc = partial[r * ldp + c];
+    for (int s = 1; s < splits; ++s) acc = __fadd_rn(acc, partial[(int64_t)s * M * ldp + r * ldp + c]);
+    C[r * ldc + c] = acc;
+}
+
+// ------------------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// 2-D byte tensor [outer][inner] with row pitch `pitch`; box {box_inner, box_outer}.
+int make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, uint64_t pitch, uint32_t box_inner,
+             uint32_t box_outer, bool swizzle128) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return HBFP_ERR_CUDA;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {pitch};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HBFP_OK : HBFP_ERR_CUDA;
+}
+
+int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            n = 148;
+    }
+    return n;
+}
+
+template <int N_TILE, int PLANES>
+int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t st) {
+    using C = Cfg<N_TILE, PLANES>;
+    CUtensorMap mA0, mA1, mB0, mB1, mEA, mEB;
+    int rc;
+    rc = make_map(&mA0, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
+    if (rc) return rc;
+    rc = make_map(&mB0, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, N_TILE, true);
+    if (rc) return rc;
+    mA1 = mA0;
+    mB1 = mB0;
+    if (PLANES == 2) {
+        rc = make_map(&mA1, a.mant + a.L.plane_stride, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
+        if (rc) return rc;
+        rc = make_map(&mB1, b.mant + b.L.plane_stride, b.L.kst, b.L.rows, b.L.kst, STAGE_K, N_TILE, true);
+        if (rc) return rc;
+    }
+    rc = make_map(&mEA, a.exps, a.L.rs, a.L.nkb, a.L.rs, TILE_M, 4, false);
+    if (rc) return rc;
+    rc = make_map(&mEB, b.exps, b.L.rs, b.L.nkb, b.L.rs, N_TILE, 4, false);
+    if (rc) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        attr_set = true;
+    }
+    const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
+    const int grid = (int)(work < sm_count() ? work : sm_count());
+    gemm_tc_kernel<N_TILE, PLANES><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
+    return launch_status();
+}
+
+}  // namespace
+
+TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, const Layout& lb, int mant_bits_a,
+                            int mant_bits_b) {
+    TensorPlan t{};
+    (void)mant_bits_a;
+    (void)mant_bits_b;
+    if (M <= 0 || N <= 0 || K <= 0) return t;
+    if (la.planes != lb.planes || la.bp != lb.bp || la.nkb != lb.nkb) return t;
+    const int64_t bp = la.bp;
+    if (!(bp == 32 || bp == 64 || bp == 128 || (bp > 128 && bp % 128 == 0))) return t;
+    if (bp > (1 << 20) || M > (1ll << 30) || N > (1ll << 30) || la.kst > (1ll << 31) - 256) return t;
+    const int64_t tiles_m = (M + TILE_M - 1) / TILE_M;
+    const int SMS = 148;                                   // planning constant: the target part
+    int n_tile;
+    if (la.planes == 2) {
+        n_tile = 64;
+    } else {
+        n_tile = 256;
+        while (n_tile > 64 && (tiles_m * ((N + n_tile - 1) / n_tile) < SMS || N <= n_tile / 2)) n_tile /= 2;
+    }
+    const int64_t tiles = tiles_m * ((N + n_tile - 1) / n_tile);
+    // split-K for small outputs with a long contraction: at least two stages per split, split
+    // boundaries on stage boundaries.
+    const int64_t stages_total = (la.nkb * bp + STAGE_K - 1) / STAGE_K;
+    int64_t splits = 1;
+    if (tiles * 2 <= SMS) {
+        splits = SMS / tiles;
+        if (splits > stages_total / 2) splits = stages_total / 2;
+        if (splits < 1) splits = 1;
+    }
+    const int64_t unit = bp >= STAGE_K ? 1 : STAGE_K / bp;   // blocks per stage
+    int64_t kbps = (la.nkb + splits - 1) / splits;
+    kbps = (kbps + unit - 1) / unit * unit;
+    splits = (la.nkb + kbps - 1) / kbps;
+    t.supported = 1;
+    t.n_tile = n_tile;
+    t.splits = (int)splits;
+    t.kb_per_split = kbps;
+    t.partial_bytes = splits > 1 ? (size_t)splits * (size_t)M * (size_t)round_up(N, 4) * sizeof(float) : 0;
+    return t;
+}
+
+int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const Packed& b, float* Cout, int64_t ldc,
+                       int32_t* P, const TensorPlan& plan, void* partial, cudaStream_t st) {
+    (void)K;
+    if (!plan.supported) return HBFP_ERR_UNSUPPORTED;
+    Problem p{};
+    p.M = M;
+    p.N = N;
+    p.nkb = a.L.nkb;
+    p.bp = (int)a.L.bp;
+    p.tiles_m = (int)((M + TILE_M - 1) / TILE_M);
+    p.tiles_n = (int)((N + plan.n_tile - 1) / plan.n_tile);
+    p.splits = P ? 1 : plan.splits;
+    p.kb_per_split = P ? a.L.nkb : plan.kb_per_split;
+    p.rsA = a.L.rs;
+    p.rsB = b.L.rs;
+    p.C = Cout;
+    p.ldc = ldc;
+    p.partial = static_cast<float*>(partial);
+    p.ldp = round_up(N, 4);
+    p.P = P;
+    p.status = device_status_word();
+    if (!p.status) return HBFP_ERR_CUDA;
+    if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
+    int rc;
+    if (a.L.planes == 2) rc = launch_cfg<64, 2>(p, a, b, st);
+    else if (plan.n_tile == 256) rc = launch_cfg<256, 1>(p, a, b, st);
+    else if (plan.n_tile == 128) rc = launch_cfg<128, 1>(p, a, b, st);
+    else rc = launch_cfg<64, 1>(p, a, b, st);
+    if (rc) return rc;
+    if (p.splits > 1) {
+        const int64_t n = M * N;
+        splitk_reduce<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(p.partial, p.splits, M, N, p.ldp, Cout, ldc);
+        return launch_status();
+    }
+    return HBFP_OK;
+}
+
+}  // namespace hbfp

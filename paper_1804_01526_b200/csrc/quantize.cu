@@ -1,0 +1,634 @@
+// FP32 -> block-floating-point conversion kernels (the FP-to-BFP step of Sec. 4.1 / Sec. 5.3)
+// and the inverse helpers used for inspection. HBM-bound: every FP32 element is read once,
+// one (or two) mantissa bytes and 1/b exponent bytes are written.
+//
+// Kernels
+//   quant_row_fast   blocks along contiguous rows, b in {32,64,128,256}: 8 elements per
+//                    thread (two 128-bit loads, one Philox call in stochastic mode), block
+//                    max by warp shuffles, exponents staged in shared memory so that the
+//                    [kb][row] exponent array is written in full 32-byte sectors.
+//   quant_col_fast   blocks down the columns, b <= 128: a b x 128 FP32 panel is read with
+//                    coalesced row loads into shared memory, reduced down the columns and
+//                    written transposed, so the output is contraction-major again.
+//   quant_tiles      t x t weight tiles (t <= 128): one pass writes both packed views and
+//                    the tile exponent grid.
+//   exps_* / mant_generic   two-pass path for every other geometry (any b, any alignment).
+#include "common.cuh"
+
+namespace hbfp {
+namespace {
+
+// ------------------------------------------------------------------------------ arithmetic
+
+struct QParams {
+    int m;          // mantissa bits
+    int qmax;       // 2^(m-1) - 1
+    int exp_mode;
+    int rounding;
+    uint32_t key0, key1, stream_id;
+};
+
+__device__ __forceinline__ uint32_t abs_bits(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+// Shared exponent (of the mantissa LSB) from the largest |x| of the block, given as its bit
+// pattern: floor(log2 amax) + 1 is the biased exponent field minus 126.
+__device__ __forceinline__ int block_exponent(uint32_t amax_bits, int m, int exp_mode) {
+    int E = (int)(amax_bits >> 23);
+    int e = E - 126;
+    if (exp_mode == 1 && E != 0 && (amax_bits & 0x7fffffu) == 0u) e -= 1;
+    int s = e - (m - 1);
+    s = s < -63 ? -63 : s;
+    return s > 127 ? 127 : s;
+}
+
+__device__ __forceinline__ float pow2f(int e) {   // 2^e for e in [-126, 127]
+    return __uint_as_float((uint32_t)(e + 127) << 23);
+}
+
+__device__ __forceinline__ int clampq(int q, int qmax) { return max(-qmax, min(qmax, q)); }
+
+// round-half-even( x * 2^-s ), saturated
+__device__ __forceinline__ int round_rne(float x, int s, int qmax) {
+    float y = __fmul_rn(x, pow2f(-s));           // s >= -63 and s <= 126 for finite input, m >= 3
+    return clampq(__float2int_rn(y), qmax);
+}
+
+// stochastic: floor( (floor(fl32(x * 2^(16-s))) + r) / 2^16 ), saturated
+__device__ __forceinline__ int round_sr(float x, int s, int qmax, uint32_t r) {
+    float y = __fmul_rn(x, pow2f(16 - s));
+    int Y = __float2int_rd(y);
+    return clampq((Y + (int)r) >> 16, qmax);
+}
+
+// Philox4x32-10 (Salmon et al., SC'11).
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 draws_of_group(const QParams& p, uint64_t g) {
+    return philox4x32_10((uint32_t)g, (uint32_t)(g >> 32), p.stream_id, 0u, p.key0, p.key1);
+}
+
+__device__ __forceinline__ uint32_t draw_from(uint4 w, uint32_t lane8) {   // lane8 = L & 7
+    uint32_t word = (lane8 >> 1) == 0 ? w.x : (lane8 >> 1) == 1 ? w.y : (lane8 >> 1) == 2 ? w.z : w.w;
+    return (word >> (16u * (lane8 & 1u))) & 0xFFFFu;
+}
+
+__device__ __forceinline__ uint32_t draw_of_element(const QParams& p, uint64_t L) {
+    return draw_from(draws_of_group(p, L >> 3), (uint32_t)(L & 7));
+}
+
+__device__ __forceinline__ int quantize_one(float x, int s, const QParams& p, uint64_t L) {
+    if (p.rounding == 0) return round_rne(x, s, p.qmax);
+    return round_sr(x, s, p.qmax, draw_of_element(p, L));
+}
+
+// ------------------------------------------------------------------------------ quant_row_fast
+
+// LPB = lanes per block (b = 8 * LPB). CTA: 256 threads, tile 32 rows x 512 columns.
+template <int LPB, bool SR, int PLANES>
+__global__ void __launch_bounds__(256)
+quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, QParams p,
+               int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
+               int8_t* __restrict__ exps, int64_t rs, int64_t nkb) {
+    constexpr int B = 8 * LPB;
+    constexpr int KB_PER_SPAN = 256 / B;            // blocks in one warp span of 256 columns
+    constexpr int KB_PER_TILE = 512 / B;
+    __shared__ int8_t s_exps[KB_PER_TILE][32];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t r0 = (int64_t)blockIdx.y * 32;
+    const int64_t c0 = (int64_t)blockIdx.x * 512;
+
+    for (int i = tid; i < KB_PER_TILE * 32; i += 256) (&s_exps[0][0])[i] = 0;
+    __syncthreads();
+
+    // warp w owns rows r0 + 4w .. +3, both spans: 8 items, in two batches of 4 rows.
+#pragma unroll
+    for (int span = 0; span < 2; ++span) {
+        float4 v[4][2];
+        const int64_t col = c0 + span * 256 + lane * 8;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t r = r0 + warp * 4 + i;
+            if (r < rows && col < K) {
+                const float4* src = reinterpret_cast<const float4*>(x + r * ld + col);
+                v[i][0] = __ldcs(src);
+                v[i][1] = __ldcs(src + 1);
+            } else {
+                v[i][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                v[i][1] = v[i][0];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t r = r0 + warp * 4 + i;
+            const float e8[8] = {v[i][0].x, v[i][0].y, v[i][0].z, v[i][0].w,
+                                 v[i][1].x, v[i][1].y, v[i][1].z, v[i][1].w};
+            uint32_t am = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) am = max(am, abs_bits(e8[j]));
+#pragma unroll
+            for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+            const int s = block_exponent(am, p.m, p.exp_mode);
+            int q[8];
+            if (SR) {
+                const uint64_t L0 = (uint64_t)(r * K + col);     // multiple of 8 on this path
+                const uint4 w = draws_of_group(p, L0 >> 3);
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    q[j] = round_sr(e8[j], s, p.qmax, (ww[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) q[j] = round_rne(e8[j], s, p.qmax);
+            }
+            if (r < rows && col < kst) {
+                if (PLANES == 1) {
+                    uint2 o;
+                    o.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
+                    o.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | ((uint32_t)(q[7] & 0xff) << 24);
+                    *reinterpret_cast<uint2*>(mant + r * kst + col) = o;
+                } else {
+                    uint2 hi, lo;
+                    hi.x = ((q[0] >> 4) & 0xff) | (((q[1] >> 4) & 0xff) << 8) | (((q[2] >> 4) & 0xff) << 16) | ((uint32_t)((q[3] >> 4) & 0xff) << 24);
+                    hi.y = ((q[4] >> 4) & 0xff) | (((q[5] >> 4) & 0xff) << 8) | (((q[6] >> 4) & 0xff) << 16) | ((uint32_t)((q[7] >> 4) & 0xff) << 24);
+                    lo.x = (q[0] & 15) | ((q[1] & 15) << 8) | ((q[2] & 15) << 16) | ((uint32_t)(q[3] & 15) << 24);
+                    lo.y = (q[4] & 15) | ((q[5] & 15) << 8) | ((q[6] & 15) << 16) | ((uint32_t)(q[7] & 15) << 24);
+                    *reinterpret_cast<uint2*>(mant + r * kst + col) = hi;
+                    *reinterpret_cast<uint2*>(mant + plane_stride + r * kst + col) = lo;
+                }
+            }
+            if ((lane % LPB) == 0 && r < rows && col < K)
+                s_exps[span * KB_PER_SPAN + lane / LPB][warp * 4 + i] = (int8_t)s;
+        }
+    }
+    __syncthreads();
+    // exponents: [kb][row], 32 rows of one block are 32 contiguous bytes.
+    const int64_t kb0 = c0 / B;
+    for (int i = tid; i < KB_PER_TILE * 8; i += 256) {
+        const int kbl = i >> 3, part = i & 7;
+        const int64_t kb = kb0 + kbl, r = r0 + part * 4;
+        if (kb < nkb && r < rs)
+            *reinterpret_cast<uint32_t*>(exps + kb * rs + r) =
+                *reinterpret_cast<const uint32_t*>(&s_exps[kbl][part * 4]);
+    }
+}
+
+// ------------------------------------------------------------------------------ quant_col_fast
+
+// Blocks down the columns of x [K][R] (contract axis 0); output rows are the columns of x.
+// CTA: 128 threads, one block of b <= 128 k-rows by 128 columns.
+constexpr int COLT = 128;
+
+template <int PLANES>
+__global__ void __launch_bounds__(128)
+quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, int b, int bp, QParams p,
+               int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
+               int8_t* __restrict__ exps, int64_t rs, int64_t nkb, int vec_ok) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* tile = reinterpret_cast<float*>(smem_raw);                 // [b][COLT]
+    uint4* rnd = reinterpret_cast<uint4*>(tile + (size_t)b * COLT);   // [b][COLT/8] (stochastic only)
+
+    const int tid = threadIdx.x;
+    const int64_t kb = blockIdx.y;
+    const int64_t c0 = (int64_t)blockIdx.x * COLT;
+    const int64_t k0 = kb * b;
+    const int blen = (int)min((int64_t)b, K - k0);
+
+    // 1. coalesced load of the panel (zero beyond the matrix).
+    if (vec_ok) {
+        for (int i = tid; i < blen * (COLT / 4); i += 128) {
+            const int kk = i / (COLT / 4), c4 = (i % (COLT / 4)) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c0 + c4 < R) v = __ldcs(reinterpret_cast<const float4*>(x + (k0 + kk) * ld + c0 + c4));
+            *reinterpret_cast<float4*>(tile + kk * COLT + c4) = v;      // R % 4 == 0 on this path
+        }
+    } else {
+        for (int i = tid; i < blen * COLT; i += 128) {
+            const int kk = i / COLT, c = i % COLT;
+            tile[kk * COLT + c] = (c0 + c < R) ? x[(k0 + kk) * ld + c0 + c] : 0.f;
+        }
+    }
+    // 2. stochastic mode: one Philox call per 8 consecutive source elements of a row.
+    const bool group_ok = (R % 8) == 0;     // then L = k*R + c has L & 7 == c & 7 and groups align
+    if (p.rounding == 1 && group_ok) {
+        for (int i = tid; i < blen * (COLT / 8); i += 128) {
+            const int kk = i / (COLT / 8), g8 = i % (COLT / 8);
+            const uint64_t L = (uint64_t)((k0 + kk) * R + c0 + g8 * 8);
+            rnd[kk * (COLT / 8) + g8] = draws_of_group(p, L >> 3);
+        }
+    }
+    __syncthreads();
+
+    // 3. thread = column: max down the block, exponent, mantissas, transposed store.
+    const int64_t c = c0 + tid;
+    uint32_t am = 0;
+    for (int kk = 0; kk < blen; ++kk) am = max(am, abs_bits(tile[kk * COLT + tid]));
+    const int s = block_exponent(am, p.m, p.exp_mode);
+    if (c < R) {
+        exps[kb * rs + c] = (int8_t)s;
+        int8_t* dst = mant + c * kst + kb * bp;
+        const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
+        for (int w0 = 0; w0 < bp; w0 += 16) {
+            uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int kk = w0 + j;
+                int q = 0;
+                if (kk < blen) {
+                    const float v = tile[kk * COLT + tid];
+                    if (p.rounding == 0) q = round_rne(v, s, p.qmax);
+                    else if (group_ok) q = round_sr(v, s, p.qmax, rnd16[(kk * (COLT / 8) + (tid >> 3)) * 8 + (tid & 7)]);
+                    else q = round_sr(v, s, p.qmax, draw_of_element(p, (uint64_t)((k0 + kk) * R + c)));
+                }
+                if (PLANES == 1) {
+                    hi[j >> 2] |= (uint32_t)(q & 0xff) << (8 * (j & 3));
+                } else {
+                    hi[j >> 2] |= (uint32_t)((q >> 4) & 0xff) << (8 * (j & 3));
+                    lo[j >> 2] |= (uint32_t)(q & 15) << (8 * (j & 3));
+                }
+            }
+            *reinterpret_cast<uint4*>(dst + w0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            if (PLANES == 2) *reinterpret_cast<uint4*>(dst + plane_stride + w0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
+        // zero the row tail [nkb*bp, kst) once, by the CTA of the last block.
+        if (kb == nkb - 1) {
+            for (int64_t o = nkb * bp; o < kst; o += 16) {
+                *reinterpret_cast<uint4*>(mant + c * kst + o) = make_uint4(0, 0, 0, 0);
+                if (PLANES == 2) *reinterpret_cast<uint4*>(mant + plane_stride + c * kst + o) = make_uint4(0, 0, 0, 0);
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------ quant_tiles
+
+// One CTA per t x t tile of w [d0][d1] (t <= 128), 256 threads.
+//   view c1: rows = d0, contraction along d1 (the stored orientation)
+//   view c0: rows = d1, contraction along d0 (the transpose)
+template <int PLANES>
+__global__ void __launch_bounds__(256)
+quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int t, int tp, QParams p,
+            int8_t* __restrict__ mant_c0, int64_t kst0, int64_t ps0, int8_t* __restrict__ exps_c0, int64_t rs0, int64_t nkb0,
+            int8_t* __restrict__ mant_c1, int64_t kst1, int64_t ps1, int8_t* __restrict__ exps_c1, int64_t rs1, int64_t nkb1,
+            int8_t* __restrict__ grid, int64_t grid_ld) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* tile = reinterpret_cast<float*>(smem_raw);                  // [t][t+1]
+    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp] zero padded
+    __shared__ uint32_t s_am[8];
+    __shared__ int s_exp;
+
+    const int tid = threadIdx.x;
+    const int64_t u = blockIdx.y, v = blockIdx.x;       // tile row (along d0), tile column (along d1)
+    const int64_t i0 = u * t, j0 = v * t;
+    const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
+
+    uint32_t am = 0;
+    for (int e = tid; e < hi * t; e += 256) {
+        const int ii = e / t, jj = e % t;
+        float val = 0.f;
+        if (jj < wj) val = w[(i0 + ii) * ld + j0 + jj];
+        tile[ii * (t + 1) + jj] = val;
+        am = max(am, abs_bits(val));
+    }
+    for (int e = tid; e < tp * tp; e += 256) qt[e] = 0;
+    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    if ((tid & 31) == 0) s_am[tid >> 5] = am;
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t a = 0;
+        for (int i = 0; i < 8; ++i) a = max(a, s_am[i]);
+        s_exp = block_exponent(a, p.m, p.exp_mode);
+        if (grid) grid[u * grid_ld + v] = (int8_t)s_exp;
+    }
+    __syncthreads();
+    const int s = s_exp;
+    for (int e = tid; e < hi * wj; e += 256) {
+        const int ii = e / wj, jj = e % wj;
+        const uint64_t L = (uint64_t)((i0 + ii) * d1 + j0 + jj);
+        qt[ii * tp + jj] = (int16_t)quantize_one(tile[ii * (t + 1) + jj], s, p, L);
+    }
+    __syncthreads();
+    // view c1: row i0+ii gets bytes [v*tp, v*tp+tp) = qt[ii][0..tp)
+    if (mant_c1) for (int e = tid; e < hi * (tp / 4); e += 256) {
+        const int ii = e / (tp / 4), g = (e % (tp / 4)) * 4;
+        uint32_t h = 0, l = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = qt[ii * tp + g + j];
+            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
+            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+        }
+        int8_t* dst = mant_c1 + (i0 + ii) * kst1 + v * tp + g;
+        *reinterpret_cast<uint32_t*>(dst) = h;
+        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps1) = l;
+    }
+    // view c0: row j0+jj gets bytes [u*tp, u*tp+tp) = qt[0..tp)[jj]
+    if (mant_c0) for (int e = tid; e < wj * (tp / 4); e += 256) {
+        const int jj = e % wj, g = (e / wj) * 4;
+        uint32_t h = 0, l = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = qt[(g + j) * tp + jj];
+            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
+            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+        }
+        int8_t* dst = mant_c0 + (j0 + jj) * kst0 + u * tp + g;
+        *reinterpret_cast<uint32_t*>(dst) = h;
+        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps0) = l;
+    }
+    // replicated exponents: exps_c1[v][i0+ii], exps_c0[u][j0+jj]
+    if (exps_c1) for (int e = tid; e < hi; e += 256) exps_c1[v * rs1 + i0 + e] = (int8_t)s;
+    if (exps_c0) for (int e = tid; e < wj; e += 256) exps_c0[u * rs0 + j0 + e] = (int8_t)s;
+    // row tails beyond the last tile: zero them (last tile column / last tile row only)
+    if (mant_c1 && v == nkb1 - 1)
+        for (int64_t e = tid; e < (int64_t)hi * ((kst1 - nkb1 * tp) / 4); e += 256) {
+            const int64_t per = (kst1 - nkb1 * tp) / 4, ii = e / per, o = nkb1 * tp + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(mant_c1 + (i0 + ii) * kst1 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c1 + ps1 + (i0 + ii) * kst1 + o) = 0;
+        }
+    if (mant_c0 && u == nkb0 - 1)
+        for (int64_t e = tid; e < (int64_t)wj * ((kst0 - nkb0 * tp) / 4); e += 256) {
+            const int64_t per = (kst0 - nkb0 * tp) / 4, jj = e / per, o = nkb0 * tp + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(mant_c0 + (j0 + jj) * kst0 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c0 + ps0 + (j0 + jj) * kst0 + o) = 0;
+        }
+}
+
+// ------------------------------------------------------------------------------ generic two-pass path
+
+// Element (r, kk) of the operand view: r = line, kk = position along the contraction axis.
+__device__ __forceinline__ float view_at(const float* x, int64_t ld, int axis, int64_t r, int64_t kk) {
+    return axis == 1 ? x[r * ld + kk] : x[kk * ld + r];
+}
+
+// Pass 1a, blocks along rows: one warp per (line, block).
+__global__ void exps_axis1(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t b,
+                           int64_t nkb, QParams p, int8_t* __restrict__ exps, int64_t rs) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t item = warp; item < rows * nkb; item += nwarps) {
+        const int64_t r = item / nkb, kb = item % nkb;
+        const int64_t k1 = min(K, (kb + 1) * b);
+        uint32_t am = 0;
+        for (int64_t kk = kb * b + lane; kk < k1; kk += 32) am = max(am, abs_bits(x[r * ld + kk]));
+        for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        if (lane == 0) exps[kb * rs + r] = (int8_t)block_exponent(am, p.m, p.exp_mode);
+    }
+}
+
+// Pass 1b, blocks down columns: one thread per (block, line); neighbouring threads read
+// neighbouring addresses.
+__global__ void exps_axis0(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t b,
+                           int64_t nkb, QParams p, int8_t* __restrict__ exps, int64_t rs) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * nkb) return;
+    const int64_t kb = i / rows, r = i % rows;
+    const int64_t k1 = min(K, (kb + 1) * b);
+    uint32_t am = 0;
+    for (int64_t kk = kb * b; kk < k1; ++kk) am = max(am, abs_bits(x[kk * ld + r]));
+    exps[kb * rs + r] = (int8_t)block_exponent(am, p.m, p.exp_mode);
+}
+
+// Pass 1c, t x t tiles of the stored matrix [d0][d1]: one warp per tile computes the tile's
+// exponent and repeats it for every line of the view that crosses the tile.
+__global__ void exps_tiles(const float* __restrict__ x, int64_t d0, int64_t d1, int64_t ld, int64_t t,
+                           QParams p, int axis, int8_t* __restrict__ exps, int64_t rs, int64_t nu, int64_t nv) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (warp >= nu * nv) return;
+    const int64_t u = warp / nv, v = warp % nv;
+    const int64_t i1 = min(d0, (u + 1) * t), j1 = min(d1, (v + 1) * t);
+    uint32_t am = 0;
+    for (int64_t i = u * t; i < i1; ++i)
+        for (int64_t j = v * t + lane; j < j1; j += 32) am = max(am, abs_bits(x[i * ld + j]));
+    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    const int8_t s = (int8_t)block_exponent(am, p.m, p.exp_mode);
+    // axis 1: lines are stored rows, block index is the tile column. axis 0: the transpose.
+    if (axis == 1) for (int64_t i = u * t + lane; i < i1; i += 32) exps[v * rs + i] = s;
+    else for (int64_t j = v * t + lane; j < j1; j += 32) exps[u * rs + j] = s;
+}
+
+// Pass 2: one thread per 4 output bytes of a line; reads the exponent written by pass 1.
+template <int PLANES>
+__global__ void mant_generic(const float* __restrict__ x, int64_t d1, int64_t rows, int64_t K, int64_t ld,
+                             int axis, int64_t b, int64_t bp, int64_t nkb, QParams p,
+                             const int8_t* __restrict__ exps, int64_t rs, int8_t* __restrict__ mant,
+                             int64_t kst, int64_t plane_stride) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t per = kst / 4;
+    if (i >= rows * per) return;
+    const int64_t r = i / per, o = (i % per) * 4;
+    uint32_t h = 0, l = 0;
+    const int64_t kb = o / bp;
+    if (kb < nkb) {
+        const int s = exps[kb * rs + r];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t within = o % bp + j, kk = kb * b + within;
+            int q = 0;
+            if (within < b && kk < K) {
+                const uint64_t L = axis == 1 ? (uint64_t)(r * d1 + kk) : (uint64_t)(kk * d1 + r);
+                q = quantize_one(view_at(x, ld, axis, r, kk), s, p, L);
+            }
+            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
+            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+        }
+    }
+    *reinterpret_cast<uint32_t*>(mant + r * kst + o) = h;
+    if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant + plane_stride + r * kst + o) = l;
+}
+
+// ------------------------------------------------------------------------------ inverse helpers
+
+__global__ void unpack_kernel(const int8_t* __restrict__ mant, const int8_t* __restrict__ exps, int64_t rows,
+                              int64_t K, int64_t b, int64_t bp, int64_t nkb, int64_t kst, int64_t plane_stride,
+                              int planes, int64_t rs, int16_t* __restrict__ q, int8_t* __restrict__ s) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q && i < rows * K) {
+        const int64_t r = i / K, kk = i % K, o = (kk / b) * bp + kk % b;
+        int v = mant[r * kst + o];
+        if (planes == 2) v = v * 16 + mant[plane_stride + r * kst + o];
+        q[i] = (int16_t)v;
+    }
+    if (s && i < rows * nkb) {
+        const int64_t r = i / nkb, kb = i % nkb;
+        s[i] = exps[kb * rs + r];
+    }
+}
+
+__global__ void dequant_kernel(const int8_t* __restrict__ mant, const int8_t* __restrict__ exps, int64_t rows,
+                               int64_t K, int64_t b, int64_t bp, int64_t kst, int64_t plane_stride, int planes,
+                               int64_t rs, float* __restrict__ out, int64_t ld) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * K) return;
+    const int64_t r = i / K, kk = i % K, kb = kk / b, o = kb * bp + kk % b;
+    int v = mant[r * kst + o];
+    if (planes == 2) v = v * 16 + mant[plane_stride + r * kst + o];
+    out[r * ld + kk] = ldexpf((float)v, (int)exps[kb * rs + r]);
+}
+
+QParams make_params(const hbfp_format* f) {
+    QParams p;
+    p.m = f->mant_bits;
+    p.qmax = (1 << (f->mant_bits - 1)) - 1;
+    p.exp_mode = f->exp_mode;
+    p.rounding = f->rounding;
+    p.key0 = (uint32_t)f->seed;
+    p.key1 = (uint32_t)(f->seed >> 32);
+    p.stream_id = f->stream_id;
+    return p;
+}
+
+inline unsigned blocks_for(int64_t n, int threads) { return (unsigned)((n + threads - 1) / threads); }
+
+template <int LPB>
+int launch_row_fast(const float* x, int64_t rows, int64_t K, int64_t ld, const QParams& p, const Layout& L,
+                    int8_t* mant, int8_t* exps, cudaStream_t st) {
+    dim3 grid((unsigned)((L.kst + 511) / 512), (unsigned)((rows + 31) / 32));
+    // the last column tile must also cover the exponent rows of blocks that start before K
+    if (p.rounding == 1) {
+        if (L.planes == 1) quant_row_fast<LPB, true, 1><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb);
+        else quant_row_fast<LPB, true, 2><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb);
+    } else {
+        if (L.planes == 1) quant_row_fast<LPB, false, 1><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb);
+        else quant_row_fast<LPB, false, 2><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb);
+    }
+    return launch_status();
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------ launchers
+
+int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis, const hbfp_format* f,
+                    int8_t* mant, int8_t* exps, cudaStream_t st) {
+    const int64_t K = axis == 1 ? d1 : d0, rows = axis == 1 ? d0 : d1;
+    Layout L;
+    int rc = make_layout(rows, K, f, &L);
+    if (rc) return rc;
+    if (rows == 0) return HBFP_OK;
+    const QParams p = make_params(f);
+    if (K == 0) {
+        HBFP_CUDA_OK(cudaMemsetAsync(mant, 0, (size_t)L.mant_bytes, st));
+        HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        return HBFP_OK;
+    }
+    const bool aligned = ((reinterpret_cast<uintptr_t>(x) & 15) == 0) && (ld % 4 == 0);
+    if (rows * L.kst >= (int64_t)1 << 40) return HBFP_ERR_UNSUPPORTED;
+
+    if (f->tile == 0 && axis == 1 && aligned && d1 % 8 == 0 && L.b == L.bp && L.b <= 256 &&
+        rows <= 32ll * 65535) {
+        switch (L.b) {
+            case 32: return launch_row_fast<4>(x, rows, K, ld, p, L, mant, exps, st);
+            case 64: return launch_row_fast<8>(x, rows, K, ld, p, L, mant, exps, st);
+            case 128: return launch_row_fast<16>(x, rows, K, ld, p, L, mant, exps, st);
+            case 256: return launch_row_fast<32>(x, rows, K, ld, p, L, mant, exps, st);
+            default: break;
+        }
+    }
+    if (f->tile == 0 && axis == 0 && L.b <= 128 && L.nkb <= 65535) {
+        const int vec_ok = aligned && (rows % 4 == 0);
+        size_t smem = (size_t)L.b * COLT * sizeof(float) + (p.rounding ? (size_t)L.b * (COLT / 8) * sizeof(uint4) : 0);
+        dim3 grid((unsigned)((rows + COLT - 1) / COLT), (unsigned)L.nkb);
+        // exponent padding bytes (lines >= rows) are documented as zero
+        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        if (L.planes == 1) {
+            HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_fast<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            quant_col_fast<1><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+        } else {
+            HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_fast<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            quant_col_fast<2><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+        }
+        return launch_status();
+    }
+
+    if (f->tile > 0 && f->tile <= 128) {
+        // single view of a tiled weight: the fused tile kernel with the other view switched off
+        return axis == 0 ? launch_quantize_tiles(x, d0, d1, ld, f, mant, exps, nullptr, nullptr, nullptr, st)
+                         : launch_quantize_tiles(x, d0, d1, ld, f, nullptr, nullptr, mant, exps, nullptr, st);
+    }
+
+    // generic two-pass path
+    HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+    if (f->tile == 0) {
+        if (axis == 1) {
+            int64_t items = rows * L.nkb;
+            int64_t want = (items + 7) / 8;
+            unsigned blocks = (unsigned)(want < 148 * 32 ? want : 148 * 32);
+            exps_axis1<<<blocks, 256, 0, st>>>(x, rows, K, ld, L.b, L.nkb, p, exps, L.rs);
+        } else {
+            exps_axis0<<<blocks_for(rows * L.nkb, 256), 256, 0, st>>>(x, rows, K, ld, L.b, L.nkb, p, exps, L.rs);
+        }
+    } else {
+        const int64_t t = f->tile, nu = (d0 + t - 1) / t, nv = (d1 + t - 1) / t;
+        exps_tiles<<<blocks_for(nu * nv * 32, 256), 256, 0, st>>>(x, d0, d1, ld, t, p, axis, exps, L.rs, nu, nv);
+    }
+    if (launch_status()) return HBFP_ERR_CUDA;
+    if (L.planes == 1)
+        mant_generic<1><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(x, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
+    else
+        mant_generic<2><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(x, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
+    return launch_status();
+}
+
+int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* f,
+                          int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                          int8_t* tile_exps, cudaStream_t st) {
+    if (f->tile <= 0 || f->tile != f->block) return HBFP_ERR_INVALID_ARG;
+    if (f->tile > 128) return HBFP_ERR_UNSUPPORTED;
+    Layout L0, L1;
+    int rc = make_layout(d1, d0, f, &L0);     // view c0: rows = d1, k = d0
+    if (rc) return rc;
+    rc = make_layout(d0, d1, f, &L1);         // view c1: rows = d0, k = d1
+    if (rc) return rc;
+    if (d0 == 0 || d1 == 0) return HBFP_OK;
+    const QParams p = make_params(f);
+    const int t = f->tile, tp = (int)L0.bp;
+    const int64_t nu = L0.nkb, nv = L1.nkb;   // tiles along d0, along d1
+    if (nu > 65535) return HBFP_ERR_UNSUPPORTED;
+    if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
+    if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
+    size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * tp * sizeof(int16_t);
+    dim3 grid((unsigned)nv, (unsigned)nu);
+    if (L0.planes == 1) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(quant_tiles<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        quant_tiles<1><<<grid, 256, smem, st>>>(w, d0, d1, ld, t, tp, p, mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb,
+                                               mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb, tile_exps, nv);
+    } else {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(quant_tiles<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        quant_tiles<2><<<grid, 256, smem, st>>>(w, d0, d1, ld, t, tp, p, mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb,
+                                               mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb, tile_exps, nv);
+    }
+    return launch_status();
+}
+
+int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st) {
+    const Layout& L = p.L;
+    int64_t n = L.rows * (L.k > L.nkb ? L.k : L.nkb);
+    if (n == 0) return HBFP_OK;
+    unpack_kernel<<<blocks_for(n, 256), 256, 0, st>>>(p.mant, p.exps, L.rows, L.k, L.b, L.bp, L.nkb, L.kst,
+                                                     L.plane_stride, (int)L.planes, L.rs, q, s);
+    return launch_status();
+}
+
+int launch_dequantize(const Packed& p, float* out, int64_t ld, cudaStream_t st) {
+    const Layout& L = p.L;
+    if (L.rows * L.k == 0) return HBFP_OK;
+    dequant_kernel<<<blocks_for(L.rows * L.k, 256), 256, 0, st>>>(p.mant, p.exps, L.rows, L.k, L.b, L.bp, L.kst,
+                                                                 L.plane_stride, (int)L.planes, L.rs, out, ld);
+    return launch_status();
+}
+
+}  // namespace hbfp

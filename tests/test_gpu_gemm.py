@@ -1,0 +1,130 @@
+"""GPU parity of the BFP GEMMs through the C ABI: per-block integer sums bit-exact, outputs within
+1e-6 of the FP32 accumulator magnitude of the oracle's order-free reference, and bit-equal to the
+oracle's sequential accumulation where the kernel accumulates blocks in ascending order."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1804_01526_b200 import workloads as wl
+from tests.helpers import gfmt, ofmt, to_dev
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-6      # of the accumulator magnitude sum_kb |T|, as the target states
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_1804_01526_b200 import binding
+    binding.lib()
+    return binding
+
+
+def run_spec(hb, sp, tensors, flags, expect_seq=True):
+    A, B = tensors[sp.a_key], tensors[sp.b_key]
+    ref = oracle.hbfp_gemm(sp.transA, sp.transB, A, B, ofmt(sp.fmt_a), ofmt(sp.fmt_b))
+    C = hb.gemm(sp.transA, sp.transB, to_dev(A), to_dev(B), gfmt(sp.fmt_a), gfmt(sp.fmt_b), flags=flags)
+    C = C.cpu().numpy()
+    assert hb.device_status() == 0
+    err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all(), (sp.name, float((err / np.maximum(ref["a_mag"], 1e-300)).max()))
+    if expect_seq:
+        assert np.array_equal(C, ref["c_seq"]), sp.name
+    return C, ref
+
+
+def impls(hb):
+    return [hb.GEMM_FORCE_SIMT, hb.GEMM_AUTO]
+
+
+@pytest.mark.parametrize("flag", ["simt", "auto"])
+def test_single_256_cube(hb, flag):
+    specs = wl.config_single_256()
+    t = wl.materialize(specs, seed=0)
+    run_spec(hb, specs[0], t, hb.GEMM_FORCE_SIMT if flag == "simt" else hb.GEMM_AUTO)
+
+
+@pytest.mark.parametrize("flag", ["simt", "auto"])
+def test_mlp_training_step_gemms(hb, flag):
+    specs = wl.config_mlp()
+    t = wl.materialize(specs, seed=1)
+    for sp in specs:
+        run_spec(hb, sp, t, hb.GEMM_FORCE_SIMT if flag == "simt" else hb.GEMM_AUTO,
+                 expect_seq=(flag == "simt"))
+
+
+@pytest.mark.parametrize("flag", ["simt", "auto"])
+def test_resnet_im2col_gemms_reduced_batch(hb, flag):
+    # batch 2 instead of 128 (M = 2048 / 512 rows): same K, N, formats and value laws
+    specs = wl.config_resnet_im2col(batch=2)
+    t = wl.materialize(specs, seed=2)
+    for sp in specs:
+        run_spec(hb, sp, t, hb.GEMM_FORCE_SIMT if flag == "simt" else hb.GEMM_AUTO,
+                 expect_seq=(flag == "simt"))
+
+
+@pytest.mark.parametrize("flag", ["simt", "auto"])
+def test_transformer_gemms_reduced(hb, flag):
+    # tokens 192, hidden 256: 12-bit hi/lo mantissas, 64 x 64 shared weight tiles, stochastic rounding
+    specs = wl.config_transformer(tokens=192, hidden=256)
+    t = wl.materialize(specs, seed=7)
+    for sp in specs:
+        run_spec(hb, sp, t, hb.GEMM_FORCE_SIMT if flag == "simt" else hb.GEMM_AUTO,
+                 expect_seq=(flag == "simt"))
+
+
+@pytest.mark.parametrize("impl", ["simt", "tensor"])
+@pytest.mark.parametrize("m,b,M,N,K", [(8, 32, 200, 136, 288), (8, 128, 130, 260, 1024), (12, 64, 96, 72, 320),
+                                       (8, 24, 50, 40, 100), (8, 0, 64, 64, 700), (8, 64, 128, 256, 512)])
+def test_block_partials_are_bit_exact(hb, impl, m, b, M, N, K):
+    A = wl.draw("lognormal", (M, K), seed=21)
+    B = wl.draw("lognormal", (K, N), seed=22)
+    fd = dict(mant_bits=m, block=b, rounding=1, seed=4)
+    qA, sA = oracle.quantize(A, 1, ofmt(fd))
+    qB, sB = oracle.quantize(B, 0, ofmt(fd, stream_id=1))
+    ref = oracle.gemm(qA, sA, qB, sB, b, want_partials=True)
+    pa = hb.quantize(to_dev(A), 1, gfmt(fd))
+    pb = hb.quantize(to_dev(B), 0, gfmt(fd, stream_id=1))
+    flag = hb.GEMM_FORCE_SIMT if impl == "simt" else hb.GEMM_FORCE_TENSOR
+    try:
+        P = hb.gemm_block_partials(pa, pb, flag)
+    except hb.HbfpError as e:
+        if impl == "tensor" and e.code == hb.ERR_UNSUPPORTED:
+            pytest.skip("no tensor-core kernel for this case")
+        raise
+    assert np.array_equal(P.cpu().numpy(), ref["P"])
+    assert hb.device_status() == 0
+
+
+def test_backward_data_uses_packed_forward_weights(hb):
+    """W is quantised ONCE into shared tiles; forward uses view c0 and backward-data view c1."""
+    t, batch, fin, fout = 24, 64, 200, 136
+    X = wl.draw("half_normal", (batch, fin), seed=31)
+    W = wl.draw("he_weight", (fin, fout), seed=32, fan_in=fin)
+    dY = wl.draw("grad", (batch, fout), seed=33)
+    fw = dict(mant_bits=8, block=t, tile=t, rounding=1, seed=1, stream_id=1)
+    fx = dict(mant_bits=8, block=t, rounding=1, seed=1, stream_id=0)
+    fg = dict(mant_bits=8, block=t, rounding=1, seed=1, stream_id=2)
+    c0, c1, _ = hb.quantize_tiles(to_dev(W), gfmt(fw))
+    Y = hb.gemm_q(batch, fout, fin, to_dev(X), c0, transA=0, fmtA=gfmt(fx), flags=hb.GEMM_FORCE_SIMT).cpu().numpy()
+    dX = hb.gemm_q(batch, fin, fout, to_dev(dY), c1, transA=0, fmtA=gfmt(fg), flags=hb.GEMM_FORCE_SIMT).cpu().numpy()
+    assert np.array_equal(Y, oracle.hbfp_gemm(0, 0, X, W, ofmt(fx), ofmt(fw))["c_seq"])
+    assert np.array_equal(dX, oracle.hbfp_gemm(0, 1, dY, W, ofmt(fg), ofmt(fw))["c_seq"])
+
+
+def test_argument_errors_are_reported_not_thrown_by_cuda(hb):
+    import torch
+    A = torch.zeros((64, 64), device="cuda")
+    f = hb.Format(8, 32)
+    with pytest.raises(hb.HbfpError) as e:
+        hb.gemm(0, 0, A, A, f, f, workspace=torch.empty(1024, dtype=torch.int8, device="cuda"))
+    assert e.value.code == hb.ERR_WORKSPACE
+    with pytest.raises(hb.HbfpError) as e:
+        hb.gemm(0, 0, A, A, f, hb.Format(8, 64))
+    assert e.value.code == hb.ERR_INVALID_ARG
+    with pytest.raises(hb.HbfpError) as e:
+        hb.quantize(A, 1, hb.Format(8, 32, rounding=5))
+    assert e.value.code == hb.ERR_INVALID_ARG
+    assert hb.device_status() == 0
+    C = hb.gemm(0, 0, A[:0], A, f, f)          # empty M
+    assert C.shape == (0, 64)
