@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the HBFP dot-product path on B200.
+
+A step is one pass of the whole hot path over one batch of synthetic input: quantise A,
+quantise B (FP32 -> block floating point), then the BFP GEMM, on the largest single-GPU
+configuration: the square GEMM of the large sweep, n = 16384, 8-bit mantissas, blocks of 128,
+round-to-nearest-even, log-normal inputs. The metric is effective TOPS of quantise+GEMM,
+2 n^3 / time. One JSON line is printed by rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--n 16384]
+                    [--mant-bits 8] [--block 128] [--rounding 0]
+
+With --gpus N > 1 (launched under torch.distributed.run) every rank runs an independent replica
+of the workload on its own GPU (the path has no exchange step); the value is the sum over ranks
+divided by the slowest rank's time. --impl reference times the CPU oracle, as it stands, on a
+bounded sub-cube of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "bfp_gemm_effective_tops_quantize_plus_gemm"
+UNIT = "TOPS"
+INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio (4.5 : 2.25 PFLOP/s)
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes of one launch of the GEMM kernel at the default workload, from the ncu capture
+# summarised under profiles/ (captured at n = 4096 and scaled). None = not captured.
+GEMM_DRAM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        for l in rows:
+            p = [x.strip() for x in l.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); smax.append(float(p[2])); power.append(float(p[3]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_desc(args) -> dict:
+    return {"workload": f"large-sweep square BFP GEMM n={args.n}: quantise A + quantise B + GEMM",
+            "M": args.n, "N": args.n, "K": args.n, "mant_bits": args.mant_bits, "block": args.block,
+            "rounding": "stochastic" if args.rounding else "nearest-even",
+            "inputs": "log-normal magnitudes (sigma 2), random signs, seed 3",
+            "l2": "inputs (2 x %.2f GiB FP32) are larger than the 126 MB L2; no flush" % (args.n * args.n * 4 / 2**30),
+            "parallelism": "independent replica per GPU"}
+
+
+# ------------------------------------------------------------------------------------ oracle arm
+
+def oracle_sample(n_full: int, mant_bits: int, block: int, rounding: int, budget_s: float = 15.0):
+    """Times the CPU oracle (quantise A, quantise B, BFP GEMM) on a sub-cube of the workload
+    sized to take about `budget_s` seconds. Returns (tops, cores, description, seconds, n_s)."""
+    import numpy as np
+    import oracle
+    from paper_1804_01526_b200 import workloads as wl
+
+    fa = oracle.Format(mant_bits, block, 0, rounding, 0, 3, 0)
+    fb = oracle.Format(mant_bits, block, 0, rounding, 0, 3, 1)
+
+    def run(ns):
+        A = wl.draw("lognormal", (ns, ns), seed=3, salt=0)
+        B = wl.draw("lognormal", (ns, ns), seed=3, salt=1)
+        t0 = time.perf_counter()
+        oracle.hbfp_gemm(0, 0, A, B, fa, fb)
+        return time.perf_counter() - t0
+
+    t_probe = run(256)
+    rate = 2 * 256 ** 3 / max(t_probe, 1e-6)
+    ns = 256
+    for cand in (512, 768, 1024, 1536, 2048, 3072, 4096):
+        if cand <= n_full and 2 * cand ** 3 / rate <= budget_s:
+            ns = cand
+    return ns, run
+
+
+def reference_arm(args):
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    ns, run = oracle_sample(args.n, args.mant_bits, args.block, args.rounding, budget_s=8.0)
+    for _ in range(args.warmup):
+        run(min(ns, 512))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run(ns)
+    dt = (time.perf_counter() - t0) / args.steps
+    tops = 2 * ns ** 3 / dt / 1e12
+    cores = oracle.num_threads()
+    sample = f"sub-cube A[:{ns},:{ns}] . B[:{ns},:{ns}] of the workload per step (quantise A, quantise B, BFP GEMM)"
+    out = {"impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "int64/f64 (oracle)", "data": "synthetic",
+           "config": workload_desc(args),
+           "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+           "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------------ GPU arm
+
+def gpu_arm(args):
+    import numpy as np
+    import torch
+    from paper_1804_01526_b200 import binding as hb, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    hb.lib()
+
+    n = args.n
+    fa = hb.Format(args.mant_bits, args.block, 0, args.rounding, 0, 3, 0)
+    fb = hb.Format(args.mant_bits, args.block, 0, args.rounding, 0, 3, 1)
+    A_h = torch.from_numpy(wl.draw("lognormal", (n, n), seed=3 + 1000 * rank, salt=0)).pin_memory()
+    B_h = torch.from_numpy(wl.draw("lognormal", (n, n), seed=3 + 1000 * rank, salt=1)).pin_memory()
+    A = A_h.cuda(non_blocking=True)
+    B = B_h.cuda(non_blocking=True)
+    C = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    C_h = torch.empty((n, n), dtype=torch.float32).pin_memory()
+    pa = hb.alloc_packed(n, n, fa)
+    pb = hb.alloc_packed(n, n, fb)
+    ws = torch.empty(max(hb.gemm_q_workspace(n, n, n, pa, pb), 1), dtype=torch.int8, device="cuda")
+    ws_full = torch.empty(max(hb.gemm_workspace(0, 0, n, n, n, fa, fb), 1), dtype=torch.int8, device="cuda")
+    torch.cuda.synchronize()
+
+    def step(events=None):
+        # the three launches hbfp_gemm makes, with events between them when asked for
+        if events is not None:
+            events[0].record()
+        hb.quantize(A, 1, fa, out=pa)
+        if events is not None:
+            events[1].record()
+        hb.quantize(B, 0, fb, out=pb)
+        if events is not None:
+            events[2].record()
+        hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
+        if events is not None:
+            events[3].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if hb.device_status() != 0:
+        raise RuntimeError("device status non-zero after warm-up")
+
+    # ---- timed region: exactly K steps, device time by CUDA events on the launching stream
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    barrier()
+    t_wall0 = time.time()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for k in range(args.steps):
+        step(evs[k])
+    end.record()
+    barrier()
+    t_wall1 = time.time()
+    clocks = sampler.stop(t_wall0, t_wall1)
+    total_ms = start.elapsed_time(end)
+    t_qa = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+    t_qb = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+    t_gemm = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    ops = 2.0 * n ** 3
+    value = world * ops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- the same step through hbfp_gemm with HOST buffers: H2D of A and B, D2H of C inside the timed region
+    e2e_steps = max(1, min(args.steps, 3))
+    def e2e_step():
+        A.copy_(A_h, non_blocking=True)
+        B.copy_(B_h, non_blocking=True)
+        hb.gemm(0, 0, A, B, fa, fb, out=C, workspace=ws_full)
+        C_h.copy_(C, non_blocking=True)
+    e2e_step()
+    barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e2.record()
+    barrier()
+    e2e_ms = s2.elapsed_time(e2) / e2e_steps
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_val = world * ops / (e2e_ms * 1e-3) / 1e12
+
+    status = hb.device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- standalone quantiser on the 1 GiB tensor (the second half of the metric), rank 0 only
+    quant = {}
+    if n * n * 4 >= 2 ** 30 or args.quantize_line:
+        for (m, b, r) in ((8, 32, 0), (8, 128, 0), (8, 32, 1), (12, 64, 1)):
+            f = hb.Format(m, b, 0, r, 0, 3, 0)
+            p = hb.alloc_packed(n, n, f)
+            for _ in range(3):
+                hb.quantize(A, 1, f, out=p)
+            torch.cuda.synchronize()
+            s3, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s3.record()
+            for _ in range(10):
+                hb.quantize(A, 1, f, out=p)
+            e3.record()
+            torch.cuda.synchronize()
+            ms = s3.elapsed_time(e3) / 10
+            nbytes = n * n * (4 + (1 if m <= 8 else 2) + 1.0 / b)
+            quant[f"m{m}_b{b}_{'sr' if r else 'rne'}"] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
+            del p
+
+    peaks, peaks_kind = load_peaks()
+    int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
+    int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
+    gemm_tops = ops / (t_gemm * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": int8_burst,
+                "unit": "TOP/s", "frac": gemm_tops / int8_burst, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
+                "peak_source": f"{peaks_kind} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
+                "frac_of_sustained_peak": gemm_tops / int8_sust, "frac_of_nominal_4500": gemm_tops / 4500.0,
+                "avg_launch_ms": t_gemm}
+    qbytes = n * n * (4 + (1 if args.mant_bits <= 8 else 2) + 1.0 / args.block)
+    breakdown = {"quantize_A_ms": t_qa, "quantize_B_ms": t_qb, "gemm_ms": t_gemm,
+                 "quantize_A_gbs": qbytes / (t_qa * 1e-3) / 1e9, "quantize_B_gbs": qbytes / (t_qb * 1e-3) / 1e9,
+                 "gemm_only_tops": gemm_tops, "hbm_peak_gbs": peaks["hbm_gbs"],
+                 "quantize_A_frac_of_hbm": qbytes / (t_qa * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                 "quantize_B_frac_of_hbm": qbytes / (t_qb * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+
+    # ---- CPU baseline: the oracle as it stands on a bounded sub-cube (about 10-20 s of CPU work)
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        ns, run = oracle_sample(n, args.mant_bits, args.block, args.rounding, budget_s=12.0)
+        dt = run(ns)
+        cpu = {"value": 2 * ns ** 3 / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"sub-cube A[:{ns},:{ns}] . B[:{ns},:{ns}] of the workload, one pass, {dt:.2f} s"}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "int8 mantissas, int32 block sums, f32 accumulate", "data": "synthetic",
+           "config": workload_desc(args), "clocks": clocks,
+           "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 2 * n * n * 4,
+                   "d2h_bytes_per_step": n * n * 4, "ms_per_step": e2e_ms, "steps": e2e_steps},
+           "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
+           "breakdown": breakdown, "quantize_standalone": quant}
+    print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n", type=int, default=16384)
+    ap.add_argument("--mant-bits", type=int, default=8)
+    ap.add_argument("--block", type=int, default=128)
+    ap.add_argument("--rounding", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quantize-line", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        return reference_arm(args)
+    return gpu_arm(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

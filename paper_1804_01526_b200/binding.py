@@ -14,7 +14,8 @@ from typing import Optional, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libhbfp.so")
+# HBFP_LIBRARY selects another build of the same library (e.g. one with debug checks).
+LIB_PATH = os.environ.get("HBFP_LIBRARY") or os.path.join(_HERE, "libhbfp.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
 GEMM_AUTO, GEMM_FORCE_SIMT, GEMM_FORCE_TENSOR = 0, 1, 2

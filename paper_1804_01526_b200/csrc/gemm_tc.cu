@@ -14,6 +14,15 @@
 // four MMAs per step into three accumulators (hi*hi, hi*lo + lo*hi, lo*lo) that the rescale warps
 // combine exactly in int32.
 //
+// Fast rescale (8-bit mantissas, blocks up to 256): the accumulator groups are pre-loaded with the
+// integer 0x4B400000 and every MMA accumulates, so that what tcgen05.ld returns, read as
+// binary32, is exactly 1.5*2^23 + P (|P| < 2^22). No integer-to-float conversion is needed:
+//   t   = fma(v, 2^sA, -1.5*2^23 * 2^sA)   = P * 2^sA          (exact)
+//   acc = fma(t, 2^sB, acc)                = acc + P*2^(sA+sB) (one rounding, as the definition)
+// both as packed two-wide FP32 FMAs; after reading a chunk the warp stores the bias back.
+// Other formats (12-bit planes, blocks longer than 256) clear the accumulator with the first
+// MMA of a block and convert with cvt.rn.f32.s32.
+//
 // Every wait on an mbarrier is bounded: when it expires the CTA records a code in the device
 // status word, raises a shared abort flag, drains its own copies and MMAs (bounded again),
 // releases tensor memory and returns.
@@ -24,12 +33,21 @@
 namespace hbfp {
 namespace {
 
+// Build-time probe for performance bisection (never set in the shipped library; results are
+// wrong when it is): 1 = rescale warps skip the tensor-memory reads and the math, 2 = no MMA is
+// issued, 4 = no mantissa tile is copied.
+#ifndef HBFP_TC_PROBE
+#define HBFP_TC_PROBE 0
+#endif
+
 constexpr int TILE_M = 128;
 constexpr int STAGE_K = 128;          // bytes of K per stage (= one 128B swizzle row)
 constexpr int RESCALE_WARPS = 8;
 constexpr int PRODUCER_WARP = 8;
 constexpr int MMA_WARP = 9;
-constexpr int THREADS = 320;
+constexpr int THREADS = 384;           // warps 10 and 11 only give their registers away
+constexpr uint32_t BIAS_BITS = 0x4B400000u;     // binary32 1.5 * 2^23
+constexpr int REGS_CONTROL = 40, REGS_RESCALE = 232;   // 128*40 + 256*232 <= 65536
 constexpr int TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
 
@@ -77,7 +95,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait. Returns false when the wait was abandoned (abort flag raised by anyone, or the
 // cycle budget ran out, in which case this thread raises the flag and records `code`).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             int32_t* status, int code, bool heed_abort) {
     const long long t0 = clock64();
     for (;;) {
@@ -139,6 +157,42 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&v)[32]) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+// 16-column variants used by the fast rescale path.
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Packed two-wide FP32 fused multiply-add (round to nearest even), operands as 64-bit pairs.
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled tile: 8-row groups 1024 bytes
@@ -173,27 +227,29 @@ struct Problem {
 
 struct Work {
     int m0, n0, split;
-    int64_t step0, step1;   // K=32 steps [step0, step1), step0 % 4 == 0
+    int step0, step1;       // K=32 steps [step0, step1), step0 % 4 == 0
 };
 
-__device__ __forceinline__ bool get_work(const Problem& p, int64_t w, Work* out) {
-    const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n;
+// 32-bit arithmetic only: this runs in warps that have given most of their registers away.
+__device__ __forceinline__ bool get_work(const Problem& p, int w, Work* out) {
+    const int tiles = p.tiles_m * p.tiles_n;
     if (w >= tiles * p.splits) return false;
-    const int split = (int)(w / tiles);
-    const int64_t t = w % tiles;
+    const int split = w / tiles;
+    const int t = w - split * tiles;
     // groups of 16 tile rows share their B panels in L2 while a group sweeps across N
     const int G = 16;
-    const int64_t per_group = (int64_t)G * p.tiles_n;
-    const int group = (int)(t / per_group);
+    const int per_group = G * p.tiles_n;
+    const int group = t / per_group;
     const int first_m = group * G;
     const int gsize = min(G, p.tiles_m - first_m);
-    const int64_t within = t % per_group;
-    out->m0 = (first_m + (int)(within % gsize)) * TILE_M;
-    out->n0 = (int)(within / gsize);
+    const int within = t - group * per_group;
+    const int nt = within / gsize;
+    out->m0 = (first_m + (within - nt * gsize)) * TILE_M;
+    out->n0 = nt;
     out->split = split;
     const int spb = p.bp / 32;
-    const int64_t kb0 = (int64_t)split * p.kb_per_split;
-    const int64_t kb1 = min(p.nkb, kb0 + p.kb_per_split);
+    const int kb0 = split * (int)p.kb_per_split;
+    const int kb1 = min((int)p.nkb, kb0 + (int)p.kb_per_split);
     out->step0 = kb0 * spb;
     out->step1 = kb1 * spb;
     return true;
@@ -201,7 +257,7 @@ __device__ __forceinline__ bool get_work(const Problem& p, int64_t w, Work* out)
 
 // ------------------------------------------------------------------------------ kernel
 
-template <int N_TILE, int PLANES>
+template <int N_TILE, int PLANES, bool MAGIC>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -210,6 +266,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     using C = Cfg<N_TILE, PLANES>;
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
     constexpr int COLS_PER_WARP = N_TILE / 2;          // each half of the rescale warps owns half the columns
+    static_assert(!(MAGIC && PLANES != 1), "the biased-accumulator path is for one-plane operands");
 
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -217,7 +274,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     const uint32_t mant_base = base;                                        // STAGES x MANT_STAGE, 1024-aligned
     const uint32_t exp_base = mant_base + STAGES * C::MANT_STAGE;           // STAGES x EXP_STAGE
     const uint32_t table_off = STAGES * (C::MANT_STAGE + C::EXP_STAGE);
-    int* tables = reinterpret_cast<int*>(base_ptr + table_off);             // [2][4][N_TILE]
+    uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [2][4][N_TILE]: bits of 2^sB (MAGIC) or sB << 23
     const uint32_t bar_off = table_off + C::TABLE_BYTES;
     const uint32_t bars = base + bar_off;
     const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
@@ -256,105 +313,127 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
 
     const int spb = p.bp / 32;                      // K=32 steps per block
 
-    if (warp == PRODUCER_WARP) {
-        // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            Work w;
-            for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-                const int n0 = w.n0 * N_TILE;
-                for (int64_t st0 = w.step0; st0 < w.step1; st0 += 4, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                    if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
-                    const uint32_t fb = full_bar + 8 * s;
-                    mbar_expect_tx(fb, C::TX_BYTES);
-                    const int kbyte = (int)(st0 * 32);
-                    const uint32_t ms = mant_base + s * C::MANT_STAGE;
-                    tma_load_2d(ms, &mapA0, kbyte, w.m0, fb);
-                    tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
-                    if (PLANES == 2) {
-                        tma_load_2d(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb);
-                        tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
+    if (warp >= RESCALE_WARPS) {
+        // the control warpgroup hands most of its registers to the rescale warps
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CONTROL));
+        if (warp == PRODUCER_WARP) {
+            // -------------------------------------------------------------- TMA producer
+            if (lane == 0) {
+                uint32_t it = 0;
+                bool ok = true;
+                Work w;
+                for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                    const int n0 = w.n0 * N_TILE;
+                    for (int st0 = w.step0; st0 < w.step1; st0 += 4, ++it) {
+                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                        if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
+                        const uint32_t fb = full_bar + 8 * s;
+                        mbar_expect_tx(fb, (HBFP_TC_PROBE & 4) ? (uint32_t)C::EXP_STAGE : C::TX_BYTES);
+                        const int kbyte = st0 * 32;
+                        const uint32_t ms = mant_base + s * C::MANT_STAGE;
+                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d(ms, &mapA0, kbyte, w.m0, fb);
+                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
+                        if (PLANES == 2 && !(HBFP_TC_PROBE & 4)) {
+                            tma_load_2d(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb);
+                            tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
+                        }
+                        const int kb = (st0 * 32) / p.bp;               // first block touched by this stage
+                        const uint32_t es = exp_base + s * C::EXP_STAGE;
+                        tma_load_2d(es, &mapEA, w.m0, kb, fb);
+                        tma_load_2d(es + C::EXP_A, &mapEB, n0, kb, fb);
                     }
-                    const int kb = (int)((st0 * 32) / p.bp);        // first block touched by this stage
-                    const uint32_t es = exp_base + s * C::EXP_STAGE;
-                    tma_load_2d(es, &mapEA, w.m0, kb, fb);
-                    tma_load_2d(es + C::EXP_A, &mapEB, n0, kb, fb);
                 }
+                // Drain: every issued copy must have landed before the CTA may exit. In a normal run
+                // the consumers already waited for all of them, so these return at once.
+                const uint32_t issued = it;
+                for (uint32_t k = issued > (uint32_t)STAGES ? issued - STAGES : 0; k < issued; ++k)
+                    mbar_wait(full_bar + 8 * (k % STAGES), (k / STAGES) & 1, abort_flag, p.status, 102, false);
             }
-            // Drain: every issued copy must have landed before the CTA may exit. In a normal run
-            // the consumers already waited for all of them, so these return at once.
-            const uint32_t issued = it;
-            for (uint32_t k = issued > (uint32_t)STAGES ? issued - STAGES : 0; k < issued; ++k)
-                mbar_wait(full_bar + 8 * (k % STAGES), (k / STAGES) & 1, abort_flag, p.status, 102, false);
-        }
-    } else if (warp == MMA_WARP) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_i8<N_TILE>();
-            uint32_t it = 0, blk = 0;
-            bool ok = true;
-            Work w;
-            for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-                for (int64_t st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                    if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 201)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t ms = mant_base + s * C::MANT_STAGE;
-                    const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
-                    const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
-                    const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
-                    for (int j = 0; j < 4; ++j) {
-                        const int64_t step = st0 + j;
-                        if (step >= w.step1) break;
-                        const int pos = (int)(step % spb);
-                        const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
-                        if (pos == 0) {
-                            if (!mbar_wait(tempty_bar + 8 * g, gph ^ 1, abort_flag, p.status, 202)) { ok = false; break; }
-                            tc_fence_after();
+        } else if (warp == MMA_WARP) {
+            // -------------------------------------------------------------- MMA issuer
+            if (lane == 0) {
+                constexpr uint32_t idesc = idesc_i8<N_TILE>();
+                uint32_t it = 0, blk = 0;
+                bool ok = true;
+                Work w;
+                for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                    for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
+                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                        if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 201)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t ms = mant_base + s * C::MANT_STAGE;
+                        const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
+                        const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
+                        const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
+                        for (int j = 0; j < 4; ++j) {
+                            const int step = st0 + j;
+                            if (step >= w.step1) break;
+                            const int pos = step % spb;
+                            const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
+                            if (pos == 0) {
+                                // the group was read (and, on the biased path, re-biased) by all rescale warps
+                                if (!mbar_wait(tempty_bar + 8 * g, gph, abort_flag, p.status, 202)) { ok = false; break; }
+                                tc_fence_after();
+                            }
+                            const uint32_t d = tmem_base + g * PARTS * N_TILE;
+                            const uint64_t ko = (uint64_t)(2 * j);          // 32 bytes per step, in 16-byte units
+                            const uint32_t acc = MAGIC ? 1u : (uint32_t)(pos != 0);
+                            if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
+                            if (PLANES == 2 && !(HBFP_TC_PROBE & 2)) {
+                                tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
+                                tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc, 1u);
+                                tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_lo + ko, idesc, acc);
+                            }
+                            if (pos == spb - 1) {
+                                tc_commit(tfull_bar + 8 * g);
+                                ++blk;
+                            }
                         }
-                        const uint32_t d = tmem_base + g * PARTS * N_TILE;
-                        const uint64_t ko = (uint64_t)(2 * j);          // 32 bytes per step, in 16-byte units
-                        const uint32_t acc = pos != 0;
-                        tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
-                        if (PLANES == 2) {
-                            tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
-                            tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc, 1u);
-                            tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_lo + ko, idesc, acc);
-                        }
-                        if (pos == spb - 1) {
-                            tc_commit(tfull_bar + 8 * g);
-                            ++blk;
-                        }
+                        tc_commit(empty_bar + 8 * s);        // the stage is free once these MMAs have read it
                     }
-                    tc_commit(empty_bar + 8 * s);        // the stage is free once these MMAs have read it
                 }
+                tc_commit(done_bar);
+                mbar_wait(done_bar, 0, abort_flag, p.status, 203, false);
             }
-            tc_commit(done_bar);
-            mbar_wait(done_bar, 0, abort_flag, p.status, 203, false);
         }
     } else {
         // ------------------------------------------------------------------ rescale warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
         const int quarter = warp & 3, half = warp >> 2;
         const int row = quarter * 32 + lane;                 // row of the tile = tensor-memory lane
         const int col0 = half * COLS_PER_WARP;
         const int tid_half = threadIdx.x & 127;
-        float acc[COLS_PER_WARP];
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
+        uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
+        uint32_t bias[16];
+        if (MAGIC) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) bias[i] = BIAS_BITS;
+            for (int g = 0; g < GROUPS; ++g)
+#pragma unroll
+                for (int ch = 0; ch < COLS_PER_WARP / 16; ++ch) tc_st16(lane_addr + g * N_TILE + ch * 16, bias);
+            tc_wait_st();
+        }
+        // every accumulator group starts out free
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0)
+            for (int g = 0; g < GROUPS; ++g) mbar_arrive(tempty_bar + 8 * g);
+
         uint32_t it = 0, blk = 0, ev = 0;
         bool ok = true;
         Work w;
-        for (int64_t wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+        for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
             const int n0 = w.n0 * N_TILE;
 #pragma unroll
-            for (int c = 0; c < COLS_PER_WARP; ++c) acc[c] = 0.f;
-            int sa_bits[4] = {0, 0, 0, 0};
+            for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
+            uint32_t sa_bits[4] = {0, 0, 0, 0};
             uint32_t tab_ev = 0;
-            for (int64_t st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
+            for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
                 const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                 if (!mbar_wait_warp(full_bar + 8 * s, ph, abort_flag, p.status, 301)) { ok = false; break; }
                 // blocks that start in this stage: build their column tables and fetch this row's exponent
-                const int first_pos = (int)(st0 % spb);
+                const int first_pos = st0 % spb;
                 const bool has_start = spb <= 4 || first_pos == 0;
                 if (has_start) {
                     const int8_t* eA = reinterpret_cast<const int8_t*>(base_ptr + (exp_base - base) + s * C::EXP_STAGE);
@@ -362,9 +441,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     const int nb = spb >= 4 ? 1 : 4 / spb;           // blocks per stage
                     tab_ev = ev & 1;
                     for (int jb = 0; jb < nb; ++jb) {
-                        sa_bits[jb] = ((int)eA[jb * TILE_M + row] + 127) << 23;
-                        for (int c = tid_half; c < COLS_PER_WARP; c += 128)
-                            tables[(tab_ev * 4 + jb) * N_TILE + col0 + c] = (int)eB[jb * N_TILE + col0 + c] << 23;
+                        sa_bits[jb] = (uint32_t)((int)eA[jb * TILE_M + row] + 127) << 23;      // bits of 2^sA
+                        for (int c = tid_half; c < COLS_PER_WARP; c += 128) {
+                            const int sb = (int)eB[jb * N_TILE + col0 + c];
+                            tables[(tab_ev * 4 + jb) * N_TILE + col0 + c] = MAGIC ? (uint32_t)(sb + 127) << 23 : (uint32_t)(sb << 23);
+                        }
                     }
                     // the four warps of this half publish their table entries to each other
                     __syncwarp();
@@ -376,48 +457,87 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 if (lane == 0) mbar_arrive(empty_bar + 8 * s);       // exponent slices of the stage are consumed
                 // blocks that end in this stage
                 for (int j = 0; j < 4; ++j) {
-                    const int64_t step = st0 + j;
+                    const int step = st0 + j;
                     if (step >= w.step1) break;
-                    if ((int)(step % spb) != spb - 1) continue;
+                    if (step % spb != spb - 1) continue;
                     const int jb = spb >= 4 ? 0 : j / spb;
                     const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
                     if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + g * PARTS * N_TILE + col0;
-                    const int* tab = tables + (tab_ev * 4 + jb) * N_TILE + col0;
-                    const int sa = sa_bits[jb];
-                    const int64_t kb = step / spb;
+                    const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
+                    const uint32_t* tab = tables + (tab_ev * 4 + jb) * N_TILE + col0;
+                    const int kb = step / spb;
+                    const int64_t gi = w.m0 + row;
+                    if (HBFP_TC_PROBE & 1) {
+                    } else if (MAGIC) {
+                        // v = 1.5*2^23 + P as binary32;  t = (v - 1.5*2^23) * 2^sA exactly;  acc += t * 2^sB
+                        const float sa_f = __uint_as_float(sa_bits[jb]);
+                        const float ca_f = -12582912.0f * sa_f;
+                        const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
+                        const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
+                        constexpr int NCH = COLS_PER_WARP / 16;
+                        uint32_t v[2][16];
+                        tc_ld16(taddr, v[0]);
 #pragma unroll
-                    for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
-                        int v[32];
-                        tc_ld32(taddr + ch * 32, v);
-                        if (PLANES == 2) {
-                            int mid[32], ll[32];
-                            tc_ld32(taddr + N_TILE + ch * 32, mid);
-                            tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
+                        for (int ch = 0; ch < NCH; ++ch) {
                             tc_wait_ld();
+                            if (ch + 1 < NCH) tc_ld16(taddr + (ch + 1) * 16, v[(ch + 1) & 1]);
+                            const uint32_t(&x)[16] = v[ch & 1];
+                            if (p.P != nullptr && gi < p.M) {
 #pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
-                        } else {
-                            tc_wait_ld();
+                                for (int c = 0; c < 16; ++c) {
+                                    const int64_t gj = n0 + col0 + ch * 16 + c;
+                                    if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)(x[c] - BIAS_BITS);
+                                }
+                            }
+#pragma unroll
+                            for (int q = 0; q < 16; q += 4) {
+                                const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 16 + q);
+                                const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
+                                const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
+                                acc2[(ch * 16 + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * 16 + q) / 2]);
+                                acc2[(ch * 16 + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * 16 + q) / 2 + 1]);
+                            }
+                            tc_st16(taddr + ch * 16, bias);          // re-arm the accumulator for its next block
                         }
-                        if (p.P != nullptr) {
-                            const int64_t gi = w.m0 + row;
-                            if (gi < p.M)
+                        tc_wait_st();
+                    } else {
+                        const int sa = (int)sa_bits[jb];
+#pragma unroll
+                        for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
+                            int v[32];
+                            tc_ld32(taddr + ch * 32, v);
+                            if (PLANES == 2) {
+                                int mid[32], ll[32];
+                                tc_ld32(taddr + N_TILE + ch * 32, mid);
+                                tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
+                            } else {
+                                tc_wait_ld();
+                            }
+                            if (p.P != nullptr && gi < p.M) {
 #pragma unroll
                                 for (int c = 0; c < 32; ++c) {
                                     const int64_t gj = n0 + col0 + ch * 32 + c;
                                     if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = v[c];
                                 }
-                        }
+                            }
 #pragma unroll
-                        for (int c4 = 0; c4 < 32; c4 += 4) {
-                            const int4 sb = *reinterpret_cast<const int4*>(tab + ch * 32 + c4);
-                            acc[ch * 32 + c4 + 0] = fmaf((float)v[c4 + 0], __int_as_float(sa + sb.x), acc[ch * 32 + c4 + 0]);
-                            acc[ch * 32 + c4 + 1] = fmaf((float)v[c4 + 1], __int_as_float(sa + sb.y), acc[ch * 32 + c4 + 1]);
-                            acc[ch * 32 + c4 + 2] = fmaf((float)v[c4 + 2], __int_as_float(sa + sb.z), acc[ch * 32 + c4 + 2]);
-                            acc[ch * 32 + c4 + 3] = fmaf((float)v[c4 + 3], __int_as_float(sa + sb.w), acc[ch * 32 + c4 + 3]);
+                            for (int c4 = 0; c4 < 32; c4 += 4) {
+                                const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 32 + c4);
+                                float a0, a1, a2, a3;
+                                unpack2(acc2[(ch * 32 + c4) / 2], a0, a1);
+                                unpack2(acc2[(ch * 32 + c4) / 2 + 1], a2, a3);
+                                a0 = fmaf((float)v[c4 + 0], __int_as_float(sa + (int)sb.x), a0);
+                                a1 = fmaf((float)v[c4 + 1], __int_as_float(sa + (int)sb.y), a1);
+                                a2 = fmaf((float)v[c4 + 2], __int_as_float(sa + (int)sb.z), a2);
+                                a3 = fmaf((float)v[c4 + 3], __int_as_float(sa + (int)sb.w), a3);
+                                acc2[(ch * 32 + c4) / 2] = pack2(__float_as_uint(a0), __float_as_uint(a1));
+                                acc2[(ch * 32 + c4) / 2 + 1] = pack2(__float_as_uint(a2), __float_as_uint(a3));
+                            }
                         }
                     }
                     tc_fence_before();
@@ -437,10 +557,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 for (int c = 0; c < COLS_PER_WARP; c += 4) {
                     const int64_t gj = n0 + col0 + c;
                     if (gj + 3 < p.N) {
-                        *reinterpret_cast<float4*>(rowp + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
+                        *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
                     } else {
+                        float e4[4];
+                        unpack2(acc2[c / 2], e4[0], e4[1]);
+                        unpack2(acc2[c / 2 + 1], e4[2], e4[3]);
+#pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            if (gj + e < p.N) rowp[c + e] = acc[c + e];
+                            if (gj + e < p.N) rowp[c + e] = e4[e];
                     }
                 }
             }
@@ -510,7 +634,7 @@ int sm_count() {
     return n;
 }
 
-template <int N_TILE, int PLANES>
+template <int N_TILE, int PLANES, bool MAGIC>
 int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t st) {
     using C = Cfg<N_TILE, PLANES>;
     CUtensorMap mA0, mA1, mB0, mB1, mEA, mEB;
@@ -533,12 +657,12 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
     if (rc) return rc;
     static bool attr_set = false;
     if (!attr_set) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         attr_set = true;
     }
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     const int grid = (int)(work < sm_count() ? work : sm_count());
-    gemm_tc_kernel<N_TILE, PLANES><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
+    gemm_tc_kernel<N_TILE, PLANES, MAGIC><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
     return launch_status();
 }
 
@@ -609,10 +733,13 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     if (!p.status) return HBFP_ERR_CUDA;
     if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
     int rc;
-    if (a.L.planes == 2) rc = launch_cfg<64, 2>(p, a, b, st);
-    else if (plan.n_tile == 256) rc = launch_cfg<256, 1>(p, a, b, st);
-    else if (plan.n_tile == 128) rc = launch_cfg<128, 1>(p, a, b, st);
-    else rc = launch_cfg<64, 1>(p, a, b, st);
+    // the biased-accumulator path needs every |P| < 2^22
+    const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
+    const bool magic = a.L.planes == 1 && qa * qb * a.L.b < (1ll << 22);
+    if (a.L.planes == 2) rc = launch_cfg<64, 2, false>(p, a, b, st);
+    else if (plan.n_tile == 256) rc = magic ? launch_cfg<256, 1, true>(p, a, b, st) : launch_cfg<256, 1, false>(p, a, b, st);
+    else if (plan.n_tile == 128) rc = magic ? launch_cfg<128, 1, true>(p, a, b, st) : launch_cfg<128, 1, false>(p, a, b, st);
+    else rc = magic ? launch_cfg<64, 1, true>(p, a, b, st) : launch_cfg<64, 1, false>(p, a, b, st);
     if (rc) return rc;
     if (p.splits > 1) {
         const int64_t n = M * N;
