@@ -2,11 +2,13 @@
 // tensor memory -> per-block rescale into FP32 registers (Eq. 2 per block, blocks accumulated in
 // floating point, Sec. 4).
 //
-// One persistent CTA per SM, 10 warps:
-//   warps 0-7  rescale: tcgen05.ld the int32 block sums, convert, scale by 2^(sA+sB), accumulate
-//              in FP32 registers (128 rows x N_TILE columns per tile), store C
-//   warp 8     TMA producer: mantissa tiles (128B-swizzled, K-major) and exponent slices
-//   warp 9     MMA issuer (one thread) and owner of the tensor-memory allocation
+// One persistent CTA per SM, 12 warps (the control warps come first: the issue logic favours low
+// warp ids, and a starved MMA issuer stalls everything):
+//   warp 0     TMA producer: mantissa tiles (128B-swizzled, K-major) and exponent slices
+//   warp 1     MMA issuer (one thread) and owner of the tensor-memory allocation
+//   warp 2     scale-table builder: turns the int8 exponent slices of each block into 2^sA / 2^sB
+//   warps 4-11 rescale: tcgen05.ld the int32 block sums, scale by 2^(sA+sB), accumulate in FP32
+//              registers (128 rows x N_TILE columns per tile), store C
 // A stage is 128 bytes of K for every row of the A (128 rows) and B (N_TILE rows) tiles, i.e. four
 // K=32 MMA steps; a K-block of bp bytes is bp/32 consecutive steps accumulated into one fresh
 // int32 accumulator group in tensor memory. Groups form a ring, so the MMA of the next block
@@ -14,19 +16,21 @@
 // four MMAs per step into three accumulators (hi*hi, hi*lo + lo*hi, lo*lo) that the rescale warps
 // combine exactly in int32.
 //
-// Fast rescale (8-bit mantissas, blocks up to 256): the accumulator groups are pre-loaded with the
-// integer 0x4B400000 and every MMA accumulates, so that what tcgen05.ld returns, read as
-// binary32, is exactly 1.5*2^23 + P (|P| < 2^22). No integer-to-float conversion is needed:
+// Fast rescale (8-bit mantissas, blocks up to 256, so |P| < 2^22): integer-to-float conversion
+// runs on a slow pipe and an integer add per element would land on the FP32 pipe, so the
+// accumulator groups are armed with the integer 0x4B400000 and every MMA accumulates on top of it:
+// what tcgen05.ld returns, read as binary32, is exactly 1.5*2^23 + P. Then
 //   t   = fma(v, 2^sA, -1.5*2^23 * 2^sA)   = P * 2^sA          (exact)
 //   acc = fma(t, 2^sB, acc)                = acc + P*2^(sA+sB) (one rounding, as the definition)
 // both as packed two-wide FP32 FMAs; after reading a chunk the warp stores the bias back.
-// Other formats (12-bit planes, blocks longer than 256) clear the accumulator with the first
-// MMA of a block and convert with cvt.rn.f32.s32.
+// Other formats (12-bit planes, longer blocks) clear the accumulator with the first MMA of a
+// block and convert with cvt.rn.f32.s32.
 //
 // Every wait on an mbarrier is bounded: when it expires the CTA records a code in the device
 // status word, raises a shared abort flag, drains its own copies and MMAs (bounded again),
 // releases tensor memory and returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "common.cuh"
 
@@ -40,16 +44,37 @@ namespace {
 #define HBFP_TC_PROBE 0
 #endif
 
+// 1: poll barriers with the non-suspending test_wait instead of try_wait.
+#ifndef HBFP_TC_TESTWAIT
+#define HBFP_TC_TESTWAIT 0
+#endif
+
+// 1: packed two-wide FP32 FMAs in the rescale; 0: scalar FMAs.
+#ifndef HBFP_TC_FFMA2
+#define HBFP_TC_FFMA2 1
+#endif
+
 constexpr int TILE_M = 128;
 constexpr int STAGE_K = 128;          // bytes of K per stage (= one 128B swizzle row)
 constexpr int RESCALE_WARPS = 8;
-constexpr int PRODUCER_WARP = 8;
-constexpr int MMA_WARP = 9;
+// The control warps take the lowest warp ids: the issue logic favours them over the rescale
+// warps of the same sub-partition, and a starved MMA issuer stalls the whole pipeline.
+constexpr int CONTROL_WARPS = 4;      // one warpgroup: producer, MMA issuer, table builder, one spare
+constexpr int PRODUCER_WARP = 0;
+constexpr int MMA_WARP = 1;
+constexpr int TABLE_WARP = 2;
 constexpr int THREADS = 384;           // warps 10 and 11 only give their registers away
 constexpr uint32_t BIAS_BITS = 0x4B400000u;     // binary32 1.5 * 2^23
-constexpr int REGS_CONTROL = 40, REGS_RESCALE = 232;   // 128*40 + 256*232 <= 65536
+#ifndef HBFP_TC_REGS_RESCALE
+#define HBFP_TC_REGS_RESCALE 208
+#endif
+#ifndef HBFP_TC_CHUNK
+#define HBFP_TC_CHUNK 16          // columns per tensor-memory load in the fast rescale path (16 or 32)
+#endif
+constexpr int REGS_RESCALE = HBFP_TC_REGS_RESCALE, REGS_CONTROL = (64512 - 256 * REGS_RESCALE) / 128;   // 128*88 + 256*208 = 64512 = 384*168: never ask for more than the launch allocation
 constexpr int TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
+constexpr uint32_t WAIT_HINT_NS = 200000u;              // one try_wait may sleep this long; the loop around it is bounded
 
 template <int N_TILE, int PLANES>
 struct Cfg {
@@ -61,7 +86,10 @@ struct Cfg {
     static constexpr int MANT_STAGE = PLANES * (A_BYTES + B_BYTES);
     static constexpr int EXP_A = 4 * TILE_M, EXP_B = 4 * N_TILE;
     static constexpr int EXP_STAGE = EXP_A + EXP_B;
-    static constexpr int TABLE_BYTES = 2 * 4 * N_TILE * 4;        // [event parity][block in stage][column]
+    // scale tables: a ring of TABLE_SLOTS blocks, each [N_TILE column scales][128 row scales], 32-bit
+    static constexpr int TABLE_SLOTS = 4;
+    static constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
+    static constexpr int TABLE_BYTES = 4 * TABLE_SLOTS * TABLE_SLOT_WORDS;
     static constexpr int STAGES_RAW = (232448 - 2048 - TABLE_BYTES) / (MANT_STAGE + EXP_STAGE);
     static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
     static constexpr int SMEM = 1024 /*align slack*/ + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024 /*barriers*/;
@@ -87,9 +115,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#if HBFP_TC_TESTWAIT
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#else
+        // the suspend-time hint lets a waiting thread sleep in hardware until the phase completes
+        // instead of spinning on issue slots that the arithmetic warps of its sub-partition need
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
     return ok != 0;
 }
 
@@ -157,6 +191,23 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, int (&v)[32]) {
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
 // 16-column variants used by the fast rescale path.
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
@@ -193,6 +244,9 @@ __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
     hi = __uint_as_float(b);
 }
 
+__device__ __forceinline__ void tc_ldn(uint32_t taddr, uint32_t (&v)[32]) { tc_ld32(taddr, v); }
+__device__ __forceinline__ void tc_ldn(uint32_t taddr, uint32_t (&v)[16]) { tc_ld16(taddr, v); }
+
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major, 128B-swizzled tile: 8-row groups 1024 bytes
@@ -223,10 +277,21 @@ struct Problem {
     int64_t ldp;
     int32_t* P;             // optional dump of block sums [M][N][nkb]
     int32_t* status;
+    long long* trace;       // probe builds only: per-role timestamps of CTA 0
 };
+
+#if HBFP_TC_PROBE & 8
+#define HBFP_TRACE(role, idx)                                                        \
+    do {                                                                              \
+        if (p.trace && blockIdx.x == 0 && (idx) < 512) p.trace[(role) * 512 + (idx)] = clock64(); \
+    } while (0)
+#else
+#define HBFP_TRACE(role, idx) do { } while (0)
+#endif
 
 struct Work {
     int m0, n0, split;
+    int kb0;                // first K-block of this item
     int step0, step1;       // K=32 steps [step0, step1), step0 % 4 == 0
 };
 
@@ -250,6 +315,7 @@ __device__ __forceinline__ bool get_work(const Problem& p, int w, Work* out) {
     const int spb = p.bp / 32;
     const int kb0 = split * (int)p.kb_per_split;
     const int kb1 = min((int)p.nkb, kb0 + (int)p.kb_per_split);
+    out->kb0 = kb0;
     out->step0 = kb0 * spb;
     out->step1 = kb1 * spb;
     return true;
@@ -257,7 +323,7 @@ __device__ __forceinline__ bool get_work(const Problem& p, int w, Work* out) {
 
 // ------------------------------------------------------------------------------ kernel
 
-template <int N_TILE, int PLANES, bool MAGIC>
+template <int N_TILE, int PLANES, bool MAGIC, bool DUMP>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -274,14 +340,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     const uint32_t mant_base = base;                                        // STAGES x MANT_STAGE, 1024-aligned
     const uint32_t exp_base = mant_base + STAGES * C::MANT_STAGE;           // STAGES x EXP_STAGE
     const uint32_t table_off = STAGES * (C::MANT_STAGE + C::EXP_STAGE);
-    uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [2][4][N_TILE]: bits of 2^sB (MAGIC) or sB << 23
+    uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [slot][N_TILE column scales | 128 row scales]
+    constexpr int TSLOTS = C::TABLE_SLOTS;
     const uint32_t bar_off = table_off + C::TABLE_BYTES;
     const uint32_t bars = base + bar_off;
     const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
     const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 8 * GROUPS;
     const uint32_t done_bar = tempty_bar + 8 * GROUPS;
-    const uint32_t tbl_bar = done_bar + 8;                 // one per half of the rescale warps
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + 16 * STAGES + 16 * GROUPS + 24);
+    const uint32_t tready_bar = done_bar + 8;              // table slot written (by the table warp)
+    const uint32_t tfree_bar = tready_bar + 8 * TSLOTS;    // table slot read by all rescale warps
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + 16 * STAGES + 16 * GROUPS + 8 + 16 * TSLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -289,15 +357,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, 1 + RESCALE_WARPS);
+            mbar_init(empty_bar + 8 * s, 2);                 // MMA commit + table warp
         }
         for (int g = 0; g < GROUPS; ++g) {
             mbar_init(tfull_bar + 8 * g, 1);
             mbar_init(tempty_bar + 8 * g, RESCALE_WARPS);
         }
         mbar_init(done_bar, 1);
-        mbar_init(tbl_bar, RESCALE_WARPS / 2);
-        mbar_init(tbl_bar + 8, RESCALE_WARPS / 2);
+        for (int i = 0; i < TSLOTS; ++i) {
+            mbar_init(tready_bar + 8 * i, 1);
+            mbar_init(tfree_bar + 8 * i, RESCALE_WARPS);
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -313,7 +383,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
 
     const int spb = p.bp / 32;                      // K=32 steps per block
 
-    if (warp >= RESCALE_WARPS) {
+    if (warp < CONTROL_WARPS) {
         // the control warpgroup hands most of its registers to the rescale warps
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CONTROL));
         if (warp == PRODUCER_WARP) {
@@ -324,9 +394,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 Work w;
                 for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
                     const int n0 = w.n0 * N_TILE;
+                    int pos = 0, kb = w.kb0;          // position inside the current block, its index
                     for (int st0 = w.step0; st0 < w.step1; st0 += 4, ++it) {
                         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                         if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
+                        HBFP_TRACE(0, it);
                         const uint32_t fb = full_bar + 8 * s;
                         mbar_expect_tx(fb, (HBFP_TC_PROBE & 4) ? (uint32_t)C::EXP_STAGE : C::TX_BYTES);
                         const int kbyte = st0 * 32;
@@ -337,10 +409,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                             tma_load_2d(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb);
                             tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
                         }
-                        const int kb = (st0 * 32) / p.bp;               // first block touched by this stage
                         const uint32_t es = exp_base + s * C::EXP_STAGE;
-                        tma_load_2d(es, &mapEA, w.m0, kb, fb);
+                        tma_load_2d(es, &mapEA, w.m0, kb, fb);          // kb = first block touched by this stage
                         tma_load_2d(es + C::EXP_A, &mapEB, n0, kb, fb);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (pos == spb - 1) { pos = 0; ++kb; } else { ++pos; }
+                        }
                     }
                 }
                 // Drain: every issued copy must have landed before the CTA may exit. In a normal run
@@ -357,27 +432,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 bool ok = true;
                 Work w;
                 for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                    int pos = 0;
                     for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
                         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
                         if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 201)) { ok = false; break; }
+                        HBFP_TRACE(2, it);
                         tc_fence_after();
                         const uint32_t ms = mant_base + s * C::MANT_STAGE;
                         const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
                         const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
                         const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
                         for (int j = 0; j < 4; ++j) {
-                            const int step = st0 + j;
-                            if (step >= w.step1) break;
-                            const int pos = step % spb;
+                            if (st0 + j >= w.step1) break;
                             const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
                             if (pos == 0) {
                                 // the group was read (and, on the biased path, re-biased) by all rescale warps
                                 if (!mbar_wait(tempty_bar + 8 * g, gph, abort_flag, p.status, 202)) { ok = false; break; }
+                                HBFP_TRACE(3, blk);
                                 tc_fence_after();
                             }
                             const uint32_t d = tmem_base + g * PARTS * N_TILE;
                             const uint64_t ko = (uint64_t)(2 * j);          // 32 bytes per step, in 16-byte units
-                            const uint32_t acc = MAGIC ? 1u : (uint32_t)(pos != 0);
+                            const uint32_t acc = MAGIC ? 1u : (uint32_t)(pos != 0);   // biased path: accumulate on top of the bias
                             if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
                             if (PLANES == 2 && !(HBFP_TC_PROBE & 2)) {
                                 tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
@@ -387,170 +463,211 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                             if (pos == spb - 1) {
                                 tc_commit(tfull_bar + 8 * g);
                                 ++blk;
+                                pos = 0;
+                            } else {
+                                ++pos;
                             }
                         }
                         tc_commit(empty_bar + 8 * s);        // the stage is free once these MMAs have read it
+                        HBFP_TRACE(4, it);
                     }
                 }
                 tc_commit(done_bar);
                 mbar_wait(done_bar, 0, abort_flag, p.status, 203, false);
             }
+        } else if (warp == TABLE_WARP) {
+            // -------------------------------------------------------------- scale-table builder
+            uint32_t it = 0, blk = 0;
+            bool ok = true;
+            Work w;
+            for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
+                int pos = 0;
+                for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
+                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                    if (!mbar_wait_warp(full_bar + 8 * s, ph, abort_flag, p.status, 401)) { ok = false; break; }
+                    const int8_t* eA = reinterpret_cast<const int8_t*>(base_ptr + (exp_base - base) + s * C::EXP_STAGE);
+                    const int8_t* eB = eA + C::EXP_A;
+                    int jb = 0;                    // row of the exponent slices: blocks that start in this stage
+                    for (int j = 0; j < 4; ++j) {
+                        if (st0 + j >= w.step1) break;
+                        if (pos == 0) {
+                            const uint32_t slot = blk % TSLOTS, sph = (blk / TSLOTS) & 1;
+                            if (!mbar_wait_warp(tfree_bar + 8 * slot, sph, abort_flag, p.status, 402)) { ok = false; break; }
+                            uint32_t* tb = tables + slot * C::TABLE_SLOT_WORDS;
+                            for (int c = lane; c < N_TILE; c += 32) {
+                                const int sb = (int)eB[jb * N_TILE + c];
+                                tb[c] = MAGIC ? (uint32_t)(sb + 127) << 23 : (uint32_t)(sb << 23);
+                            }
+                            for (int r = lane; r < TILE_M; r += 32)
+                                tb[N_TILE + r] = (uint32_t)((int)eA[jb * TILE_M + r] + 127) << 23;
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(tready_bar + 8 * slot);
+                            ++blk;
+                            ++jb;
+                        }
+                        pos = pos == spb - 1 ? 0 : pos + 1;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar + 8 * s);      // the exponent slices are consumed
+                }
+            }
         }
     } else {
         // ------------------------------------------------------------------ rescale warps
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
-        const int quarter = warp & 3, half = warp >> 2;
+        const int rwarp = warp - CONTROL_WARPS;              // 0..7
+        const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4
         const int row = quarter * 32 + lane;                 // row of the tile = tensor-memory lane
         const int col0 = half * COLS_PER_WARP;
-        const int tid_half = threadIdx.x & 127;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
-        uint32_t bias[16];
+#if !HBFP_TC_FFMA2
+        float accf[MAGIC ? COLS_PER_WARP : 1];
+#endif
+        uint32_t bias[8];
         if (MAGIC) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) bias[i] = BIAS_BITS;
+            for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
             for (int g = 0; g < GROUPS; ++g)
 #pragma unroll
-                for (int ch = 0; ch < COLS_PER_WARP / 16; ++ch) tc_st16(lane_addr + g * N_TILE + ch * 16, bias);
+                for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
             tc_wait_st();
         }
-        // every accumulator group starts out free
+        // every accumulator group and every table slot starts out free
         tc_fence_before();
         __syncwarp();
-        if (lane == 0)
+        if (lane == 0) {
             for (int g = 0; g < GROUPS; ++g) mbar_arrive(tempty_bar + 8 * g);
+            for (int i = 0; i < TSLOTS; ++i) mbar_arrive(tfree_bar + 8 * i);
+        }
 
-        uint32_t it = 0, blk = 0, ev = 0;
+        uint32_t blk = 0;
         bool ok = true;
         Work w;
         for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
             const int n0 = w.n0 * N_TILE;
+            const int64_t gi = w.m0 + row;
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
-            uint32_t sa_bits[4] = {0, 0, 0, 0};
-            uint32_t tab_ev = 0;
-            for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
-                const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                if (!mbar_wait_warp(full_bar + 8 * s, ph, abort_flag, p.status, 301)) { ok = false; break; }
-                // blocks that start in this stage: build their column tables and fetch this row's exponent
-                const int first_pos = st0 % spb;
-                const bool has_start = spb <= 4 || first_pos == 0;
-                if (has_start) {
-                    const int8_t* eA = reinterpret_cast<const int8_t*>(base_ptr + (exp_base - base) + s * C::EXP_STAGE);
-                    const int8_t* eB = eA + C::EXP_A;
-                    const int nb = spb >= 4 ? 1 : 4 / spb;           // blocks per stage
-                    tab_ev = ev & 1;
-                    for (int jb = 0; jb < nb; ++jb) {
-                        sa_bits[jb] = (uint32_t)((int)eA[jb * TILE_M + row] + 127) << 23;      // bits of 2^sA
-                        for (int c = tid_half; c < COLS_PER_WARP; c += 128) {
-                            const int sb = (int)eB[jb * N_TILE + col0 + c];
-                            tables[(tab_ev * 4 + jb) * N_TILE + col0 + c] = MAGIC ? (uint32_t)(sb + 127) << 23 : (uint32_t)(sb << 23);
-                        }
-                    }
-                    // the four warps of this half publish their table entries to each other
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tbl_bar + 8 * half);
-                    if (!mbar_wait_warp(tbl_bar + 8 * half, ev & 1, abort_flag, p.status, 303)) { ok = false; break; }
-                    ++ev;
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar + 8 * s);       // exponent slices of the stage are consumed
-                // blocks that end in this stage
-                for (int j = 0; j < 4; ++j) {
-                    const int step = st0 + j;
-                    if (step >= w.step1) break;
-                    if (step % spb != spb - 1) continue;
-                    const int jb = spb >= 4 ? 0 : j / spb;
-                    const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
-                    if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
-                    const uint32_t* tab = tables + (tab_ev * 4 + jb) * N_TILE + col0;
-                    const int kb = step / spb;
-                    const int64_t gi = w.m0 + row;
-                    if (HBFP_TC_PROBE & 1) {
-                    } else if (MAGIC) {
-                        // v = 1.5*2^23 + P as binary32;  t = (v - 1.5*2^23) * 2^sA exactly;  acc += t * 2^sB
-                        const float sa_f = __uint_as_float(sa_bits[jb]);
-                        const float ca_f = -12582912.0f * sa_f;
-                        const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
-                        const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
-                        constexpr int NCH = COLS_PER_WARP / 16;
-                        uint32_t v[2][16];
-                        tc_ld16(taddr, v[0]);
+#if !HBFP_TC_FFMA2
+            if (MAGIC) {
 #pragma unroll
-                        for (int ch = 0; ch < NCH; ++ch) {
+                for (int c = 0; c < COLS_PER_WARP; ++c) accf[c] = 0.f;
+            }
+#endif
+            const int nblk = (w.step1 - w.step0) / spb;      // (once per tile; spb divides the range)
+            for (int kb = w.kb0; kb < w.kb0 + nblk; ++kb, ++blk) {
+                const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
+                const uint32_t slot = blk % TSLOTS, sph = (blk / TSLOTS) & 1;
+                if (!mbar_wait_warp(tready_bar + 8 * slot, sph, abort_flag, p.status, 303)) { ok = false; break; }
+                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
+                if (threadIdx.x == CONTROL_WARPS * 32) HBFP_TRACE(7, blk);
+                if (lane == 0) HBFP_TRACE(17 + rwarp, blk);
+                tc_fence_after();
+                const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
+                const uint32_t* tab = tables + slot * C::TABLE_SLOT_WORDS + col0;
+                const uint32_t sa_u = tables[slot * C::TABLE_SLOT_WORDS + N_TILE + row];
+                if (HBFP_TC_PROBE & 1) {
+                } else if (MAGIC) {
+                    // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
+                    // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
+                    const float sa_f = __uint_as_float(sa_u);
+                    const float ca_f = -12582912.0f * sa_f;
+                    const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
+                    const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
+                    constexpr int CH = HBFP_TC_CHUNK;
+                    constexpr int NCHK = COLS_PER_WARP / CH;
+                    uint32_t v[2][CH];
+                    tc_ldn(taddr, v[0]);
+#pragma unroll
+                    for (int ch = 0; ch < NCHK; ++ch) {
+                        tc_wait_ld();
+                        if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & 1]);
+                        const uint32_t(&x)[CH] = v[ch & 1];
+                        if (DUMP && p.P != nullptr && gi < p.M) {
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) {
+                                const int64_t gj = n0 + col0 + ch * CH + c;
+                                if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)(x[c] - BIAS_BITS);
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < CH; q += 4) {
+                            const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CH + q);
+#if HBFP_TC_FFMA2
+                            const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
+                            const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
+                            acc2[(ch * CH + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
+                            acc2[(ch * CH + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CH + q) / 2 + 1]);
+#else
+                            accf[ch * CH + q + 0] = fmaf(fmaf(__uint_as_float(x[q + 0]), sa_f, ca_f), __uint_as_float(sb.x), accf[ch * CH + q + 0]);
+                            accf[ch * CH + q + 1] = fmaf(fmaf(__uint_as_float(x[q + 1]), sa_f, ca_f), __uint_as_float(sb.y), accf[ch * CH + q + 1]);
+                            accf[ch * CH + q + 2] = fmaf(fmaf(__uint_as_float(x[q + 2]), sa_f, ca_f), __uint_as_float(sb.z), accf[ch * CH + q + 2]);
+                            accf[ch * CH + q + 3] = fmaf(fmaf(__uint_as_float(x[q + 3]), sa_f, ca_f), __uint_as_float(sb.w), accf[ch * CH + q + 3]);
+#endif
+                        }
+#pragma unroll
+                        for (int c8 = 0; c8 < CH / 8; ++c8) tc_st8(taddr + ch * CH + c8 * 8, bias);   // re-arm
+                    }
+                    tc_wait_st();
+                } else {
+                    const int sa = (int)sa_u;
+#pragma unroll
+                    for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
+                        int v[32];
+                        tc_ld32(taddr + ch * 32, v);
+                        if (PLANES == 2) {
+                            int mid[32], ll[32];
+                            tc_ld32(taddr + N_TILE + ch * 32, mid);
+                            tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
                             tc_wait_ld();
-                            if (ch + 1 < NCH) tc_ld16(taddr + (ch + 1) * 16, v[(ch + 1) & 1]);
-                            const uint32_t(&x)[16] = v[ch & 1];
-                            if (p.P != nullptr && gi < p.M) {
 #pragma unroll
-                                for (int c = 0; c < 16; ++c) {
-                                    const int64_t gj = n0 + col0 + ch * 16 + c;
-                                    if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)(x[c] - BIAS_BITS);
-                                }
-                            }
-#pragma unroll
-                            for (int q = 0; q < 16; q += 4) {
-                                const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 16 + q);
-                                const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
-                                const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
-                                acc2[(ch * 16 + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * 16 + q) / 2]);
-                                acc2[(ch * 16 + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * 16 + q) / 2 + 1]);
-                            }
-                            tc_st16(taddr + ch * 16, bias);          // re-arm the accumulator for its next block
+                            for (int c = 0; c < 32; ++c)
+                                v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
+                        } else {
+                            tc_wait_ld();
                         }
-                        tc_wait_st();
-                    } else {
-                        const int sa = (int)sa_bits[jb];
+                        if (DUMP && p.P != nullptr && gi < p.M) {
 #pragma unroll
-                        for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
-                            int v[32];
-                            tc_ld32(taddr + ch * 32, v);
-                            if (PLANES == 2) {
-                                int mid[32], ll[32];
-                                tc_ld32(taddr + N_TILE + ch * 32, mid);
-                                tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
-                                tc_wait_ld();
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
-                            } else {
-                                tc_wait_ld();
+                            for (int c = 0; c < 32; ++c) {
+                                const int64_t gj = n0 + col0 + ch * 32 + c;
+                                if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = v[c];
                             }
-                            if (p.P != nullptr && gi < p.M) {
+                        }
 #pragma unroll
-                                for (int c = 0; c < 32; ++c) {
-                                    const int64_t gj = n0 + col0 + ch * 32 + c;
-                                    if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = v[c];
-                                }
-                            }
-#pragma unroll
-                            for (int c4 = 0; c4 < 32; c4 += 4) {
-                                const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 32 + c4);
-                                float a0, a1, a2, a3;
-                                unpack2(acc2[(ch * 32 + c4) / 2], a0, a1);
-                                unpack2(acc2[(ch * 32 + c4) / 2 + 1], a2, a3);
-                                a0 = fmaf((float)v[c4 + 0], __int_as_float(sa + (int)sb.x), a0);
-                                a1 = fmaf((float)v[c4 + 1], __int_as_float(sa + (int)sb.y), a1);
-                                a2 = fmaf((float)v[c4 + 2], __int_as_float(sa + (int)sb.z), a2);
-                                a3 = fmaf((float)v[c4 + 3], __int_as_float(sa + (int)sb.w), a3);
-                                acc2[(ch * 32 + c4) / 2] = pack2(__float_as_uint(a0), __float_as_uint(a1));
-                                acc2[(ch * 32 + c4) / 2 + 1] = pack2(__float_as_uint(a2), __float_as_uint(a3));
-                            }
+                        for (int c4 = 0; c4 < 32; c4 += 4) {
+                            const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 32 + c4);
+                            float a0, a1, a2, a3;
+                            unpack2(acc2[(ch * 32 + c4) / 2], a0, a1);
+                            unpack2(acc2[(ch * 32 + c4) / 2 + 1], a2, a3);
+                            a0 = fmaf((float)v[c4 + 0], __int_as_float(sa + (int)sb.x), a0);
+                            a1 = fmaf((float)v[c4 + 1], __int_as_float(sa + (int)sb.y), a1);
+                            a2 = fmaf((float)v[c4 + 2], __int_as_float(sa + (int)sb.z), a2);
+                            a3 = fmaf((float)v[c4 + 3], __int_as_float(sa + (int)sb.w), a3);
+                            acc2[(ch * 32 + c4) / 2] = pack2(__float_as_uint(a0), __float_as_uint(a1));
+                            acc2[(ch * 32 + c4) / 2 + 1] = pack2(__float_as_uint(a2), __float_as_uint(a3));
                         }
                     }
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(tempty_bar + 8 * g);
-                    ++blk;
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(tempty_bar + 8 * g);
+                    mbar_arrive(tfree_bar + 8 * slot);
+                }
+                if (threadIdx.x == CONTROL_WARPS * 32) HBFP_TRACE(8, blk);
+                if (lane == 0) HBFP_TRACE(9 + rwarp, blk);
             }
             if (!ok) break;
+#if !HBFP_TC_FFMA2
+            if (MAGIC) {
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = pack2(__float_as_uint(accf[2 * c]), __float_as_uint(accf[2 * c + 1]));
+            }
+#endif
             // ---- store the tile (or this split's partial tile)
             float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
             const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
-            const int64_t gi = w.m0 + row;
             if (dst != nullptr && gi < p.M) {
                 float* rowp = dst + gi * ldd + n0 + col0;
 #pragma unroll
@@ -634,7 +751,7 @@ int sm_count() {
     return n;
 }
 
-template <int N_TILE, int PLANES, bool MAGIC>
+template <int N_TILE, int PLANES, bool MAGIC, bool DUMP>
 int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t st) {
     using C = Cfg<N_TILE, PLANES>;
     CUtensorMap mA0, mA1, mB0, mB1, mEA, mEB;
@@ -657,16 +774,21 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
     if (rc) return rc;
     static bool attr_set = false;
     if (!attr_set) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         attr_set = true;
     }
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     const int grid = (int)(work < sm_count() ? work : sm_count());
-    gemm_tc_kernel<N_TILE, PLANES, MAGIC><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
+    gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
     return launch_status();
 }
 
 }  // namespace
+
+#if HBFP_TC_PROBE & 8
+long long* g_probe_trace = nullptr;
+extern "C" __attribute__((visibility("default"))) void hbfp_probe_set_trace(long long* ptr) { g_probe_trace = ptr; }
+#endif
 
 TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, const Layout& lb, int mant_bits_a,
                             int mant_bits_b) {
@@ -687,6 +809,9 @@ TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, c
         n_tile = 256;
         while (n_tile > 64 && (tiles_m * ((N + n_tile - 1) / n_tile) < SMS || N <= n_tile / 2)) n_tile /= 2;
     }
+#if HBFP_TC_PROBE
+    if (const char* e = getenv("HBFP_TC_NTILE")) n_tile = atoi(e);
+#endif
     const int64_t tiles = tiles_m * ((N + n_tile - 1) / n_tile);
     // split-K for small outputs with a long contraction: at least two stages per split, split
     // boundaries on stage boundaries.
@@ -730,16 +855,23 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     p.ldp = round_up(N, 4);
     p.P = P;
     p.status = device_status_word();
+#if HBFP_TC_PROBE & 8
+    p.trace = g_probe_trace;
+#endif
     if (!p.status) return HBFP_ERR_CUDA;
     if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
     int rc;
     // the biased-accumulator path needs every |P| < 2^22
     const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
     const bool magic = a.L.planes == 1 && qa * qb * a.L.b < (1ll << 22);
-    if (a.L.planes == 2) rc = launch_cfg<64, 2, false>(p, a, b, st);
-    else if (plan.n_tile == 256) rc = magic ? launch_cfg<256, 1, true>(p, a, b, st) : launch_cfg<256, 1, false>(p, a, b, st);
-    else if (plan.n_tile == 128) rc = magic ? launch_cfg<128, 1, true>(p, a, b, st) : launch_cfg<128, 1, false>(p, a, b, st);
-    else rc = magic ? launch_cfg<64, 1, true>(p, a, b, st) : launch_cfg<64, 1, false>(p, a, b, st);
+    if (P) {   // the inspection build of the kernel: 64-column tiles, writes the block sums
+        p.tiles_n = (int)((N + 63) / 64);
+        if (a.L.planes == 2) rc = launch_cfg<64, 2, false, true>(p, a, b, st);
+        else rc = magic ? launch_cfg<64, 1, true, true>(p, a, b, st) : launch_cfg<64, 1, false, true>(p, a, b, st);
+    } else if (a.L.planes == 2) rc = launch_cfg<64, 2, false, false>(p, a, b, st);
+    else if (plan.n_tile == 256) rc = magic ? launch_cfg<256, 1, true, false>(p, a, b, st) : launch_cfg<256, 1, false, false>(p, a, b, st);
+    else if (plan.n_tile == 128) rc = magic ? launch_cfg<128, 1, true, false>(p, a, b, st) : launch_cfg<128, 1, false, false>(p, a, b, st);
+    else rc = magic ? launch_cfg<64, 1, true, false>(p, a, b, st) : launch_cfg<64, 1, false, false>(p, a, b, st);
     if (rc) return rc;
     if (p.splits > 1) {
         const int64_t n = M * N;
