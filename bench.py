@@ -7,7 +7,7 @@ configuration: the square GEMM of the large sweep, n = 16384, 8-bit mantissas, b
 round-to-nearest-even, log-normal inputs. The metric is effective TOPS of quantise+GEMM,
 2 n^3 / time. One JSON line is printed by rank 0.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--n 16384]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--size 16384]
                     [--mant-bits 8] [--block 128] [--rounding 0]
 
 With --gpus N > 1 (launched under torch.distributed.run) every rank runs an independent replica
@@ -167,16 +167,12 @@ def reference_arm(args):
 def gpu_arm(args):
     import numpy as np
     import torch
-    from paper_1804_01526_b200 import binding as hb, workloads as wl
+    from paper_1804_01526_b200 import binding as hb, replicas, workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rep = replicas.init("nccl" if int(os.environ.get("WORLD_SIZE", "1")) > 1 else None, torch.device("cuda", local))
+    world, rank = rep.world, rep.rank
     hb.lib()
 
     n = args.n
@@ -209,8 +205,7 @@ def gpu_arm(args):
             events[3].record()
 
     def barrier():
-        if dist is not None:
-            dist.barrier()
+        replicas.barrier(rep)
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -238,13 +233,10 @@ def gpu_arm(args):
     t_qa = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
     t_qb = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
     t_gemm = statistics.mean(e[2].elapsed_time(e[3]) for e in evs)
-    if world > 1:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = replicas.max_over_ranks(rep, total_ms, "cuda")
     ms_per_step = total_ms / args.steps
     ops = 2.0 * n ** 3
-    value = world * ops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.aggregate_throughput(rep, ops, ms_per_step * 1e-3) / 1e12
 
     # ---- the same step through hbfp_gemm with HOST buffers: H2D of A and B, D2H of C inside the timed region
     e2e_steps = max(1, min(args.steps, 3))
@@ -262,18 +254,14 @@ def gpu_arm(args):
     e2.record()
     barrier()
     e2e_ms = s2.elapsed_time(e2) / e2e_steps
-    if world > 1:
-        tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_val = world * ops / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = replicas.max_over_ranks(rep, e2e_ms, "cuda")
+    e2e_val = replicas.aggregate_throughput(rep, ops, e2e_ms * 1e-3) / 1e12
 
     status = hb.device_status()
     if status != 0:
         raise RuntimeError(f"device status {status}")
     if rank != 0:
-        if dist is not None:
-            dist.destroy_process_group()
+        replicas.shutdown(rep)
         return 0
 
     # ---- standalone quantiser on the 1 GiB tensor (the second half of the metric), rank 0 only
@@ -330,8 +318,7 @@ def gpu_arm(args):
            "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
            "breakdown": breakdown, "quantize_standalone": quant}
     print(json.dumps(out), flush=True)
-    if dist is not None:
-        dist.destroy_process_group()
+    replicas.shutdown(rep)
     return 0
 
 
@@ -341,7 +328,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--n", type=int, default=16384)
+    ap.add_argument("--size", dest="n", type=int, default=16384, help="n of the square GEMM")
     ap.add_argument("--mant-bits", type=int, default=8)
     ap.add_argument("--block", type=int, default=128)
     ap.add_argument("--rounding", type=int, default=0)
