@@ -68,7 +68,8 @@ typedef enum hbfp_status {
     HBFP_ERR_ALIGNMENT = 3,   /* a packed buffer or C is not aligned as documented           */
     HBFP_ERR_WORKSPACE = 4,   /* workspace pointer null or smaller than the query returned   */
     HBFP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor map, ...)  */
-    HBFP_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (see hbfp_device_status) */
+    HBFP_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (see hbfp_device_status) */
+    HBFP_ERR_STATIC_LIMIT = 7 /* hbfp_gemm_static: the problem needs more than the built-in scratch */
 } hbfp_status;
 
 #define HBFP_ROUND_NEAREST_EVEN 0
@@ -181,6 +182,30 @@ HBFP_API int hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K, 
                        int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                        const hbfp_format* fmtA, const hbfp_format* fmtB, void* workspace,
                        size_t workspace_bytes, uint32_t flags, void* stream);
+
+/* Built-in scratch of hbfp_gemm_static, in bytes. */
+#define HBFP_STATIC_WORKSPACE_BYTES (16u << 20)
+
+/* hbfp_gemm for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a property of the library, not of the method). Who they are: code that runs inside another
+ * program's memory discipline - a plug-in whose host framework has taken the whole device for
+ * its own pool, so that a cudaMalloc from the plug-in fails; a serving or real-time loop in which
+ * an allocation is forbidden because it may synchronise the device and stall every stream.
+ * Same arguments and result as hbfp_gemm, minus the workspace: the packed operands and the split-K
+ * partial tiles live in a fixed HBFP_STATIC_WORKSPACE_BYTES array in device memory that belongs to
+ * the library (every GPU that loads the library holds it until the process exits). The call
+ * allocates and frees nothing. Problems whose hbfp_gemm_workspace() exceeds the array are
+ * rejected with HBFP_ERR_STATIC_LIMIT and nothing is launched (at 8-bit mantissas roughly
+ * M*K + N*K <= 15 million elements, e.g. every GEMM of the 784-1024-1024-10 MLP at batch 128).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call outside any stream capture. All calls share the one
+ * array and it keeps the previous call's contents: nothing in it needs clearing between calls,
+ * but two calls that overlap on the GPU (different streams, or a captured graph replayed
+ * concurrently) race on it - run them on one stream or order them yourself. */
+HBFP_API int hbfp_gemm_static(int transA, int transB, int64_t M, int64_t N, int64_t K, const float* A,
+                              int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
+                              const hbfp_format* fmtA, const hbfp_format* fmtB, uint32_t flags,
+                              void* stream);
 
 /* Same product with each operand either FP32 (quantised by the call) or already packed: the
  * steady state of training, where W is quantised once per step into shared tiles and used by

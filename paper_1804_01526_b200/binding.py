@@ -17,7 +17,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 # HBFP_LIBRARY selects another build of the same library (e.g. one with debug checks).
 LIB_PATH = os.environ.get("HBFP_LIBRARY") or os.path.join(_HERE, "libhbfp.so")
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(7)
+(OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT,
+ ERR_STATIC_LIMIT) = range(8)
+STATIC_WORKSPACE_BYTES = 16 << 20
 GEMM_AUTO, GEMM_FORCE_SIMT, GEMM_FORCE_TENSOR = 0, 1, 2
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 
@@ -25,7 +27,7 @@ EXPORTS = [
     "hbfp_status_string", "hbfp_packed_layout", "hbfp_packed_sizes", "hbfp_quantize",
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
-    "hbfp_device_status",
+    "hbfp_device_status", "hbfp_gemm_static",
 ]
 
 
@@ -93,6 +95,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_gemm_q_workspace.argtypes = [i64, i64, i64, p, p, p]
         L.hbfp_gemm.argtypes = [i32, i32, i64, i64, i64, p, i64, p, i64, p, i64, p, p, p, sz, u32, p]
         L.hbfp_gemm_q.argtypes = [i64, i64, i64, p, p, p, i64, p, sz, u32, p]
+        L.hbfp_gemm_static.argtypes = [i32, i32, i64, i64, i64, p, i64, p, i64, p, i64, p, p, u32, p]
         L.hbfp_gemm_block_partials.argtypes = [i64, i64, i64, p, p, p, u32, p]
         L.hbfp_device_status.argtypes = [p, p]
         for name in EXPORTS[1:]:
@@ -242,6 +245,23 @@ def gemm(transA: int, transB: int, A: torch.Tensor, B: torch.Tensor, fmtA: Forma
     _check(lib().hbfp_gemm(transA, transB, M, N, K, _dptr(A), _ld(A), _dptr(B), _ld(B), _dptr(out), _ld(out),
                            ctypes.byref(fa), ctypes.byref(fb), _dptr(workspace), workspace.numel(), flags,
                            _stream()), "hbfp_gemm")
+    return out
+
+
+def gemm_static(transA: int, transB: int, A: torch.Tensor, B: torch.Tensor, fmtA: Format, fmtB: Format,
+                out: Optional[torch.Tensor] = None, flags: int = GEMM_AUTO) -> torch.Tensor:
+    """hbfp_gemm_static: hbfp_gemm on the library's built-in scratch, for callers that cannot
+    allocate device memory. Pass ``out`` if the output, too, must come from memory you already
+    own; problems larger than the built-in scratch raise ``HbfpError`` (ERR_STATIC_LIMIT)."""
+    _check_f32(A, "A")
+    _check_f32(B, "B")
+    M, N, K = _gemm_dims(transA, transB, A, B)
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    fa, fb = fmtA.c(), fmtB.c()
+    _check(lib().hbfp_gemm_static(transA, transB, M, N, K, _dptr(A), _ld(A), _dptr(B), _ld(B), _dptr(out),
+                                  _ld(out), ctypes.byref(fa), ctypes.byref(fb), flags, _stream()),
+           "hbfp_gemm_static")
     return out
 
 

@@ -149,6 +149,7 @@ const char* hbfp_status_string(int status) {
         case HBFP_ERR_WORKSPACE: return "workspace missing or too small";
         case HBFP_ERR_CUDA: return "CUDA call failed";
         case HBFP_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case HBFP_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of hbfp_gemm_static";
         default: return "unknown status";
     }
 }
