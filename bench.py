@@ -34,9 +34,9 @@ METRIC = "bfp_gemm_effective_tops_quantize_plus_gemm"
 UNIT = "TOPS"
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes of one launch of the GEMM kernel at the default workload, from the ncu capture
-# summarised under profiles/ (captured at n = 4096 and scaled). None = not captured.
-GEMM_DRAM_TRAFFIC_BYTES = None
+# DRAM bytes (read + write) of one launch of the GEMM kernel at the default workload (n = 16384, m = 8,
+# b = 128), from the single-pass ncu capture summarised in profiles/bench_launch_list_n16384_m8_b128.md.
+GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 4046596608 + 1107060480}
 
 
 def load_peaks():
@@ -289,7 +289,9 @@ def gpu_arm(args):
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
     gemm_tops = ops / (t_gemm * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": int8_burst,
-                "unit": "TOP/s", "frac": gemm_tops / int8_burst, "traffic": GEMM_DRAM_TRAFFIC_BYTES,
+                "unit": "TOP/s", "frac": gemm_tops / int8_burst,
+                "traffic": GEMM_DRAM_TRAFFIC_BYTES.get((n, args.mant_bits, args.block)),
+                "algorithmic_bytes": 2 * n * n * ((1 if args.mant_bits <= 8 else 2) + 1.0 / args.block) + 4 * n * n,
                 "peak_source": f"{peaks_kind} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
                 "frac_of_sustained_peak": gemm_tops / int8_sust, "frac_of_nominal_4500": gemm_tops / 4500.0,
                 "avg_launch_ms": t_gemm}

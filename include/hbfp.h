@@ -176,8 +176,9 @@ HBFP_API int hbfp_gemm_q_workspace(int64_t M, int64_t N, int64_t K, const hbfp_o
  * forward Y = X W is (0,0); backward-data dX = dY W^T is (0,1); backward-weight dW = X^T dY is
  * (1,0). Without split-K the blocks are accumulated in ascending order with one FP32 rounding
  * each; with split-K (chosen for small C and long K) each split does so and the splits are
- * summed in ascending order. The exact range of the scaled FP32 accumulation needs
- * sA + sB in [-126, 127], sA <= 110 (|A| < 2^117) for 8-bit mantissas. */
+ * summed in ascending order. Exactness of the scaled FP32 accumulation needs sA + sB in
+ * [-126, 127] (else the true product is outside binary32) and, on the tensor-core path,
+ * sA <= 103 (|A| < 2^110 at 8-bit mantissas). */
 HBFP_API int hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K, const float* A,
                        int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                        const hbfp_format* fmtA, const hbfp_format* fmtB, void* workspace,
