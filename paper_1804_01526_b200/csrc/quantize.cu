@@ -7,9 +7,9 @@
 //                    thread (two 128-bit loads, one Philox call in stochastic mode), block
 //                    max by warp shuffles, exponents staged in shared memory so that the
 //                    [kb][row] exponent array is written in full 32-byte sectors.
-//   quant_col_fast   blocks down the columns, b <= 128: a b x 128 FP32 panel is read with
-//                    coalesced row loads into shared memory, reduced down the columns and
-//                    written transposed, so the output is contraction-major again.
+//   quant_col_fast   blocks down the columns, b <= 128: a (<=128) x 32 FP32 panel is read with
+//                    coalesced row loads into shared memory, reduced down the columns by four
+//                    threads per column and written transposed (contraction-major again).
 //   quant_tiles      t x t weight tiles (t <= 128): one pass writes both packed views and
 //                    the tile exponent grid.
 //   exps_* / mant_generic   two-pass path for every other geometry (any b, any alignment).
@@ -187,85 +187,104 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
 // ------------------------------------------------------------------------------ quant_col_fast
 
 // Blocks down the columns of x [K][R] (contract axis 0); output rows are the columns of x.
-// CTA: 128 threads, one block of b <= 128 k-rows by 128 columns.
-constexpr int COLT = 128;
+// CTA: 128 threads = 32 columns x 4 row slots; panel = G blocks of b <= 128 k-rows (G*b <= 128)
+// by 32 columns: 16 KB of shared memory, so a dozen CTAs fit an SM and cover the memory latency.
+constexpr int COLT = 32;
 
 template <int PLANES>
 __global__ void __launch_bounds__(128)
-quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, int b, int bp, QParams p,
+quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, int b, int bp, int G, QParams p,
                int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
                int8_t* __restrict__ exps, int64_t rs, int64_t nkb, int vec_ok) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* tile = reinterpret_cast<float*>(smem_raw);                 // [b][COLT]
-    uint4* rnd = reinterpret_cast<uint4*>(tile + (size_t)b * COLT);   // [b][COLT/8] (stochastic only)
+    const int krows = G * b;
+    float* tile = reinterpret_cast<float*>(smem_raw);                      // [krows][COLT]
+    uint32_t* pmax = reinterpret_cast<uint32_t*>(tile + (size_t)krows * COLT);   // [G][4][COLT]
+    uint4* rnd = reinterpret_cast<uint4*>(pmax + (size_t)G * 4 * COLT);    // [krows][COLT/8] (stochastic only)
 
-    const int tid = threadIdx.x;
-    const int64_t kb = blockIdx.y;
+    const int tid = threadIdx.x, c = tid & 31, q = tid >> 5;
+    const int64_t kb0 = (int64_t)blockIdx.y * G;
     const int64_t c0 = (int64_t)blockIdx.x * COLT;
-    const int64_t k0 = kb * b;
-    const int blen = (int)min((int64_t)b, K - k0);
+    const int64_t k0 = kb0 * b;
+    const int rows_here = (int)min((int64_t)krows, K - k0);
 
     // 1. coalesced load of the panel (zero beyond the matrix).
     if (vec_ok) {
-        for (int i = tid; i < blen * (COLT / 4); i += 128) {
-            const int kk = i / (COLT / 4), c4 = (i % (COLT / 4)) * 4;
+        for (int i = tid; i < rows_here * (COLT / 4); i += 128) {
+            const int kk = i >> 3, c4 = (i & 7) * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c0 + c4 < R) v = __ldcs(reinterpret_cast<const float4*>(x + (k0 + kk) * ld + c0 + c4));
-            *reinterpret_cast<float4*>(tile + kk * COLT + c4) = v;      // R % 4 == 0 on this path
+            if (c0 + c4 < R) v = __ldcs(reinterpret_cast<const float4*>(x + (k0 + kk) * ld + c0 + c4));   // R % 4 == 0 here
+            *reinterpret_cast<float4*>(tile + kk * COLT + c4) = v;
         }
     } else {
-        for (int i = tid; i < blen * COLT; i += 128) {
-            const int kk = i / COLT, c = i % COLT;
-            tile[kk * COLT + c] = (c0 + c < R) ? x[(k0 + kk) * ld + c0 + c] : 0.f;
+        for (int i = tid; i < rows_here * COLT; i += 128) {
+            const int kk = i >> 5, cc = i & 31;
+            tile[kk * COLT + cc] = (c0 + cc < R) ? x[(k0 + kk) * ld + c0 + cc] : 0.f;
         }
     }
     // 2. stochastic mode: one Philox call per 8 consecutive source elements of a row.
-    const bool group_ok = (R % 8) == 0;     // then L = k*R + c has L & 7 == c & 7 and groups align
+    const bool group_ok = (R % 8) == 0;     // then L = k*R + col has L & 7 == col & 7 and groups align
     if (p.rounding == 1 && group_ok) {
-        for (int i = tid; i < blen * (COLT / 8); i += 128) {
-            const int kk = i / (COLT / 8), g8 = i % (COLT / 8);
+        for (int i = tid; i < rows_here * (COLT / 8); i += 128) {
+            const int kk = i >> 2, g8 = i & 3;
             const uint64_t L = (uint64_t)((k0 + kk) * R + c0 + g8 * 8);
-            rnd[kk * (COLT / 8) + g8] = draws_of_group(p, L >> 3);
+            rnd[i] = draws_of_group(p, L >> 3);
         }
     }
     __syncthreads();
 
-    // 3. thread = column: max down the block, exponent, mantissas, transposed store.
-    const int64_t c = c0 + tid;
-    uint32_t am = 0;
-    for (int kk = 0; kk < blen; ++kk) am = max(am, abs_bits(tile[kk * COLT + tid]));
-    const int s = block_exponent(am, p.m, p.exp_mode);
-    if (c < R) {
-        exps[kb * rs + c] = (int8_t)s;
-        int8_t* dst = mant + c * kst + kb * bp;
-        const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
-        for (int w0 = 0; w0 < bp; w0 += 16) {
-            uint32_t hi[4] = {0, 0, 0, 0}, lo[4] = {0, 0, 0, 0};
+    // 3. thread (q, c): quarter q of every block of column c. Partial maxima first.
+    const int rq = bp / 4;                  // padded rows per thread and block: 8, 16 or 32
+    for (int g = 0; g < G; ++g) {
+        uint32_t am = 0;
+        const int r0 = g * b + q * rq;
+        for (int j = 0; j < rq; ++j) {
+            const int kk = r0 + j;
+            if (q * rq + j < b && kk < rows_here) am = max(am, abs_bits(tile[kk * COLT + c]));
+        }
+        pmax[(g * 4 + q) * COLT + c] = am;
+    }
+    __syncthreads();
+
+    const int64_t col = c0 + c;
+    const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
+    for (int g = 0; g < G; ++g) {
+        const int64_t kb = kb0 + g;
+        if (kb >= nkb) break;
+        const uint32_t am = max(max(pmax[(g * 4 + 0) * COLT + c], pmax[(g * 4 + 1) * COLT + c]),
+                                max(pmax[(g * 4 + 2) * COLT + c], pmax[(g * 4 + 3) * COLT + c]));
+        const int s = block_exponent(am, p.m, p.exp_mode);
+        if (col >= R) continue;
+        if (q == 0) exps[kb * rs + col] = (int8_t)s;
+        int8_t* dst = mant + col * kst + kb * bp + q * rq;
+        const int r0 = g * b + q * rq;
+        for (int w0 = 0; w0 < rq; w0 += 8) {
+            uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int kk = w0 + j;
-                int q = 0;
-                if (kk < blen) {
-                    const float v = tile[kk * COLT + tid];
-                    if (p.rounding == 0) q = round_rne(v, s, p.qmax);
-                    else if (group_ok) q = round_sr(v, s, p.qmax, rnd16[(kk * (COLT / 8) + (tid >> 3)) * 8 + (tid & 7)]);
-                    else q = round_sr(v, s, p.qmax, draw_of_element(p, (uint64_t)((k0 + kk) * R + c)));
+            for (int j = 0; j < 8; ++j) {
+                const int kk = r0 + w0 + j;
+                int qv = 0;
+                if (q * rq + w0 + j < b && kk < rows_here) {
+                    const float v = tile[kk * COLT + c];
+                    if (p.rounding == 0) qv = round_rne(v, s, p.qmax);
+                    else if (group_ok) qv = round_sr(v, s, p.qmax, rnd16[(kk * (COLT / 8) + (c >> 3)) * 8 + (c & 7)]);
+                    else qv = round_sr(v, s, p.qmax, draw_of_element(p, (uint64_t)((k0 + kk) * R + col)));
                 }
                 if (PLANES == 1) {
-                    hi[j >> 2] |= (uint32_t)(q & 0xff) << (8 * (j & 3));
+                    hi[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
                 } else {
-                    hi[j >> 2] |= (uint32_t)((q >> 4) & 0xff) << (8 * (j & 3));
-                    lo[j >> 2] |= (uint32_t)(q & 15) << (8 * (j & 3));
+                    hi[j >> 2] |= (uint32_t)((qv >> 4) & 0xff) << (8 * (j & 3));
+                    lo[j >> 2] |= (uint32_t)(qv & 15) << (8 * (j & 3));
                 }
             }
-            *reinterpret_cast<uint4*>(dst + w0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            if (PLANES == 2) *reinterpret_cast<uint4*>(dst + plane_stride + w0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            *reinterpret_cast<uint2*>(dst + w0) = make_uint2(hi[0], hi[1]);
+            if (PLANES == 2) *reinterpret_cast<uint2*>(dst + plane_stride + w0) = make_uint2(lo[0], lo[1]);
         }
-        // zero the row tail [nkb*bp, kst) once, by the CTA of the last block.
-        if (kb == nkb - 1) {
+        // zero the row tail [nkb*bp, kst) once, by the threads that wrote the last block's first quarter
+        if (kb == nkb - 1 && q == 0) {
             for (int64_t o = nkb * bp; o < kst; o += 16) {
-                *reinterpret_cast<uint4*>(mant + c * kst + o) = make_uint4(0, 0, 0, 0);
-                if (PLANES == 2) *reinterpret_cast<uint4*>(mant + plane_stride + c * kst + o) = make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(mant + col * kst + o) = make_uint4(0, 0, 0, 0);
+                if (PLANES == 2) *reinterpret_cast<uint4*>(mant + plane_stride + col * kst + o) = make_uint4(0, 0, 0, 0);
             }
         }
     }
@@ -538,22 +557,24 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
             default: break;
         }
     }
-    if (f->tile == 0 && axis == 0 && L.b <= 128 && L.nkb <= 65535) {
+    if (f->tile == 0 && axis == 0 && L.b <= 128) {
         const int vec_ok = aligned && (rows % 4 == 0);
-        size_t smem = (size_t)L.b * COLT * sizeof(float) + (p.rounding ? (size_t)L.b * (COLT / 8) * sizeof(uint4) : 0);
-        dim3 grid((unsigned)((rows + COLT - 1) / COLT), (unsigned)L.nkb);
-        // exponent padding bytes (lines >= rows) are documented as zero
-        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
-        if (L.planes == 1) {
-            HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_fast<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            quant_col_fast<1><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
-        } else {
-            HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_fast<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            quant_col_fast<2><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+        const int G = (int)(128 / L.b) > 16 ? 16 : ((int)(128 / L.b) > 0 ? (int)(128 / L.b) : 1);
+        const int64_t gy = (L.nkb + G - 1) / G;
+        if (gy <= 65535) {
+            const size_t krows = (size_t)G * L.b;
+            size_t smem = krows * COLT * sizeof(float) + (size_t)G * 4 * COLT * sizeof(uint32_t) +
+                          (p.rounding ? krows * (COLT / 8) * sizeof(uint4) : 0);
+            dim3 grid((unsigned)((rows + COLT - 1) / COLT), (unsigned)gy);
+            // exponent padding bytes (lines >= rows) are documented as zero
+            if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+            if (L.planes == 1)
+                quant_col_fast<1><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, G, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+            else
+                quant_col_fast<2><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, G, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+            return launch_status();
         }
-        return launch_status();
     }
-
     if (f->tile > 0 && f->tile <= 128) {
         // single view of a tiled weight: the fused tile kernel with the other view switched off
         return axis == 0 ? launch_quantize_tiles(x, d0, d1, ld, f, mant, exps, nullptr, nullptr, nullptr, st)
