@@ -36,7 +36,7 @@ INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio (4.5 : 2.
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one launch of the GEMM kernel at the default workload (n = 16384, m = 8,
 # b = 128), from the single-pass ncu capture summarised in profiles/bench_launch_list_n16384_m8_b128.md.
-GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 4046596608 + 1107060480}
+GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 3885147648 + 1110151680}
 
 
 def load_peaks():

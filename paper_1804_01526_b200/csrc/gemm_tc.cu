@@ -56,22 +56,31 @@ namespace {
 
 constexpr int TILE_M = 128;
 constexpr int STAGE_K = 128;          // bytes of K per stage (= one 128B swizzle row)
-constexpr int RESCALE_WARPS = 8;
+#ifndef HBFP_TC_RWARPS
+#define HBFP_TC_RWARPS 8              // rescale warps: 8 (two per sub-partition) or 16 (four)
+#endif
+constexpr int RESCALE_WARPS = HBFP_TC_RWARPS;
+constexpr int COL_GROUPS = RESCALE_WARPS / 4;      // warps sharing a lane quarter split the columns
 // The control warps take the lowest warp ids: the issue logic favours them over the rescale
 // warps of the same sub-partition, and a starved MMA issuer stalls the whole pipeline.
 constexpr int CONTROL_WARPS = 4;      // one warpgroup: producer, MMA issuer, table builder, one spare
 constexpr int PRODUCER_WARP = 0;
 constexpr int MMA_WARP = 1;
 constexpr int TABLE_WARP = 2;
-constexpr int THREADS = 384;           // warps 10 and 11 only give their registers away
+constexpr int THREADS = 32 * (4 + RESCALE_WARPS);
 constexpr uint32_t BIAS_BITS = 0x4B400000u;     // binary32 1.5 * 2^23
 #ifndef HBFP_TC_REGS_RESCALE
-#define HBFP_TC_REGS_RESCALE 208
+#define HBFP_TC_REGS_RESCALE (HBFP_TC_RWARPS == 8 ? 208 : 104)
 #endif
 #ifndef HBFP_TC_CHUNK
 #define HBFP_TC_CHUNK 16          // columns per tensor-memory load in the fast rescale path (16 or 32)
 #endif
-constexpr int REGS_RESCALE = HBFP_TC_REGS_RESCALE, REGS_CONTROL = (64512 - 256 * REGS_RESCALE) / 128;   // 128*88 + 256*208 = 64512 = 384*168: never ask for more than the launch allocation
+// setmaxnreg totals must never exceed what the launch allocated (threads x registers at launch,
+// 384 x 168 or 640 x 96): a request the register file cannot satisfy blocks forever.
+constexpr int REGS_LAUNCH_TOTAL = RESCALE_WARPS == 8 ? 384 * 168 : 640 * 96;
+constexpr int REGS_RESCALE = HBFP_TC_REGS_RESCALE;
+constexpr int REGS_CONTROL = ((REGS_LAUNCH_TOTAL - 32 * RESCALE_WARPS * REGS_RESCALE) / 128) / 8 * 8;
+static_assert(REGS_CONTROL >= 24 && 128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= REGS_LAUNCH_TOTAL, "register split");
 constexpr int TMEM_COLS = 512;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
 constexpr uint32_t WAIT_HINT_NS = 200000u;              // one try_wait may sleep this long; the loop around it is bounded
@@ -155,6 +164,14 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
                                                int32_t* status, int code) {
     const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
     return __all_sync(0xffffffffu, ok);
+}
+
+// Same copy with an L2 eviction-priority hint (a createpolicy-style 64-bit descriptor).
+constexpr uint64_t L2_EVICT_FIRST = 0x12F0000000000000ull, L2_EVICT_LAST = 0x14F0000000000000ull;
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(hint) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
@@ -331,7 +348,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                const Problem p) {
     using C = Cfg<N_TILE, PLANES>;
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
-    constexpr int COLS_PER_WARP = N_TILE / 2;          // each half of the rescale warps owns half the columns
+    constexpr int COLS_PER_WARP = N_TILE / COL_GROUPS;  // warps that share a lane quarter split the columns
     static_assert(!(MAGIC && PLANES != 1), "the biased-accumulator path is for one-plane operands");
 
     extern __shared__ unsigned char smem_dyn[];
@@ -403,10 +420,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         mbar_expect_tx(fb, (HBFP_TC_PROBE & 4) ? (uint32_t)C::EXP_STAGE : C::TX_BYTES);
                         const int kbyte = st0 * 32;
                         const uint32_t ms = mant_base + s * C::MANT_STAGE;
-                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d(ms, &mapA0, kbyte, w.m0, fb);
+                        // A panels are re-used by every column tile of a group of 16 tile rows: ask L2 to keep
+                        // them while the B panels stream past (marking B evict-first doubled the DRAM reads:
+                        // the 16 CTAs that share a B panel do not read it at the same instant).
+                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d_hint(ms, &mapA0, kbyte, w.m0, fb, L2_EVICT_LAST);
                         if (!(HBFP_TC_PROBE & 4)) tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
                         if (PLANES == 2 && !(HBFP_TC_PROBE & 4)) {
-                            tma_load_2d(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb);
+                            tma_load_2d_hint(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb, L2_EVICT_LAST);
                             tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
                         }
                         const uint32_t es = exp_base + s * C::EXP_STAGE;
@@ -516,7 +536,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         // ------------------------------------------------------------------ rescale warps
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
         const int rwarp = warp - CONTROL_WARPS;              // 0..7
-        const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4
+        const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4; half = column group
         const int row = quarter * 32 + lane;                 // row of the tile = tensor-memory lane
         const int col0 = half * COLS_PER_WARP;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
@@ -577,13 +597,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
                     constexpr int CH = HBFP_TC_CHUNK;
                     constexpr int NCHK = COLS_PER_WARP / CH;
-                    uint32_t v[2][CH];
-                    tc_ldn(taddr, v[0]);
+                    constexpr int NBUF = RESCALE_WARPS == 8 ? 2 : 1;   // four warps per sub-partition hide the load latency themselves
+                    uint32_t v[NBUF][CH];
+                    if (NBUF == 2) tc_ldn(taddr, v[0]);
 #pragma unroll
                     for (int ch = 0; ch < NCHK; ++ch) {
+                        if (NBUF == 1) tc_ldn(taddr + ch * CH, v[0]);
                         tc_wait_ld();
-                        if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & 1]);
-                        const uint32_t(&x)[CH] = v[ch & 1];
+                        if (NBUF == 2 && ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & (NBUF - 1)]);
+                        const uint32_t(&x)[CH] = v[ch & (NBUF - 1)];
                         if (DUMP && p.P != nullptr && gi < p.M) {
 #pragma unroll
                             for (int c = 0; c < CH; ++c) {
@@ -591,9 +613,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                                 if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)(x[c] - BIAS_BITS);
                             }
                         }
+#if HBFP_TC_PROBE & 16
+                        acc2[ch] ^= pack2(x[0], x[CH - 1]);
+                        continue;
+#endif
 #pragma unroll
                         for (int q = 0; q < CH; q += 4) {
+#if HBFP_TC_PROBE & 1024
+                            const uint4 sb = make_uint4(sa_u, sa_u + q, sa_u, sa_u + ch);
+#else
                             const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CH + q);
+#endif
 #if HBFP_TC_FFMA2
                             const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
                             const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
@@ -606,46 +636,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                             accf[ch * CH + q + 3] = fmaf(fmaf(__uint_as_float(x[q + 3]), sa_f, ca_f), __uint_as_float(sb.w), accf[ch * CH + q + 3]);
 #endif
                         }
+#if !(HBFP_TC_PROBE & 2048)
 #pragma unroll
                         for (int c8 = 0; c8 < CH / 8; ++c8) tc_st8(taddr + ch * CH + c8 * 8, bias);   // re-arm
+#endif
                     }
                     tc_wait_st();
                 } else {
                     const int sa = (int)sa_u;
 #pragma unroll
-                    for (int ch = 0; ch < COLS_PER_WARP / 32; ++ch) {
-                        int v[32];
-                        tc_ld32(taddr + ch * 32, v);
+                    for (int ch = 0; ch < COLS_PER_WARP / 16; ++ch) {
+                        uint32_t v[16];
+                        tc_ld16(taddr + ch * 16, v);
                         if (PLANES == 2) {
-                            int mid[32], ll[32];
-                            tc_ld32(taddr + N_TILE + ch * 32, mid);
-                            tc_ld32(taddr + 2 * N_TILE + ch * 32, ll);
+                            uint32_t mid[16], ll[16];
+                            tc_ld16(taddr + N_TILE + ch * 16, mid);
+                            tc_ld16(taddr + 2 * N_TILE + ch * 16, ll);
                             tc_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                v[c] = (int)(((uint32_t)v[c] << 8) + ((uint32_t)mid[c] << 4) + (uint32_t)ll[c]);
+                            for (int c = 0; c < 16; ++c) v[c] = (v[c] << 8) + (mid[c] << 4) + ll[c];
                         } else {
                             tc_wait_ld();
                         }
                         if (DUMP && p.P != nullptr && gi < p.M) {
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                const int64_t gj = n0 + col0 + ch * 32 + c;
-                                if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = v[c];
+                            for (int c = 0; c < 16; ++c) {
+                                const int64_t gj = n0 + col0 + ch * 16 + c;
+                                if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)v[c];
                             }
                         }
 #pragma unroll
-                        for (int c4 = 0; c4 < 32; c4 += 4) {
-                            const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 32 + c4);
+                        for (int c4 = 0; c4 < 16; c4 += 4) {
+                            const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * 16 + c4);
                             float a0, a1, a2, a3;
-                            unpack2(acc2[(ch * 32 + c4) / 2], a0, a1);
-                            unpack2(acc2[(ch * 32 + c4) / 2 + 1], a2, a3);
-                            a0 = fmaf((float)v[c4 + 0], __int_as_float(sa + (int)sb.x), a0);
-                            a1 = fmaf((float)v[c4 + 1], __int_as_float(sa + (int)sb.y), a1);
-                            a2 = fmaf((float)v[c4 + 2], __int_as_float(sa + (int)sb.z), a2);
-                            a3 = fmaf((float)v[c4 + 3], __int_as_float(sa + (int)sb.w), a3);
-                            acc2[(ch * 32 + c4) / 2] = pack2(__float_as_uint(a0), __float_as_uint(a1));
-                            acc2[(ch * 32 + c4) / 2 + 1] = pack2(__float_as_uint(a2), __float_as_uint(a3));
+                            unpack2(acc2[(ch * 16 + c4) / 2], a0, a1);
+                            unpack2(acc2[(ch * 16 + c4) / 2 + 1], a2, a3);
+                            a0 = fmaf((float)(int)v[c4 + 0], __int_as_float(sa + (int)sb.x), a0);
+                            a1 = fmaf((float)(int)v[c4 + 1], __int_as_float(sa + (int)sb.y), a1);
+                            a2 = fmaf((float)(int)v[c4 + 2], __int_as_float(sa + (int)sb.z), a2);
+                            a3 = fmaf((float)(int)v[c4 + 3], __int_as_float(sa + (int)sb.w), a3);
+                            acc2[(ch * 16 + c4) / 2] = pack2(__float_as_uint(a0), __float_as_uint(a1));
+                            acc2[(ch * 16 + c4) / 2 + 1] = pack2(__float_as_uint(a2), __float_as_uint(a3));
                         }
                     }
                 }
