@@ -187,15 +187,18 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
 // ------------------------------------------------------------------------------ quant_col_fast
 
 // Blocks down the columns of x [K][R] (contract axis 0); output rows are the columns of x.
-// CTA: 128 threads = 32 columns x 4 row slots; panel = G blocks of b <= 128 k-rows (G*b <= 128)
-// by 32 columns: 16 KB of shared memory, so a dozen CTAs fit an SM and cover the memory latency.
+// CTA: 128 threads = 32 columns x 4 row slots; panel = G blocks of b <= 128 k-rows (G * padded b
+// = 128) by 32 columns: 16 KB of shared memory, so a dozen CTAs fit an SM and cover the memory
+// latency. Each thread keeps its 32 values in registers between the max and the rounding pass.
 constexpr int COLT = 32;
 
-template <int PLANES>
+template <int PLANES, int RQ>      // RQ = bp / 4: padded rows per thread and block (8, 16 or 32)
 __global__ void __launch_bounds__(128)
-quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, int b, int bp, int G, QParams p,
+quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, int b, QParams p,
                int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
                int8_t* __restrict__ exps, int64_t rs, int64_t nkb, int vec_ok) {
+    constexpr int G = 32 / RQ;             // blocks per panel: G * bp = 128 padded rows
+    constexpr int BP = 4 * RQ;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int krows = G * b;
     float* tile = reinterpret_cast<float*>(smem_raw);                      // [krows][COLT]
@@ -233,58 +236,61 @@ quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, in
     }
     __syncthreads();
 
-    // 3. thread (q, c): quarter q of every block of column c. Partial maxima first.
-    const int rq = bp / 4;                  // padded rows per thread and block: 8, 16 or 32
+    // 3. thread (q, c) takes quarter q of every block of column c into registers.
+    float v[G][RQ];
+#pragma unroll
     for (int g = 0; g < G; ++g) {
         uint32_t am = 0;
-        const int r0 = g * b + q * rq;
-        for (int j = 0; j < rq; ++j) {
-            const int kk = r0 + j;
-            if (q * rq + j < b && kk < rows_here) am = max(am, abs_bits(tile[kk * COLT + c]));
+#pragma unroll
+        for (int j = 0; j < RQ; ++j) {
+            const int kk = g * b + q * RQ + j;
+            const bool valid = q * RQ + j < b && kk < rows_here;
+            v[g][j] = valid ? tile[kk * COLT + c] : 0.f;
+            am = max(am, abs_bits(v[g][j]));
         }
         pmax[(g * 4 + q) * COLT + c] = am;
     }
     __syncthreads();
 
     const int64_t col = c0 + c;
+    if (col >= R) return;
     const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
+#pragma unroll
     for (int g = 0; g < G; ++g) {
         const int64_t kb = kb0 + g;
-        if (kb >= nkb) break;
-        const uint32_t am = max(max(pmax[(g * 4 + 0) * COLT + c], pmax[(g * 4 + 1) * COLT + c]),
-                                max(pmax[(g * 4 + 2) * COLT + c], pmax[(g * 4 + 3) * COLT + c]));
-        const int s = block_exponent(am, p.m, p.exp_mode);
-        if (col >= R) continue;
-        if (q == 0) exps[kb * rs + col] = (int8_t)s;
-        int8_t* dst = mant + col * kst + kb * bp + q * rq;
-        const int r0 = g * b + q * rq;
-        for (int w0 = 0; w0 < rq; w0 += 8) {
-            uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
+        if (kb < nkb) {
+            const uint32_t am = max(max(pmax[(g * 4 + 0) * COLT + c], pmax[(g * 4 + 1) * COLT + c]),
+                                    max(pmax[(g * 4 + 2) * COLT + c], pmax[(g * 4 + 3) * COLT + c]));
+            const int s = block_exponent(am, p.m, p.exp_mode);
+            if (q == 0) exps[kb * rs + col] = (int8_t)s;
+            int8_t* dst = mant + col * kst + kb * BP + q * RQ;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int kk = r0 + w0 + j;
-                int qv = 0;
-                if (q * rq + w0 + j < b && kk < rows_here) {
-                    const float v = tile[kk * COLT + c];
-                    if (p.rounding == 0) qv = round_rne(v, s, p.qmax);
-                    else if (group_ok) qv = round_sr(v, s, p.qmax, rnd16[(kk * (COLT / 8) + (c >> 3)) * 8 + (c & 7)]);
-                    else qv = round_sr(v, s, p.qmax, draw_of_element(p, (uint64_t)((k0 + kk) * R + col)));
+            for (int w0 = 0; w0 < RQ; w0 += 8) {
+                uint32_t hi[2] = {0, 0}, lo[2] = {0, 0};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int kk = g * b + q * RQ + w0 + j;
+                    int qv;
+                    if (p.rounding == 0) qv = round_rne(v[g][w0 + j], s, p.qmax);
+                    else if (group_ok) qv = round_sr(v[g][w0 + j], s, p.qmax, rnd16[((kk < rows_here ? kk : 0) * (COLT / 8) + (c >> 3)) * 8 + (c & 7)]);
+                    else qv = round_sr(v[g][w0 + j], s, p.qmax, draw_of_element(p, (uint64_t)((k0 + kk) * R + col)));
+                    if (!(q * RQ + w0 + j < b && kk < rows_here)) qv = 0;     // padding stays zero whatever the draw
+                    if (PLANES == 1) {
+                        hi[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
+                    } else {
+                        hi[j >> 2] |= (uint32_t)((qv >> 4) & 0xff) << (8 * (j & 3));
+                        lo[j >> 2] |= (uint32_t)(qv & 15) << (8 * (j & 3));
+                    }
                 }
-                if (PLANES == 1) {
-                    hi[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
-                } else {
-                    hi[j >> 2] |= (uint32_t)((qv >> 4) & 0xff) << (8 * (j & 3));
-                    lo[j >> 2] |= (uint32_t)(qv & 15) << (8 * (j & 3));
-                }
+                *reinterpret_cast<uint2*>(dst + w0) = make_uint2(hi[0], hi[1]);
+                if (PLANES == 2) *reinterpret_cast<uint2*>(dst + plane_stride + w0) = make_uint2(lo[0], lo[1]);
             }
-            *reinterpret_cast<uint2*>(dst + w0) = make_uint2(hi[0], hi[1]);
-            if (PLANES == 2) *reinterpret_cast<uint2*>(dst + plane_stride + w0) = make_uint2(lo[0], lo[1]);
-        }
-        // zero the row tail [nkb*bp, kst) once, by the threads that wrote the last block's first quarter
-        if (kb == nkb - 1 && q == 0) {
-            for (int64_t o = nkb * bp; o < kst; o += 16) {
-                *reinterpret_cast<uint4*>(mant + col * kst + o) = make_uint4(0, 0, 0, 0);
-                if (PLANES == 2) *reinterpret_cast<uint4*>(mant + plane_stride + col * kst + o) = make_uint4(0, 0, 0, 0);
+            // zero the row tail [nkb*bp, kst) once
+            if (kb == nkb - 1 && q == 0) {
+                for (int64_t o = nkb * BP; o < kst; o += 16) {
+                    *reinterpret_cast<uint4*>(mant + col * kst + o) = make_uint4(0, 0, 0, 0);
+                    if (PLANES == 2) *reinterpret_cast<uint4*>(mant + plane_stride + col * kst + o) = make_uint4(0, 0, 0, 0);
+                }
             }
         }
     }
@@ -559,7 +565,7 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
     }
     if (f->tile == 0 && axis == 0 && L.b <= 128) {
         const int vec_ok = aligned && (rows % 4 == 0);
-        const int G = (int)(128 / L.b) > 16 ? 16 : ((int)(128 / L.b) > 0 ? (int)(128 / L.b) : 1);
+        const int G = (int)(128 / L.bp);                   // blocks per panel
         const int64_t gy = (L.nkb + G - 1) / G;
         if (gy <= 65535) {
             const size_t krows = (size_t)G * L.b;
@@ -568,10 +574,10 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
             dim3 grid((unsigned)((rows + COLT - 1) / COLT), (unsigned)gy);
             // exponent padding bytes (lines >= rows) are documented as zero
             if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
-            if (L.planes == 1)
-                quant_col_fast<1><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, G, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
-            else
-                quant_col_fast<2><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, (int)L.bp, G, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok);
+#define HBFP_QCOL(PL, RQ) quant_col_fast<PL, RQ><<<grid, 128, smem, st>>>(x, K, rows, ld, (int)L.b, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, vec_ok)
+            if (L.planes == 1) { if (L.bp == 32) HBFP_QCOL(1, 8); else if (L.bp == 64) HBFP_QCOL(1, 16); else HBFP_QCOL(1, 32); }
+            else { if (L.bp == 32) HBFP_QCOL(2, 8); else if (L.bp == 64) HBFP_QCOL(2, 16); else HBFP_QCOL(2, 32); }
+#undef HBFP_QCOL
             return launch_status();
         }
     }
