@@ -106,7 +106,7 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
     GemmPlan g;
     int rc = make_plan(M, N, K, a, b, &g);
     if (rc) return rc;
-    if (flags > HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_INVALID_ARG;
+    if (flags > HBFP_GEMM_FORCE_TENSOR_2SM) return HBFP_ERR_INVALID_ARG;
     if (P) {   // the inspection hook never splits K and needs no scratch
         g.total -= align_up(g.tp.partial_bytes, 1024);
         g.tp.partial_bytes = 0;
@@ -127,9 +127,13 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
     if (rc) return rc;
     const bool want_tensor = flags != HBFP_GEMM_FORCE_SIMT && g.tp.supported &&
                              (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc % 4) == 0;
-    if (want_tensor)
+    if (want_tensor) {
+        const bool pair_ok = !P && flags != HBFP_GEMM_FORCE_TENSOR_1SM && pair_gemm_eligible(M, N, pa, pb, g.tp);
+        if (pair_ok) return launch_gemm_tensor_pair(M, N, pa, pb, C, ldc, g.tp, ws ? ws + g.off_partial : nullptr, st);
+        if (flags == HBFP_GEMM_FORCE_TENSOR_2SM) return HBFP_ERR_UNSUPPORTED;
         return launch_gemm_tensor(M, N, K, pa, pb, C, ldc, P, g.tp, ws ? ws + g.off_partial : nullptr, st);
-    if (flags == HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_UNSUPPORTED;
+    }
+    if (flags >= HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_UNSUPPORTED;
     return launch_gemm_simt(M, N, K, pa, pb, C, ldc, P, st);
 }
 

@@ -89,6 +89,12 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
                        int64_t ldc, int32_t* P, const TensorPlan& plan, void* partial,
                        cudaStream_t st);
 
+// Paired-SM variant (two CTAs of a cluster per 256 x 256 tile): 8-bit mantissas, blocks up to 128,
+// no split-K, enough tiles to occupy every SM pair.
+bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, const TensorPlan& plan);
+int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed& b, float* C, int64_t ldc,
+                            const TensorPlan& plan, void* partial, cudaStream_t st);
+
 // Device status word (bounded waits report here).
 int32_t* device_status_word();   // device address, per current device
 int read_clear_device_status(cudaStream_t st, int32_t* out);

@@ -1,0 +1,644 @@
+// Paired-SM tensor-core BFP GEMM for sm_100a (8-bit mantissas, blocks of 32, 64 or 128 elements).
+//
+// Two CTAs of a cluster (one SM each) compute one 256 x 256 output tile: tcgen05.mma
+// cta_group::2 with M = 256 reads the A rows of both CTAs and one half of the B rows from each
+// CTA's shared memory, and leaves rows 0-127 of the int32 block sums in the first CTA's tensor
+// memory and rows 128-255 in the second one's. Per SM this is the same arithmetic and the same
+// rescale work as a 128 x 256 tile on one SM, but only half of the B panel crosses from L2 into
+// each SM, which is what limits the single-SM kernel on large problems.
+//
+// Roles per CTA (12 warps) as in the single-SM kernel: warp 0 TMA producer, warp 1 MMA issuer
+// (only in the cluster's first CTA, the leader) and tensor-memory owner, warp 2 scale-table
+// builder, warps 4-11 rescale (Eq. 2 per block, blocks accumulated in FP32, Sec. 4).
+//
+// Barriers. Mantissa tiles of both CTAs complete on the leader's full[s]; exponent slices on a
+// local efull[s]; the leader's MMA thread commits to tfull[g] and empty[s] of both CTAs; the
+// rescale warps of both CTAs arrive on the leader's tempty[g]. Every wait is bounded: when one
+// expires the CTA records a code in the device status word, raises its abort flag, drains what
+// it can wait for and leaves through the common teardown (cluster barrier, tensor memory freed).
+#include <cuda.h>
+
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace hbfp {
+namespace {
+
+constexpr int N_TILE = 256;            // columns of the pair tile = accumulator columns per CTA
+constexpr int PAIR_M = 2 * TILE_M;     // rows of the pair tile
+constexpr int B_HALF = N_TILE / 2;     // B rows staged in each CTA
+constexpr int RESCALE_WARPS = 8;
+constexpr int CONTROL_WARPS = 4;
+#ifndef HBFP_TC2_TABLE_WARP
+#define HBFP_TC2_TABLE_WARP 2
+#endif
+constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = HBFP_TC2_TABLE_WARP;
+constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
+// setmaxnreg totals must not exceed the launch allocation (384 threads x 168 registers)
+constexpr int REGS_RESCALE = 208, REGS_CONTROL = 88;
+static_assert(128 * REGS_CONTROL + 256 * REGS_RESCALE <= 384 * 168, "register split");
+
+constexpr int GROUPS = TMEM_COLS / N_TILE;                  // 2 accumulator groups
+constexpr int A_BYTES = TILE_M * STAGE_K, B_BYTES = B_HALF * STAGE_K;
+constexpr int MANT_STAGE = A_BYTES + B_BYTES;               // 32 KB per CTA and stage
+constexpr int EXP_A = 4 * TILE_M, EXP_B = 4 * N_TILE;       // up to four blocks start in a stage
+constexpr int EXP_STAGE = EXP_A + EXP_B;
+constexpr int TSLOTS = 4;
+constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
+constexpr int TABLE_BYTES = 4 * TSLOTS * TABLE_SLOT_WORDS;
+constexpr int STAGES = 6;
+constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024;
+static_assert(SMEM <= 232448, "shared memory");
+constexpr int CH = 16;                                      // columns per tensor-memory load
+
+// Build-time probe for performance bisection (never set in the shipped library; results are wrong
+// when it is): 1 = rescale warps skip the tensor-memory traffic and the math, 2 = no MMA is issued,
+// 4 = no mantissa tile is copied, 8 = cluster 0 records per-role timestamps.
+#ifndef HBFP_TC2_PROBE
+#define HBFP_TC2_PROBE 0
+#endif
+#ifndef HBFP_TC2_ARRIVE
+#define HBFP_TC2_ARRIVE 0
+#endif
+#ifndef HBFP_TC2_TABLE_POLL
+#define HBFP_TC2_TABLE_POLL 1
+#endif
+#ifndef HBFP_TC2_WAIT
+#define HBFP_TC2_WAIT 0
+#endif
+
+struct Problem {
+    int64_t M, N;
+    int64_t nkb;
+    int bp;
+    int tiles_m, tiles_n;   // pair tiles
+    long long* trace;       // probe builds only
+    int splits;
+    int64_t kb_per_split;
+    float* C;
+    int64_t ldc;
+    float* partial;
+    int64_t ldp;
+    int32_t* status;
+};
+
+#if HBFP_TC2_PROBE & 8
+#define TC2_TRACE(role, idx)                                                                     \
+    do {                                                                                          \
+        if (p.trace && cluster == 0 && (idx) < 512) p.trace[((int)rank * 32 + (role)) * 512 + (idx)] = clock64(); \
+    } while (0)
+#else
+#define TC2_TRACE(role, idx) do { } while (0)
+#endif
+
+struct Work {
+    int m0, n0, split;
+    int kb0, nblk;          // first K-block and number of K-blocks of this item
+};
+
+// Same traversal as the single-SM kernel: groups of tile rows (2048 matrix rows) sweep across N
+// so that their B panels are shared in L2. 32-bit arithmetic only; returned by value so that the
+// fields stay in registers.
+__device__ __forceinline__ Work get_work(const Problem& p, int w) {
+    Work out;
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int split = w / tiles;
+    const int t = w - split * tiles;
+    const int G = 8;
+    const int per_group = G * p.tiles_n;
+    const int group = t / per_group;
+    const int first_m = group * G;
+    const int gsize = min(G, p.tiles_m - first_m);
+    const int within = t - group * per_group;
+    const int nt = within / gsize;
+    out.m0 = (first_m + (within - nt * gsize)) * PAIR_M;
+    out.n0 = nt * N_TILE;
+    out.split = split;
+    out.kb0 = split * (int)p.kb_per_split;
+    out.nblk = min((int)p.nkb, out.kb0 + (int)p.kb_per_split) - out.kb0;
+    return out;
+}
+
+// ------------------------------------------------------------------------------ cluster PTX
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in the CTA of the given rank.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+#if HBFP_TC2_ARRIVE == 0
+    // release at CTA scope: what the arrival has to order are this warp's tensor-memory accesses, and
+    // tcgen05.wait + tcgen05.fence::before_thread_sync do that; a cluster-scope release costs ~1000 cycles
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+#else
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+#endif
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+
+// Wait on a barrier that threads of the other CTA arrive on (acquire at cluster scope).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+#if HBFP_TC_TESTWAIT
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#elif HBFP_TC2_WAIT == 0
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+#else
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+#endif
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  int32_t* status, int code) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicCAS(status, 0, code);
+            return false;
+        }
+    }
+}
+
+// Bounded polling wait (test_wait + nanosleep) for a whole warp: used where a suspended try_wait
+// would sit on a barrier that other warps of the same sub-partition are suspended on too.
+__device__ __forceinline__ bool mbar_poll_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
+    bool ok = true;
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (!done) {
+        const long long t0 = clock64();
+        for (;;) {
+            __nanosleep(64);
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            if (done) break;
+            if (*abort_flag) { ok = false; break; }
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicCAS(status, 0, code);
+                ok = false;
+                break;
+            }
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+// Tile copy issued by one CTA of a pair; the completion bytes may be counted on a barrier of
+// either CTA (`bar` is a cluster-window address). Plain copy: no multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "l"(hint) : "memory");
+}
+constexpr uint64_t L2_EVICT_NORMAL = 0x1000000000000000ull;
+
+// D[tmem of both CTAs] (+)= A * B, int8 x int8 -> int32, M = 256 (128 rows per CTA), K = 32.
+__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrives (once all earlier MMAs of this thread have completed) on the barrier at this offset in
+// every CTA of the mask.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(cta_mask) : "memory");
+}
+__device__ __forceinline__ constexpr uint32_t idesc_i8_pair() {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+}
+
+// 2^e as binary32 bits, e = signed byte i of a packed word of four exponents.
+__device__ __forceinline__ uint32_t exp_to_scale(uint32_t packed, int i) {
+    const int e = (int)(int8_t)(packed >> (8 * i));
+    return (uint32_t)(e + 127) << 23;
+}
+
+// ------------------------------------------------------------------------------ kernel
+
+// Advances a ring position (stage, accumulator group or table slot) and its phase bit.
+template <int N>
+__device__ __forceinline__ void ring_next(uint32_t& i, uint32_t& ph) {
+    if (++i == N) { i = 0; ph ^= 1u; }
+}
+
+// LB = log2(K-blocks per 128-byte stage): 0 for blocks of 128 bytes, 1 for 64, 2 for 32.
+template <int LB>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                const __grid_constant__ CUtensorMap mapEA, const __grid_constant__ CUtensorMap mapEB,
+                const Problem p) {
+    constexpr int BPS = 1 << LB;          // K-blocks per stage
+    constexpr int SPB = 4 >> LB;          // K=32 MMA steps per block
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    const uint32_t mant_base = base;                                     // STAGES x MANT_STAGE, 1024-aligned
+    const uint32_t exp_base = mant_base + STAGES * MANT_STAGE;           // STAGES x EXP_STAGE
+    const uint32_t table_off = STAGES * (MANT_STAGE + EXP_STAGE);
+    uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [slot][256 column scales | 128 row scales]
+    const uint32_t bar_off = table_off + TABLE_BYTES;
+    const uint32_t bars = base + bar_off;
+    const uint32_t full_bar = bars;                          // leader: mantissa tiles of both CTAs landed
+    const uint32_t efull_bar = full_bar + 8 * STAGES;        // local: exponent slices landed
+    const uint32_t empty_bar = efull_bar + 8 * STAGES;       // local: stage consumed (MMA commit + table warp)
+    const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums complete (MMA commit) and scale table written
+    const uint32_t tempty_bar = tfull_bar + 8 * GROUPS;      // leader: group read and re-armed by both CTAs
+    const uint32_t done_bar = tempty_bar + 8 * GROUPS;
+    constexpr int BAR_BYTES = 24 * STAGES + 16 * GROUPS + 8;
+    static_assert(BAR_BYTES + 8 <= 1024, "barrier area");
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + BAR_BYTES);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();                 // 0 = leader
+    const int cluster = (int)cluster_id_x(), nclusters = (int)cluster_count_x();
+    const int total_work = p.tiles_m * p.tiles_n * p.splits;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(efull_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 2);
+        }
+        for (int g = 0; g < GROUPS; ++g) {
+            mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + this CTA's table warp
+            mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS);
+        }
+        mbar_init(done_bar, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == MMA_WARP) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();            // both CTAs' barriers and tensor memory exist before anyone signals across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp < CONTROL_WARPS) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CONTROL));
+        if (warp == PRODUCER_WARP) {
+            // -------------------------------------------------------------- TMA producer (both CTAs)
+            if (lane == 0) {
+                const uint32_t leader_full = map_to_rank(full_bar, 0);
+                uint32_t s = 0, ph = 0, it = 0;
+                bool ok = true;
+                for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
+                    const Work w = get_work(p, wi);
+                    const int my_m = w.m0 + (int)rank * TILE_M;      // this CTA's A rows
+                    const int my_n = w.n0 + (int)rank * B_HALF;      // this CTA's half of the B rows
+                    const int nst = (w.nblk + BPS - 1) >> LB;
+                    int kb = w.kb0, kbyte = w.kb0 * (128 >> LB);
+                    for (int si = 0; si < nst; ++si, kb += BPS, kbyte += STAGE_K, ++it) {
+                        if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 111)) { ok = false; break; }
+                        TC2_TRACE(0, it);
+                        if (rank == 0 && !(HBFP_TC2_PROBE & 4)) mbar_expect_tx(full_bar + 8 * s, 2u * MANT_STAGE);
+                        if (rank == 0 && (HBFP_TC2_PROBE & 4)) mbar_arrive(full_bar + 8 * s);
+                        mbar_expect_tx(efull_bar + 8 * s, (uint32_t)EXP_STAGE);
+                        const uint32_t ms = mant_base + s * MANT_STAGE;
+                        if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms, &mapA, kbyte, my_m, leader_full + 8 * s, L2_EVICT_LAST);
+                        if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES, &mapB, kbyte, my_n, leader_full + 8 * s, L2_EVICT_NORMAL);
+                        const uint32_t es = exp_base + s * EXP_STAGE;
+                        tma_load_2d(es, &mapEA, my_m, kb, efull_bar + 8 * s);
+                        tma_load_2d(es + EXP_A, &mapEB, w.n0, kb, efull_bar + 8 * s);
+                        ring_next<STAGES>(s, ph);
+                    }
+                }
+                // Drain the copies this CTA can wait for: its exponent slices, and on the leader the
+                // mantissa tiles of both CTAs. In a normal run the consumers already waited for all
+                // of them, so these return at once.
+                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                for (uint32_t k = 0; k < back; ++k) {
+                    if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+                    mbar_wait(efull_bar + 8 * s, ph, abort_flag, p.status, 112, false);
+                    if (rank == 0) mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 113, false);
+                }
+            }
+        } else if (warp == MMA_WARP) {
+            // -------------------------------------------------------------- MMA issuer (leader only)
+            if (lane == 0 && rank == 0) {
+                constexpr uint32_t idesc = idesc_i8_pair();
+                uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
+                bool ok = true;
+                for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
+                    const Work w = get_work(p, wi);
+                    const int nst = (w.nblk + BPS - 1) >> LB;
+                    int left = w.nblk;
+                    for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
+                        if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 211)) { ok = false; break; }
+                        TC2_TRACE(1, it);
+                        tc_fence_after();
+                        const uint32_t ms = mant_base + s * MANT_STAGE;
+                        const uint64_t a_desc = smem_desc_sw128(ms), b_desc = smem_desc_sw128(ms + A_BYTES);
+#pragma unroll
+                        for (int jb = 0; jb < BPS; ++jb) {
+                            if (jb < left) {
+                                // the group was read and re-armed by the rescale warps of both CTAs
+                                if (!mbar_wait_cluster(tempty_bar + 8 * g, gph, abort_flag, p.status, 212)) { ok = false; break; }
+                                TC2_TRACE(2, blk);
+                                tc_fence_after();
+                                const uint32_t d = tmem_base + g * N_TILE;
+#pragma unroll
+                                for (int q = 0; q < SPB; ++q) {
+                                    const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
+                                    if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, b_desc + ko, idesc, 1u);   // on top of the bias
+                                }
+                                tc_commit_pair(tfull_bar + 8 * g, 3);
+                                TC2_TRACE(3, blk);
+                                ring_next<GROUPS>(g, gph);
+                                ++blk;
+                            }
+                        }
+                        tc_commit_pair(empty_bar + 8 * s, 3);        // the stage is free in both CTAs
+                        ring_next<STAGES>(s, ph);
+                    }
+                }
+                tc_commit_pair(done_bar, 1);
+                mbar_wait(done_bar, 0, abort_flag, p.status, 213, false);
+            }
+        } else if (warp == TABLE_WARP) {
+            // -------------------------------------------------------------- scale-table builder
+            // The table of block b goes to slot b % 4 and its arrival counts on tfull[b % 2]. It is
+            // written once the phase of block b - 2 on that barrier is complete: the MMAs of b - 2 were
+            // issued only after every rescale warp had finished b - 4, the last reader of the slot, and
+            // the barrier is back in the phase that the arrival for b belongs to.
+            uint32_t s = 0, ph = 0, g = 0, gph = 0, slot = 0, it = 0, blk = 0;
+            bool ok = true;
+            for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
+                const Work w = get_work(p, wi);
+                const int nst = (w.nblk + BPS - 1) >> LB;
+                int left = w.nblk;
+                for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
+                    if (!mbar_wait_warp(efull_bar + 8 * s, ph, abort_flag, p.status, 411)) { ok = false; break; }
+                    if (lane == 0) TC2_TRACE(20, it);
+                    const unsigned char* eA = base_ptr + (exp_base - base) + s * EXP_STAGE;
+                    const unsigned char* eB = eA + EXP_A;
+#pragma unroll
+                    for (int jb = 0; jb < BPS; ++jb) {
+                        if (jb < left) {
+                            // this lane's 8 column exponents and 4 row exponents of block jb of the stage
+                            const uint2 cb = *reinterpret_cast<const uint2*>(eB + jb * N_TILE + 8 * lane);
+                            const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
+                            uint4 c0, c1, r0;
+                            c0.x = exp_to_scale(cb.x, 0); c0.y = exp_to_scale(cb.x, 1); c0.z = exp_to_scale(cb.x, 2); c0.w = exp_to_scale(cb.x, 3);
+                            c1.x = exp_to_scale(cb.y, 0); c1.y = exp_to_scale(cb.y, 1); c1.z = exp_to_scale(cb.y, 2); c1.w = exp_to_scale(cb.y, 3);
+                            r0.x = exp_to_scale(ra, 0); r0.y = exp_to_scale(ra, 1); r0.z = exp_to_scale(ra, 2); r0.w = exp_to_scale(ra, 3);
+#if HBFP_TC2_TABLE_POLL
+                            if (!mbar_poll_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
+#else
+                            if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
+#endif
+                            if (lane == 0) TC2_TRACE(21, blk);
+                            uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
+                            *reinterpret_cast<uint4*>(tb + 8 * lane) = c0;
+                            *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
+                            *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
+                            if (lane == 0) TC2_TRACE(22, blk);
+                            ring_next<GROUPS>(g, gph);
+                            slot = (slot + 1) & (TSLOTS - 1);
+                            ++blk;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar + 8 * s);      // the exponent slices are consumed
+                    if (lane == 0) TC2_TRACE(25, it);
+                    ring_next<STAGES>(s, ph);
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ rescale warps (both CTAs)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
+        constexpr int COLS_PER_WARP = N_TILE / 2;            // two warps share a lane quarter and split the columns
+        const int rwarp = warp - CONTROL_WARPS;              // 0..7
+        const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4
+        const int row = quarter * 32 + lane;                 // row of this CTA's half tile = tensor-memory lane
+        const int col0 = half * COLS_PER_WARP;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
+        const uint32_t leader_tempty = map_to_rank(tempty_bar, 0);
+        uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
+        uint32_t bias[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
+        for (int g = 0; g < GROUPS; ++g)
+#pragma unroll
+            for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
+        tc_wait_st();
+        // Read the bias back as one eight-register tuple: a tuple that is born as such is passed to
+        // every re-arming store in place, while eight separately defined registers would be copied
+        // into a fresh tuple for each store (eight extra instructions per store).
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(bias[0]), "=r"(bias[1]), "=r"(bias[2]), "=r"(bias[3]), "=r"(bias[4]), "=r"(bias[5]), "=r"(bias[6]), "=r"(bias[7])
+                     : "r"(lane_addr) : "memory");
+        tc_wait_ld();
+        // every accumulator group starts out free
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0)
+            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * g);
+
+        uint32_t g = 0, gph = 0, slot = 0, blk = 0;
+        bool ok = true;
+        for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
+            const Work w = get_work(p, wi);
+            const int64_t gi = w.m0 + (int)rank * TILE_M + row;
+#pragma unroll
+            for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
+            for (int kb = 0; kb < w.nblk; ++kb, ++blk) {
+                // one wait per block: the block sums are complete and this CTA's scale table is written
+                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 312)) { ok = false; break; }
+                if (lane == 0) TC2_TRACE(4 + rwarp, blk);
+                tc_fence_after();
+                const uint32_t taddr = lane_addr + g * N_TILE;
+                const uint32_t* tab = tables + slot * TABLE_SLOT_WORDS + col0;
+                // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
+                // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
+                const float sa_f = __uint_as_float(tables[slot * TABLE_SLOT_WORDS + N_TILE + row]);
+                const float ca_f = -12582912.0f * sa_f;
+                const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
+                const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
+                constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : COLS_PER_WARP / CH;
+                uint32_t v[2][CH];
+                if (NCHK) tc_ldn(taddr, v[0]);
+#pragma unroll
+                for (int ch = 0; ch < NCHK; ++ch) {
+                    tc_wait_ld();
+                    if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & 1]);
+                    const uint32_t(&x)[CH] = v[ch & 1];
+#pragma unroll
+                    for (int q = 0; q < CH; q += 4) {
+                        const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CH + q);
+                        const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
+                        const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
+                        acc2[(ch * CH + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
+                        acc2[(ch * CH + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CH + q) / 2 + 1]);
+                    }
+#pragma unroll
+                    for (int c8 = 0; c8 < CH / 8; ++c8) tc_st8(taddr + ch * CH + c8 * 8, bias);   // re-arm
+                }
+                if (lane == 0 && rwarp == 0) TC2_TRACE(29, blk);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_remote(leader_tempty + 8 * g);
+                    TC2_TRACE(12 + rwarp, blk);
+                }
+                ring_next<GROUPS>(g, gph);
+                slot = (slot + 1) & (TSLOTS - 1);
+            }
+            if (!ok) break;
+            // ---- store this CTA's 128 rows of the tile (or of this split's partial tile)
+            float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
+            const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
+            if (gi < p.M) {
+                float* rowp = dst + gi * ldd + w.n0 + col0;
+#pragma unroll
+                for (int c = 0; c < COLS_PER_WARP; c += 4) {
+                    const int64_t gj = w.n0 + col0 + c;
+                    if (gj + 3 < p.N) {
+                        *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
+                    } else {
+                        float e4[4];
+                        unpack2(acc2[c / 2], e4[0], e4[1]);
+                        unpack2(acc2[c / 2 + 1], e4[2], e4[3]);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            if (gj + e < p.N) rowp[c + e] = e4[e];
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------------ teardown
+    // Neither CTA may leave while the other can still signal its barriers or read its shared memory.
+    tc_fence_before();
+    __syncthreads();
+    cluster_barrier();
+    if (warp == MMA_WARP) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+int max_clusters() {
+    static int n = 0;
+    if (!n) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 148, 1, 1);
+        cfg.blockDim = dim3(THREADS, 1, 1);
+        cfg.dynamicSmemBytes = SMEM;
+        int c = 0;
+        if (cudaOccupancyMaxActiveClusters(&c, gemm_tc2_kernel<0>, &cfg) != cudaSuccess || c < 1) {
+            cudaGetLastError();
+            c = -1;
+        }
+        n = c;
+    }
+    return n;
+}
+
+}  // namespace
+
+#if HBFP_TC2_PROBE & 8
+long long* g_probe_trace2 = nullptr;
+extern "C" __attribute__((visibility("default"))) void hbfp_probe_set_trace2(long long* ptr) { g_probe_trace2 = ptr; }
+#endif
+
+bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, const TensorPlan& plan) {
+    if (a.L.planes != 1 || b.L.planes != 1) return false;
+    if (a.L.bp > 128 || plan.n_tile != 256) return false;
+    const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
+    if (qa * qb * a.L.b >= (1ll << 22)) return false;        // the biased accumulator needs |P| < 2^22
+    if (plan.splits != 1) return false;
+    // enough pair tiles to occupy every SM pair
+    const int64_t tiles = ((M + PAIR_M - 1) / PAIR_M) * ((N + N_TILE - 1) / N_TILE);
+    return tiles >= 74;
+}
+
+int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed& b, float* Cout, int64_t ldc,
+                            const TensorPlan& plan, void* partial, cudaStream_t st) {
+    Problem p{};
+    p.M = M;
+    p.N = N;
+    p.nkb = a.L.nkb;
+    p.bp = (int)a.L.bp;
+    p.tiles_m = (int)((M + PAIR_M - 1) / PAIR_M);
+    p.tiles_n = (int)((N + N_TILE - 1) / N_TILE);
+    p.splits = plan.splits;
+    p.kb_per_split = plan.kb_per_split;
+    p.C = Cout;
+    p.ldc = ldc;
+    p.partial = static_cast<float*>(partial);
+    p.ldp = round_up(N, 4);
+    p.status = device_status_word();
+    if (!p.status) return HBFP_ERR_CUDA;
+    if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
+#if HBFP_TC2_PROBE & 8
+    p.trace = g_probe_trace2;
+#endif
+    CUtensorMap mA, mB, mEA, mEB;
+    int rc;
+    rc = make_map(&mA, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
+    if (rc) return rc;
+    rc = make_map(&mB, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, B_HALF, true);
+    if (rc) return rc;
+    rc = make_map(&mEA, a.exps, a.L.rs, a.L.nkb, a.L.rs, TILE_M, 4, false);
+    if (rc) return rc;
+    rc = make_map(&mEB, b.exps, b.L.rs, b.L.nkb, b.L.rs, N_TILE, 4, false);
+    if (rc) return rc;
+    static bool attr_set = false;
+    if (!attr_set) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+        attr_set = true;
+    }
+    const int clusters_max = max_clusters();
+    if (clusters_max < 1) return HBFP_ERR_UNSUPPORTED;
+    const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
+    const int clusters = (int)(work < clusters_max ? work : clusters_max);
+    if (p.bp == 128) gemm_tc2_kernel<0><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);
+    else if (p.bp == 64) gemm_tc2_kernel<1><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);
+    else gemm_tc2_kernel<2><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);
+    return launch_status();
+}
+
+}  // namespace hbfp

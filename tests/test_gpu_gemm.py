@@ -128,3 +128,60 @@ def test_argument_errors_are_reported_not_thrown_by_cuda(hb):
     assert hb.device_status() == 0
     C = hb.gemm(0, 0, A[:0], A, f, f)          # empty M
     assert C.shape == (0, 64)
+
+
+# The paired-SM kernel (two CTAs per 256 x 256 tile) needs at least 74 such tiles; these shapes span
+# several tiles per SM pair, ragged edges in M, N and K, a second CTA whose half tile lies entirely
+# outside the matrix (M % 256 <= 128, N % 256 <= 128), and all three blocks-per-stage variants.
+PAIR_CASES = [
+    # m, block, M, N, K
+    (8, 128, 2560, 2048, 640),
+    (8, 128, 2400, 2100, 1000),
+    (8, 64, 2660, 2304, 448),
+    (6, 64, 2304, 2188, 200),
+    (8, 32, 2560, 2048, 288),
+    (8, 100, 2688, 2176, 1000),
+    (4, 16, 2330, 2332, 176),
+]
+
+
+@pytest.mark.parametrize("m,b,M,N,K", PAIR_CASES)
+def test_paired_sm_kernel_matches_oracle_bit_for_bit(hb, m, b, M, N, K):
+    A = wl.draw("lognormal", (M, K), seed=31)
+    B = wl.draw("lognormal", (K, N), seed=32)
+    fd = dict(mant_bits=m, block=b, rounding=0, seed=0)
+    ref = oracle.hbfp_gemm(0, 0, A, B, ofmt(fd), ofmt(fd))
+    C2 = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), flags=hb.GEMM_FORCE_TENSOR_2SM).cpu().numpy()
+    assert hb.device_status() == 0
+    err = np.abs(C2.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+    assert np.array_equal(C2, ref["c_seq"])      # blocks accumulated in ascending order, no split-K
+    C1 = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), flags=hb.GEMM_FORCE_TENSOR_1SM).cpu().numpy()
+    assert np.array_equal(C1, C2)
+    Ca = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), flags=hb.GEMM_AUTO).cpu().numpy()
+    assert np.array_equal(Ca, C2)
+
+
+def test_paired_sm_kernel_transposed_operands_and_stochastic_rounding(hb):
+    # wgrad-shaped call: both operands are contracted along their row axis (column quantiser)
+    M, N, K = 2304, 2304, 384
+    X = wl.draw("half_normal", (K, M), seed=41)
+    dY = wl.draw("grad", (K, N), seed=42)
+    fa = dict(mant_bits=8, block=128, rounding=1, seed=9)
+    ref = oracle.hbfp_gemm(1, 0, X, dY, ofmt(fa), ofmt(fa, stream_id=1))
+    C = hb.gemm(1, 0, to_dev(X), to_dev(dY), gfmt(fa), gfmt(fa, stream_id=1), flags=hb.GEMM_FORCE_TENSOR_2SM).cpu().numpy()
+    assert hb.device_status() == 0
+    assert np.array_equal(C, ref["c_seq"])
+
+
+def test_paired_sm_kernel_refuses_what_it_cannot_run(hb):
+    A = to_dev(wl.draw("normal", (256, 256), seed=1))
+    f8 = dict(mant_bits=8, block=128, rounding=0, seed=0)
+    with pytest.raises(hb.HbfpError) as e:           # too few tiles to occupy the SM pairs
+        hb.gemm(0, 0, A, A, gfmt(f8), gfmt(f8), flags=hb.GEMM_FORCE_TENSOR_2SM)
+    assert e.value.code == hb.ERR_UNSUPPORTED
+    big = to_dev(wl.draw("normal", (2560, 2048), seed=2))
+    f12 = dict(mant_bits=12, block=64, rounding=0, seed=0)
+    with pytest.raises(hb.HbfpError) as e:           # two mantissa planes
+        hb.gemm(0, 1, big, big, gfmt(f12), gfmt(f12), flags=hb.GEMM_FORCE_TENSOR_2SM)
+    assert e.value.code == hb.ERR_UNSUPPORTED

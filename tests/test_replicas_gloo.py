@@ -18,7 +18,8 @@ mine = 1.0 + rep.rank            # rank 1 is slower
 worst = replicas.max_over_ranks(rep, mine)
 agg = replicas.aggregate_throughput(rep, 100.0, worst)
 replicas.barrier(rep)
-print(json.dumps(dict(rank=rep.rank, world=rep.world, worst=worst, agg=agg, root=rep.is_root)))
+with open(os.path.join({out!r}, "rank%d.json" % rep.rank), "w") as f:   # one file per rank: stdout lines of two ranks can interleave
+    json.dump(dict(rank=rep.rank, world=rep.world, worst=worst, agg=agg, root=rep.is_root), f)
 replicas.shutdown(rep)
 """
 
@@ -40,10 +41,10 @@ def _torchrun(args, nproc=2, timeout=180):
 
 def test_two_gloo_ranks_agree_on_the_slowest_time(tmp_path):
     script = tmp_path / "worker.py"
-    script.write_text(WORKER.format(root=ROOT))
+    script.write_text(WORKER.format(root=ROOT, out=str(tmp_path)))
     r = _torchrun([str(script)])
     assert r.returncode == 0, r.stderr[-2000:]
-    rows = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    rows = [json.loads((tmp_path / f"rank{i}.json").read_text()) for i in range(2)]
     assert sorted(x["rank"] for x in rows) == [0, 1]
     for x in rows:
         assert x["world"] == 2 and x["worst"] == 2.0 and x["agg"] == 2 * 100.0 / 2.0
