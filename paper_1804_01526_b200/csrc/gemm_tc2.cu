@@ -26,7 +26,13 @@ namespace {
 
 constexpr int N_TILE = 256;            // columns of the pair tile = accumulator columns per CTA
 constexpr int PAIR_M = 2 * TILE_M;     // rows of the pair tile
-constexpr int B_HALF = N_TILE / 2;     // B rows staged in each CTA
+#ifndef HBFP_TC2_HALVES
+#define HBFP_TC2_HALVES 1
+#endif
+constexpr int HALVES = HBFP_TC2_HALVES; // 2: the tile is computed as two column halves with their own barriers; 1: as a whole
+constexpr int N_HALF = N_TILE / HALVES; // columns of one MMA
+constexpr int B_HALF = N_TILE / 2;      // B rows staged in each CTA
+constexpr int B_BOX = N_HALF / 2;       // rows of one B copy (this CTA's share of one MMA's columns)
 constexpr int RESCALE_WARPS = 8;
 constexpr int CONTROL_WARPS = 4;
 #ifndef HBFP_TC2_TABLE_WARP
@@ -35,7 +41,10 @@ constexpr int CONTROL_WARPS = 4;
 constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = HBFP_TC2_TABLE_WARP;
 constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
 // setmaxnreg totals must not exceed the launch allocation (384 threads x 168 registers)
-constexpr int REGS_RESCALE = 208, REGS_CONTROL = 88;
+#ifndef HBFP_TC2_REGS_RESCALE
+#define HBFP_TC2_REGS_RESCALE 216
+#endif
+constexpr int REGS_RESCALE = HBFP_TC2_REGS_RESCALE, REGS_CONTROL = (384 * 168 - 256 * HBFP_TC2_REGS_RESCALE) / 128 / 8 * 8;
 static_assert(128 * REGS_CONTROL + 256 * REGS_RESCALE <= 384 * 168, "register split");
 
 constexpr int GROUPS = TMEM_COLS / N_TILE;                  // 2 accumulator groups
@@ -211,6 +220,13 @@ __device__ __forceinline__ bool mbar_poll_warp(uint32_t bar, uint32_t parity, vo
     return __all_sync(0xffffffffu, ok);
 }
 
+// Non-blocking look at a barrier phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+
 // Tile copy issued by one CTA of a pair; the completion bytes may be counted on a barrier of
 // either CTA (`bar` is a cluster-window address). Plain copy: no multicast.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t hint) {
@@ -234,7 +250,7 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) 
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(cta_mask) : "memory");
 }
 __device__ __forceinline__ constexpr uint32_t idesc_i8_pair() {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_HALF >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
 }
 
 // 2^e as binary32 bits, e = signed byte i of a packed word of four exponents.
@@ -271,10 +287,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t full_bar = bars;                          // leader: mantissa tiles of both CTAs landed
     const uint32_t efull_bar = full_bar + 8 * STAGES;        // local: exponent slices landed
     const uint32_t empty_bar = efull_bar + 8 * STAGES;       // local: stage consumed (MMA commit + table warp)
-    const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums complete (MMA commit) and scale table written
-    const uint32_t tempty_bar = tfull_bar + 8 * GROUPS;      // leader: group read and re-armed by both CTAs
-    const uint32_t done_bar = tempty_bar + 8 * GROUPS;
-    constexpr int BAR_BYTES = 24 * STAGES + 16 * GROUPS + 8;
+    // accumulator barriers exist per group and column half: index 2 * g + h
+    const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums of a half complete (MMA commit) and scale table written
+    const uint32_t tempty_bar = tfull_bar + 16 * GROUPS;     // leader: half group read and re-armed by its warps in both CTAs
+    const uint32_t done_bar = tempty_bar + 16 * GROUPS;
+    constexpr int BAR_BYTES = 24 * STAGES + 32 * GROUPS + 8;
     static_assert(BAR_BYTES + 8 <= 1024, "barrier area");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + BAR_BYTES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -290,12 +307,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             mbar_init(efull_bar + 8 * s, 1);
             mbar_init(empty_bar + 8 * s, 2);
         }
-        for (int g = 0; g < GROUPS; ++g) {
+        for (int g = 0; g < 2 * GROUPS; ++g) {
             mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + this CTA's table warp
-            mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS);
+            mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS / HALVES);    // the warps of the half (or of the whole group) in both CTAs
         }
         mbar_init(done_bar, 1);
         *abort_flag = 0;
+        for (int i = 0; i < 4; ++i) reinterpret_cast<uint32_t*>(base_ptr + bar_off + 512)[i] = BIAS_BITS;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -320,7 +338,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
                     const Work w = get_work(p, wi);
                     const int my_m = w.m0 + (int)rank * TILE_M;      // this CTA's A rows
-                    const int my_n = w.n0 + (int)rank * B_HALF;      // this CTA's half of the B rows
+                    const int my_n = w.n0 + (int)rank * B_BOX;       // this CTA's share of the B rows of column half 0
                     const int nst = (w.nblk + BPS - 1) >> LB;
                     int kb = w.kb0, kbyte = w.kb0 * (128 >> LB);
                     for (int si = 0; si < nst; ++si, kb += BPS, kbyte += STAGE_K, ++it) {
@@ -332,6 +350,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                         const uint32_t ms = mant_base + s * MANT_STAGE;
                         if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms, &mapA, kbyte, my_m, leader_full + 8 * s, L2_EVICT_LAST);
                         if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES, &mapB, kbyte, my_n, leader_full + 8 * s, L2_EVICT_NORMAL);
+                        if (HALVES == 2 && !(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES + B_BYTES / 2, &mapB, kbyte, my_n + N_HALF, leader_full + 8 * s, L2_EVICT_NORMAL);
                         const uint32_t es = exp_base + s * EXP_STAGE;
                         tma_load_2d(es, &mapEA, my_m, kb, efull_bar + 8 * s);
                         tma_load_2d(es + EXP_A, &mapEB, w.n0, kb, efull_bar + 8 * s);
@@ -353,32 +372,58 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             if (lane == 0 && rank == 0) {
                 constexpr uint32_t idesc = idesc_i8_pair();
                 uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
+                // The barriers the next MMAs will need are polled (without blocking) just before the last
+                // MMA of a half is issued, while earlier MMAs still occupy the tensor pipe; a barrier found
+                // complete then is not waited on again, so the pipe is refilled without a bubble.
+                bool pre_full = false, pre_tempty = false;
                 bool ok = true;
                 for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
                     const Work w = get_work(p, wi);
                     const int nst = (w.nblk + BPS - 1) >> LB;
                     int left = w.nblk;
                     for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
-                        if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 211)) { ok = false; break; }
+                        if (pre_full) pre_full = false;
+                        else if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 211)) { ok = false; break; }
                         TC2_TRACE(1, it);
                         tc_fence_after();
                         const uint32_t ms = mant_base + s * MANT_STAGE;
                         const uint64_t a_desc = smem_desc_sw128(ms), b_desc = smem_desc_sw128(ms + A_BYTES);
+                        const int nb = left < BPS ? left : BPS;       // blocks of this stage
 #pragma unroll
                         for (int jb = 0; jb < BPS; ++jb) {
-                            if (jb < left) {
-                                // the group was read and re-armed by the rescale warps of both CTAs
-                                if (!mbar_wait_cluster(tempty_bar + 8 * g, gph, abort_flag, p.status, 212)) { ok = false; break; }
-                                TC2_TRACE(2, blk);
-                                tc_fence_after();
-                                const uint32_t d = tmem_base + g * N_TILE;
+                            if (jb < nb) {
 #pragma unroll
-                                for (int q = 0; q < SPB; ++q) {
-                                    const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
-                                    if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, b_desc + ko, idesc, 1u);   // on top of the bias
+                                for (int h = 0; h < HALVES; ++h) {
+                                    // the half group was read and re-armed by its rescale warps in both CTAs
+                                    if (pre_tempty) pre_tempty = false;
+                                    else if (!mbar_wait_cluster(tempty_bar + 8 * (2 * g + h), gph, abort_flag, p.status, 212)) { ok = false; break; }
+                                    if (h == 0) TC2_TRACE(2, blk);
+                                    tc_fence_after();
+                                    const uint32_t d = tmem_base + g * N_TILE + h * N_HALF;
+                                    const uint64_t bh = b_desc + (uint64_t)(h * (B_BYTES / 2) >> 4);
+#pragma unroll
+                                    for (int q = 0; q < SPB; ++q) {
+                                        if (q == SPB - 1) {
+                                            if (h < HALVES - 1) {
+                                                pre_tempty = mbar_test_wait(tempty_bar + 8 * (2 * g + 1), gph);
+                                            } else {
+                                                uint32_t g2 = g, gph2 = gph;
+                                                ring_next<GROUPS>(g2, gph2);
+                                                pre_tempty = mbar_test_wait(tempty_bar + 8 * (2 * g2), gph2);
+                                                if (jb == nb - 1) {
+                                                    uint32_t s2 = s, ph2 = ph;
+                                                    ring_next<STAGES>(s2, ph2);
+                                                    pre_full = mbar_test_wait(full_bar + 8 * s2, ph2);
+                                                }
+                                            }
+                                        }
+                                        const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
+                                        if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, bh + ko, idesc, 1u);   // on top of the bias
+                                    }
+                                    tc_commit_pair(tfull_bar + 8 * (2 * g + h), 3);
+                                    if (h == HALVES - 1) TC2_TRACE(3, blk);
                                 }
-                                tc_commit_pair(tfull_bar + 8 * g, 3);
-                                TC2_TRACE(3, blk);
+                                if (!ok) break;
                                 ring_next<GROUPS>(g, gph);
                                 ++blk;
                             }
@@ -418,9 +463,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                             c1.x = exp_to_scale(cb.y, 0); c1.y = exp_to_scale(cb.y, 1); c1.z = exp_to_scale(cb.y, 2); c1.w = exp_to_scale(cb.y, 3);
                             r0.x = exp_to_scale(ra, 0); r0.y = exp_to_scale(ra, 1); r0.z = exp_to_scale(ra, 2); r0.w = exp_to_scale(ra, 3);
 #if HBFP_TC2_TABLE_POLL
-                            if (!mbar_poll_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
+                            if (!mbar_poll_warp(tfull_bar + 8 * (2 * g + HALVES - 1), gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
 #else
-                            if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
+                            if (!mbar_wait_warp(tfull_bar + 8 * (2 * g + HALVES - 1), gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
 #endif
                             if (lane == 0) TC2_TRACE(21, blk);
                             uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
@@ -428,7 +473,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                             *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
                             *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
+                            if (lane == 0) {
+                                mbar_arrive(tfull_bar + 8 * (2 * g));
+                                if (HALVES == 2) mbar_arrive(tfull_bar + 8 * (2 * g + 1));
+                            }
                             if (lane == 0) TC2_TRACE(22, blk);
                             ring_next<GROUPS>(g, gph);
                             slot = (slot + 1) & (TSLOTS - 1);
@@ -446,32 +494,35 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         // ------------------------------------------------------------------ rescale warps (both CTAs)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
         constexpr int COLS_PER_WARP = N_TILE / 2;            // two warps share a lane quarter and split the columns
+        constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : COLS_PER_WARP / CH;
         const int rwarp = warp - CONTROL_WARPS;              // 0..7
         const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4
         const int row = quarter * 32 + lane;                 // row of this CTA's half tile = tensor-memory lane
         const int col0 = half * COLS_PER_WARP;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         const uint32_t leader_tempty = map_to_rank(tempty_bar, 0);
+        const int hb = HALVES == 2 ? half : 0;               // which of the group's barriers this warp uses
         uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
-        uint32_t bias[8];
+        {
+            uint32_t bias[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
-        for (int g = 0; g < GROUPS; ++g)
+            for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
+            for (int g = 0; g < GROUPS; ++g)
 #pragma unroll
-            for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
-        tc_wait_st();
-        // Read the bias back as one eight-register tuple: a tuple that is born as such is passed to
-        // every re-arming store in place, while eight separately defined registers would be copied
-        // into a fresh tuple for each store (eight extra instructions per store).
-        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                     : "=r"(bias[0]), "=r"(bias[1]), "=r"(bias[2]), "=r"(bias[3]), "=r"(bias[4]), "=r"(bias[5]), "=r"(bias[6]), "=r"(bias[7])
-                     : "r"(lane_addr) : "memory");
+                for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
+            tc_wait_st();
+        }
+        // Read the bias back as one sixteen-register tuple: a tuple that is born as such is passed to
+        // every re-arming store in place, while separately defined registers are copied into a fresh
+        // tuple for each store (one extra instruction per register and store).
+        uint32_t bias16[16];
+        tc_ld16(lane_addr, bias16);
         tc_wait_ld();
         // every accumulator group starts out free
         tc_fence_before();
         __syncwarp();
         if (lane == 0)
-            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * g);
+            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * (2 * g + hb));
 
         uint32_t g = 0, gph = 0, slot = 0, blk = 0;
         bool ok = true;
@@ -481,11 +532,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
             for (int kb = 0; kb < w.nblk; ++kb, ++blk) {
-                // one wait per block: the block sums are complete and this CTA's scale table is written
-                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 312)) { ok = false; break; }
-                if (lane == 0) TC2_TRACE(4 + rwarp, blk);
-                tc_fence_after();
                 const uint32_t taddr = lane_addr + g * N_TILE;
+                uint32_t v[2][CH];
+                // one wait per block: the block sums are complete and this CTA's scale table is written
+                if (!mbar_wait_warp(tfull_bar + 8 * (2 * g + hb), gph, abort_flag, p.status, 312)) { ok = false; break; }
+                tc_fence_after();
+                if (NCHK) tc_ldn(taddr, v[0]);
+                if (lane == 0) TC2_TRACE(4 + rwarp, blk);
                 const uint32_t* tab = tables + slot * TABLE_SLOT_WORDS + col0;
                 // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
                 // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
@@ -493,9 +546,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 const float ca_f = -12582912.0f * sa_f;
                 const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
                 const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
-                constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : COLS_PER_WARP / CH;
-                uint32_t v[2][CH];
-                if (NCHK) tc_ldn(taddr, v[0]);
 #pragma unroll
                 for (int ch = 0; ch < NCHK; ++ch) {
                     tc_wait_ld();
@@ -509,15 +559,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                         acc2[(ch * CH + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
                         acc2[(ch * CH + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CH + q) / 2 + 1]);
                     }
-#pragma unroll
-                    for (int c8 = 0; c8 < CH / 8; ++c8) tc_st8(taddr + ch * CH + c8 * 8, bias);   // re-arm
+#if !(HBFP_TC2_PROBE & 16)
+                    tc_st16(taddr + ch * CH, bias16);          // re-arm
+#endif
                 }
-                if (lane == 0 && rwarp == 0) TC2_TRACE(29, blk);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_remote(leader_tempty + 8 * g);
+                    mbar_arrive_remote(leader_tempty + 8 * (2 * g + hb));
                     TC2_TRACE(12 + rwarp, blk);
                 }
                 ring_next<GROUPS>(g, gph);
@@ -618,7 +668,7 @@ int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed&
     int rc;
     rc = make_map(&mA, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
     if (rc) return rc;
-    rc = make_map(&mB, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, B_HALF, true);
+    rc = make_map(&mB, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, B_BOX, true);
     if (rc) return rc;
     rc = make_map(&mEA, a.exps, a.L.rs, a.L.nkb, a.L.rs, TILE_M, 4, false);
     if (rc) return rc;
