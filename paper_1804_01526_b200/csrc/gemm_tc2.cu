@@ -13,9 +13,13 @@
 //
 // Barriers. Mantissa tiles of both CTAs complete on the leader's full[s]; exponent slices on a
 // local efull[s]; the leader's MMA thread commits to tfull[g] and empty[s] of both CTAs; the
-// rescale warps of both CTAs arrive on the leader's tempty[g]. Every wait is bounded: when one
-// expires the CTA records a code in the device status word, raises its abort flag, drains what
-// it can wait for and leaves through the common teardown (cluster barrier, tensor memory freed).
+// rescale warps of both CTAs arrive on the leader's tempty[g]. A rescale warp does one wait and
+// one arrival per K-block: the table warp's "scales written" arrival is counted on tfull[g]
+// together with the MMA commit, and the table warp learns that a table slot is free again from
+// the completion of tfull two blocks back (the MMAs of that block were issued only after every
+// rescale warp had finished the slot's last reader). Every wait is bounded: when one expires the
+// CTA records a code in the device status word, raises its abort flag, drains what it can wait
+// for and leaves through the common teardown (cluster barrier, tensor memory freed).
 #include <cuda.h>
 
 #include "common.cuh"
@@ -26,25 +30,13 @@ namespace {
 
 constexpr int N_TILE = 256;            // columns of the pair tile = accumulator columns per CTA
 constexpr int PAIR_M = 2 * TILE_M;     // rows of the pair tile
-#ifndef HBFP_TC2_HALVES
-#define HBFP_TC2_HALVES 1
-#endif
-constexpr int HALVES = HBFP_TC2_HALVES; // 2: the tile is computed as two column halves with their own barriers; 1: as a whole
-constexpr int N_HALF = N_TILE / HALVES; // columns of one MMA
-constexpr int B_HALF = N_TILE / 2;      // B rows staged in each CTA
-constexpr int B_BOX = N_HALF / 2;       // rows of one B copy (this CTA's share of one MMA's columns)
+constexpr int B_HALF = N_TILE / 2;     // B rows staged in each CTA
 constexpr int RESCALE_WARPS = 8;
 constexpr int CONTROL_WARPS = 4;
-#ifndef HBFP_TC2_TABLE_WARP
-#define HBFP_TC2_TABLE_WARP 2
-#endif
-constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = HBFP_TC2_TABLE_WARP;
+constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = 2;
 constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
 // setmaxnreg totals must not exceed the launch allocation (384 threads x 168 registers)
-#ifndef HBFP_TC2_REGS_RESCALE
-#define HBFP_TC2_REGS_RESCALE 216
-#endif
-constexpr int REGS_RESCALE = HBFP_TC2_REGS_RESCALE, REGS_CONTROL = (384 * 168 - 256 * HBFP_TC2_REGS_RESCALE) / 128 / 8 * 8;
+constexpr int REGS_RESCALE = 216, REGS_CONTROL = 72;
 static_assert(128 * REGS_CONTROL + 256 * REGS_RESCALE <= 384 * 168, "register split");
 
 constexpr int GROUPS = TMEM_COLS / N_TILE;                  // 2 accumulator groups
@@ -65,15 +57,6 @@ constexpr int CH = 16;                                      // columns per tenso
 // 4 = no mantissa tile is copied, 8 = cluster 0 records per-role timestamps.
 #ifndef HBFP_TC2_PROBE
 #define HBFP_TC2_PROBE 0
-#endif
-#ifndef HBFP_TC2_ARRIVE
-#define HBFP_TC2_ARRIVE 0
-#endif
-#ifndef HBFP_TC2_TABLE_POLL
-#define HBFP_TC2_TABLE_POLL 1
-#endif
-#ifndef HBFP_TC2_WAIT
-#define HBFP_TC2_WAIT 0
 #endif
 
 struct Problem {
@@ -152,30 +135,21 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     return r;
 }
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-#if HBFP_TC2_ARRIVE == 0
     // release at CTA scope: what the arrival has to order are this warp's tensor-memory accesses, and
     // tcgen05.wait + tcgen05.fence::before_thread_sync do that; a cluster-scope release costs ~1000 cycles
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-#else
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-#endif
 }
 __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
 }
 
-// Wait on a barrier that threads of the other CTA arrive on (acquire at cluster scope).
+// Wait on a barrier that threads of the other CTA arrive on. What the arrivals order are tensor-memory
+// accesses, fenced with tcgen05.fence on both sides, so the default (CTA-scope) acquire is enough.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-#if HBFP_TC_TESTWAIT
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#elif HBFP_TC2_WAIT == 0
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-#else
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
     return ok != 0;
@@ -194,30 +168,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
             return false;
         }
     }
-}
-
-// Bounded polling wait (test_wait + nanosleep) for a whole warp: used where a suspended try_wait
-// would sit on a barrier that other warps of the same sub-partition are suspended on too.
-__device__ __forceinline__ bool mbar_poll_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
-    bool ok = true;
-    uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (!done) {
-        const long long t0 = clock64();
-        for (;;) {
-            __nanosleep(64);
-            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-            if (done) break;
-            if (*abort_flag) { ok = false; break; }
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicCAS(status, 0, code);
-                ok = false;
-                break;
-            }
-        }
-    }
-    return __all_sync(0xffffffffu, ok);
 }
 
 // Non-blocking look at a barrier phase.
@@ -250,7 +200,7 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) 
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(cta_mask) : "memory");
 }
 __device__ __forceinline__ constexpr uint32_t idesc_i8_pair() {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_HALF >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
 }
 
 // 2^e as binary32 bits, e = signed byte i of a packed word of four exponents.
@@ -287,11 +237,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t full_bar = bars;                          // leader: mantissa tiles of both CTAs landed
     const uint32_t efull_bar = full_bar + 8 * STAGES;        // local: exponent slices landed
     const uint32_t empty_bar = efull_bar + 8 * STAGES;       // local: stage consumed (MMA commit + table warp)
-    // accumulator barriers exist per group and column half: index 2 * g + h
-    const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums of a half complete (MMA commit) and scale table written
-    const uint32_t tempty_bar = tfull_bar + 16 * GROUPS;     // leader: half group read and re-armed by its warps in both CTAs
-    const uint32_t done_bar = tempty_bar + 16 * GROUPS;
-    constexpr int BAR_BYTES = 24 * STAGES + 32 * GROUPS + 8;
+    const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums complete (MMA commit) and scale table written
+    const uint32_t tempty_bar = tfull_bar + 8 * GROUPS;      // leader: group read and re-armed by the rescale warps of both CTAs
+    const uint32_t done_bar = tempty_bar + 8 * GROUPS;
+    constexpr int BAR_BYTES = 24 * STAGES + 16 * GROUPS + 8;
     static_assert(BAR_BYTES + 8 <= 1024, "barrier area");
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + BAR_BYTES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -307,13 +256,12 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             mbar_init(efull_bar + 8 * s, 1);
             mbar_init(empty_bar + 8 * s, 2);
         }
-        for (int g = 0; g < 2 * GROUPS; ++g) {
+        for (int g = 0; g < GROUPS; ++g) {
             mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + this CTA's table warp
-            mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS / HALVES);    // the warps of the half (or of the whole group) in both CTAs
+            mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS);
         }
         mbar_init(done_bar, 1);
         *abort_flag = 0;
-        for (int i = 0; i < 4; ++i) reinterpret_cast<uint32_t*>(base_ptr + bar_off + 512)[i] = BIAS_BITS;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -338,7 +286,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
                     const Work w = get_work(p, wi);
                     const int my_m = w.m0 + (int)rank * TILE_M;      // this CTA's A rows
-                    const int my_n = w.n0 + (int)rank * B_BOX;       // this CTA's share of the B rows of column half 0
+                    const int my_n = w.n0 + (int)rank * B_HALF;      // this CTA's half of the B rows
                     const int nst = (w.nblk + BPS - 1) >> LB;
                     int kb = w.kb0, kbyte = w.kb0 * (128 >> LB);
                     for (int si = 0; si < nst; ++si, kb += BPS, kbyte += STAGE_K, ++it) {
@@ -350,7 +298,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                         const uint32_t ms = mant_base + s * MANT_STAGE;
                         if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms, &mapA, kbyte, my_m, leader_full + 8 * s, L2_EVICT_LAST);
                         if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES, &mapB, kbyte, my_n, leader_full + 8 * s, L2_EVICT_NORMAL);
-                        if (HALVES == 2 && !(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES + B_BYTES / 2, &mapB, kbyte, my_n + N_HALF, leader_full + 8 * s, L2_EVICT_NORMAL);
                         const uint32_t es = exp_base + s * EXP_STAGE;
                         tma_load_2d(es, &mapEA, my_m, kb, efull_bar + 8 * s);
                         tma_load_2d(es + EXP_A, &mapEB, w.n0, kb, efull_bar + 8 * s);
@@ -373,7 +320,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 constexpr uint32_t idesc = idesc_i8_pair();
                 uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
                 // The barriers the next MMAs will need are polled (without blocking) just before the last
-                // MMA of a half is issued, while earlier MMAs still occupy the tensor pipe; a barrier found
+                // MMA of a block is issued, while earlier MMAs still occupy the tensor pipe; a barrier found
                 // complete then is not waited on again, so the pipe is refilled without a bubble.
                 bool pre_full = false, pre_tempty = false;
                 bool ok = true;
@@ -392,38 +339,30 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 #pragma unroll
                         for (int jb = 0; jb < BPS; ++jb) {
                             if (jb < nb) {
+                                // the group was read and re-armed by the rescale warps of both CTAs
+                                if (pre_tempty) pre_tempty = false;
+                                else if (!mbar_wait_cluster(tempty_bar + 8 * g, gph, abort_flag, p.status, 212)) { ok = false; break; }
+                                TC2_TRACE(2, blk);
+                                tc_fence_after();
+                                const uint32_t d = tmem_base + g * N_TILE;
 #pragma unroll
-                                for (int h = 0; h < HALVES; ++h) {
-                                    // the half group was read and re-armed by its rescale warps in both CTAs
-                                    if (pre_tempty) pre_tempty = false;
-                                    else if (!mbar_wait_cluster(tempty_bar + 8 * (2 * g + h), gph, abort_flag, p.status, 212)) { ok = false; break; }
-                                    if (h == 0) TC2_TRACE(2, blk);
-                                    tc_fence_after();
-                                    const uint32_t d = tmem_base + g * N_TILE + h * N_HALF;
-                                    const uint64_t bh = b_desc + (uint64_t)(h * (B_BYTES / 2) >> 4);
-#pragma unroll
-                                    for (int q = 0; q < SPB; ++q) {
-                                        if (q == SPB - 1) {
-                                            if (h < HALVES - 1) {
-                                                pre_tempty = mbar_test_wait(tempty_bar + 8 * (2 * g + 1), gph);
-                                            } else {
-                                                uint32_t g2 = g, gph2 = gph;
-                                                ring_next<GROUPS>(g2, gph2);
-                                                pre_tempty = mbar_test_wait(tempty_bar + 8 * (2 * g2), gph2);
-                                                if (jb == nb - 1) {
-                                                    uint32_t s2 = s, ph2 = ph;
-                                                    ring_next<STAGES>(s2, ph2);
-                                                    pre_full = mbar_test_wait(full_bar + 8 * s2, ph2);
-                                                }
-                                            }
+                                for (int q = 0; q < SPB; ++q) {
+                                    if (q == SPB - 1) {
+                                        // look ahead while the tensor pipe still has the earlier MMAs to run
+                                        uint32_t g2 = g, gph2 = gph;
+                                        ring_next<GROUPS>(g2, gph2);
+                                        pre_tempty = mbar_test_wait(tempty_bar + 8 * g2, gph2);
+                                        if (jb == nb - 1) {
+                                            uint32_t s2 = s, ph2 = ph;
+                                            ring_next<STAGES>(s2, ph2);
+                                            pre_full = mbar_test_wait(full_bar + 8 * s2, ph2);
                                         }
-                                        const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
-                                        if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, bh + ko, idesc, 1u);   // on top of the bias
                                     }
-                                    tc_commit_pair(tfull_bar + 8 * (2 * g + h), 3);
-                                    if (h == HALVES - 1) TC2_TRACE(3, blk);
+                                    const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
+                                    if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, b_desc + ko, idesc, 1u);   // on top of the bias
                                 }
-                                if (!ok) break;
+                                tc_commit_pair(tfull_bar + 8 * g, 3);
+                                TC2_TRACE(3, blk);
                                 ring_next<GROUPS>(g, gph);
                                 ++blk;
                             }
@@ -462,21 +401,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                             c0.x = exp_to_scale(cb.x, 0); c0.y = exp_to_scale(cb.x, 1); c0.z = exp_to_scale(cb.x, 2); c0.w = exp_to_scale(cb.x, 3);
                             c1.x = exp_to_scale(cb.y, 0); c1.y = exp_to_scale(cb.y, 1); c1.z = exp_to_scale(cb.y, 2); c1.w = exp_to_scale(cb.y, 3);
                             r0.x = exp_to_scale(ra, 0); r0.y = exp_to_scale(ra, 1); r0.z = exp_to_scale(ra, 2); r0.w = exp_to_scale(ra, 3);
-#if HBFP_TC2_TABLE_POLL
-                            if (!mbar_poll_warp(tfull_bar + 8 * (2 * g + HALVES - 1), gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
-#else
-                            if (!mbar_wait_warp(tfull_bar + 8 * (2 * g + HALVES - 1), gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
-#endif
+                            if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
                             if (lane == 0) TC2_TRACE(21, blk);
                             uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
                             *reinterpret_cast<uint4*>(tb + 8 * lane) = c0;
                             *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
                             *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
                             __syncwarp();
-                            if (lane == 0) {
-                                mbar_arrive(tfull_bar + 8 * (2 * g));
-                                if (HALVES == 2) mbar_arrive(tfull_bar + 8 * (2 * g + 1));
-                            }
+                            if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
                             if (lane == 0) TC2_TRACE(22, blk);
                             ring_next<GROUPS>(g, gph);
                             slot = (slot + 1) & (TSLOTS - 1);
@@ -501,7 +433,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int col0 = half * COLS_PER_WARP;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         const uint32_t leader_tempty = map_to_rank(tempty_bar, 0);
-        const int hb = HALVES == 2 ? half : 0;               // which of the group's barriers this warp uses
         uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
         {
             uint32_t bias[8];
@@ -522,7 +453,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         tc_fence_before();
         __syncwarp();
         if (lane == 0)
-            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * (2 * g + hb));
+            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * g);
 
         uint32_t g = 0, gph = 0, slot = 0, blk = 0;
         bool ok = true;
@@ -535,7 +466,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 const uint32_t taddr = lane_addr + g * N_TILE;
                 uint32_t v[2][CH];
                 // one wait per block: the block sums are complete and this CTA's scale table is written
-                if (!mbar_wait_warp(tfull_bar + 8 * (2 * g + hb), gph, abort_flag, p.status, 312)) { ok = false; break; }
+                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 312)) { ok = false; break; }
                 tc_fence_after();
                 if (NCHK) tc_ldn(taddr, v[0]);
                 if (lane == 0) TC2_TRACE(4 + rwarp, blk);
@@ -567,7 +498,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_remote(leader_tempty + 8 * (2 * g + hb));
+                    mbar_arrive_remote(leader_tempty + 8 * g);
                     TC2_TRACE(12 + rwarp, blk);
                 }
                 ring_next<GROUPS>(g, gph);
@@ -668,7 +599,7 @@ int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed&
     int rc;
     rc = make_map(&mA, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
     if (rc) return rc;
-    rc = make_map(&mB, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, B_BOX, true);
+    rc = make_map(&mB, b.mant, b.L.kst, b.L.rows, b.L.kst, STAGE_K, B_HALF, true);
     if (rc) return rc;
     rc = make_map(&mEA, a.exps, a.L.rs, a.L.nkb, a.L.rs, TILE_M, 4, false);
     if (rc) return rc;
