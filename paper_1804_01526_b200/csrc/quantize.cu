@@ -7,13 +7,17 @@
 //                    thread (two 128-bit loads, one Philox call in stochastic mode), block
 //                    max by warp shuffles, exponents staged in shared memory so that the
 //                    [kb][row] exponent array is written in full 32-byte sectors.
-//   quant_col_fast   blocks down the columns, b <= 128: a (<=128) x 32 FP32 panel is read with
-//                    coalesced row loads into shared memory, reduced down the columns by four
-//                    threads per column and written transposed (contraction-major again).
+//   quant_col_tma    blocks down the columns, b in {32,64,128}, 16-byte aligned pitch: persistent
+//                    CTAs stream 128 x 64 FP32 tiles through a TMA pipeline and write the packed,
+//                    transposed tile with a swizzled TMA store (full lines in both directions).
+//   quant_col_fast   blocks down the columns, any b <= 128 and any pitch: a (<=128) x 32 FP32
+//                    panel is read with coalesced row loads into shared memory, reduced down the
+//                    columns by four threads per column and written transposed.
 //   quant_tiles      t x t weight tiles (t <= 128): one pass writes both packed views and
 //                    the tile exponent grid.
 //   exps_* / mant_generic   two-pass path for every other geometry (any b, any alignment).
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace hbfp {
 namespace {
@@ -504,6 +508,173 @@ __global__ void dequant_kernel(const int8_t* __restrict__ mant, const int8_t* __
     out[r * ld + kk] = ldexpf((float)v, (int)exps[kb * rs + r]);
 }
 
+// ------------------------------------------------------------------------------ quant_col_tma
+
+// Blocks down the columns of x [K][R] for b in {32, 64, 128}, the layout of the B operand of a
+// forward GEMM. Persistent CTAs stream 128 (k) x 64 (columns) FP32 tiles through a two-stage TMA
+// pipeline; thread (column n, quarter q) keeps 32 consecutive k of its column in registers between
+// the block maximum and the rounding pass, and the packed tile (64 output rows x 128 mantissa bytes,
+// contraction-major) goes back to global memory as one 128B-swizzled TMA store per plane, so both
+// directions move full lines whatever the matrix pitch.
+constexpr int QC_COLS = 64, QC_ROWS = 128, QC_STAGES = 2, QC_THREADS = 256;
+constexpr int QC_IN_BYTES = QC_ROWS * QC_COLS * 4;          // 32 KB
+constexpr int QC_OUT_BYTES = QC_COLS * QC_ROWS;             // 8 KB per plane
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+
+template <int PLANES, int LB, bool SR>      // b = 128 >> LB
+__global__ void __launch_bounds__(QC_THREADS)
+quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapM0,
+              const __grid_constant__ CUtensorMap mapM1, QParams p, int8_t* __restrict__ exps, int64_t rs,
+              int64_t nkb, int64_t K, int64_t R, int tiles_n, int total_tiles, int32_t* status) {
+    extern __shared__ unsigned char smem_dyn[];
+    const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+    // [out planes | in stages | draws (stochastic) | block maxima | barriers]
+    constexpr int OFF_IN = PLANES * QC_OUT_BYTES;
+    constexpr int OFF_RND = OFF_IN + QC_STAGES * QC_IN_BYTES;
+    constexpr int OFF_PMAX = OFF_RND + (SR ? QC_ROWS * QC_COLS * 2 : 0);
+    constexpr int OFF_BAR = OFF_PMAX + 4 * QC_COLS * 4;
+    const float* in = reinterpret_cast<const float*>(base_ptr + OFF_IN);
+    uint4* rnd = reinterpret_cast<uint4*>(base_ptr + OFF_RND);
+    uint32_t* pmax = reinterpret_cast<uint32_t*>(base_ptr + OFF_PMAX);
+    const uint32_t full_bar = base + OFF_BAR;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_BAR + 8 * QC_STAGES);
+
+    const int tid = threadIdx.x, n = tid & (QC_COLS - 1), q = tid >> 6;
+    if (tid == 0) {
+        for (int s = 0; s < QC_STAGES; ++s) mbar_init(full_bar + 8 * s, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const int first = blockIdx.x, step = gridDim.x;
+    if (tid == 0) {
+        for (int s = 0; s < QC_STAGES; ++s) {
+            const int t = first + s * step;
+            if (t < total_tiles) {
+                mbar_expect_tx(full_bar + 8 * s, QC_IN_BYTES);
+                tma_load_2d(base + OFF_IN + s * QC_IN_BYTES, &mapX, (t % tiles_n) * (QC_COLS * 4), (t / tiles_n) * QC_ROWS, full_bar + 8 * s);
+            }
+        }
+    }
+    uint32_t s = 0, ph = 0;
+    bool stores_pending = false;
+    for (int t = first; t < total_tiles; t += step) {
+        const int nt = t % tiles_n, kt = t / tiles_n;
+        const int64_t col = (int64_t)nt * QC_COLS + n;
+        // (uniform verdict: a wait that gave up in some threads only would split the CTA barriers below)
+        if (!__syncthreads_and(mbar_wait(full_bar + 8 * s, ph, abort_flag, status, 601))) break;
+        const float* tile = in + (size_t)s * (QC_IN_BYTES / 4);
+        if (SR) {
+            // one Philox call per eight consecutive source elements of a row (R % 8 == 0 here)
+            for (int i = tid; i < QC_ROWS * (QC_COLS / 8); i += QC_THREADS) {
+                const uint64_t L = (uint64_t)((int64_t)kt * QC_ROWS + (i >> 3)) * (uint64_t)R + (uint64_t)(nt * QC_COLS + (i & 7) * 8);
+                rnd[i] = draws_of_group(p, L >> 3);
+            }
+        }
+        float v[32];
+        uint32_t am = 0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            v[j] = tile[(q * 32 + j) * QC_COLS + n];
+            am = max(am, abs_bits(v[j]));
+        }
+        if (LB < 2) pmax[q * QC_COLS + n] = am;
+        // the packed tile of the previous iteration must have left shared memory before it is rewritten
+        if (tid == 0 && stores_pending) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncthreads();
+        // every thread holds its values in registers now: refill this stage with the tile after next
+        if (tid == 0) {
+            const int t2 = t + QC_STAGES * step;
+            if (t2 < total_tiles) {
+                mbar_expect_tx(full_bar + 8 * s, QC_IN_BYTES);
+                tma_load_2d(base + OFF_IN + s * QC_IN_BYTES, &mapX, (t2 % tiles_n) * (QC_COLS * 4), (t2 / tiles_n) * QC_ROWS, full_bar + 8 * s);
+            }
+        }
+        if (LB == 0) am = max(max(pmax[n], pmax[QC_COLS + n]), max(pmax[2 * QC_COLS + n], pmax[3 * QC_COLS + n]));
+        if (LB == 1) am = max(pmax[(q & 2) * QC_COLS + n], pmax[((q & 2) + 1) * QC_COLS + n]);
+        const int sexp = block_exponent(am, p.m, p.exp_mode);
+        const int64_t kb = ((int64_t)kt << LB) + (q >> (2 - LB));
+        if ((q & ((4 >> LB) - 1)) == 0 && kb < nkb && col < R) exps[kb * rs + col] = (int8_t)sexp;
+
+        uint32_t hi[8], lo[8];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { hi[w] = 0; lo[w] = 0; }
+        const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            int qv;
+            if (SR) qv = round_sr(v[j], sexp, p.qmax, rnd16[(q * 32 + j) * QC_COLS + n]);
+            else qv = round_rne(v[j], sexp, p.qmax);
+            if (PLANES == 1) {
+                hi[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
+            } else {
+                hi[j >> 2] |= (uint32_t)((qv >> 4) & 0xff) << (8 * (j & 3));
+                lo[j >> 2] |= (uint32_t)(qv & 15) << (8 * (j & 3));
+            }
+        }
+        // 128B swizzle of the store tile: 16-byte chunk c of row n sits at chunk position c ^ (n % 8)
+        unsigned char* orow = base_ptr + (n >> 3) * 1024 + (n & 7) * 128;
+        const int c0 = ((2 * q) ^ (n & 7)) << 4, c1 = ((2 * q + 1) ^ (n & 7)) << 4;
+        *reinterpret_cast<uint4*>(orow + c0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(orow + c1) = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+        if (PLANES == 2) {
+            *reinterpret_cast<uint4*>(orow + QC_OUT_BYTES + c0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+            *reinterpret_cast<uint4*>(orow + QC_OUT_BYTES + c1) = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncthreads();
+        if (tid == 0) {
+            tma_store_2d(&mapM0, kt * QC_ROWS, nt * QC_COLS, base);
+            if (PLANES == 2) tma_store_2d(&mapM1, kt * QC_ROWS, nt * QC_COLS, base + QC_OUT_BYTES);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        stores_pending = true;
+        if (++s == QC_STAGES) { s = 0; ph ^= 1u; }
+    }
+    // the stores must be complete when the CTA leaves (a load still in flight after an abandoned
+    // wait has had the whole wait budget, seconds, to land)
+    if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+template <int PLANES, int LB, bool SR>
+int launch_col_tma(const float* x, int64_t K, int64_t rows, int64_t ld, const QParams& p, const Layout& L,
+                   int8_t* mant, int8_t* exps, cudaStream_t st) {
+    CUtensorMap mX, mM0, mM1;
+    int rc = make_map(&mX, x, (uint64_t)rows * 4, (uint64_t)K, (uint64_t)ld * 4, QC_COLS * 4, QC_ROWS, false);
+    if (rc) return rc;
+    rc = make_map(&mM0, mant, (uint64_t)L.kst, (uint64_t)rows, (uint64_t)L.kst, QC_ROWS, QC_COLS, true);
+    if (rc) return rc;
+    mM1 = mM0;
+    if (PLANES == 2) {
+        rc = make_map(&mM1, mant + L.plane_stride, (uint64_t)L.kst, (uint64_t)rows, (uint64_t)L.kst, QC_ROWS, QC_COLS, true);
+        if (rc) return rc;
+    }
+    constexpr int smem = 1024 + PLANES * QC_OUT_BYTES + QC_STAGES * QC_IN_BYTES + (SR ? QC_ROWS * QC_COLS * 2 : 0) +
+                         4 * QC_COLS * 4 + 64;
+    static int ctas_per_sm = 0;
+    if (!ctas_per_sm) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_tma<PLANES, LB, SR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        int nb = 0;
+        HBFP_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, quant_col_tma<PLANES, LB, SR>, QC_THREADS, smem));
+        ctas_per_sm = nb > 0 ? nb : 1;
+    }
+    int32_t* status = device_status_word();
+    if (!status) return HBFP_ERR_CUDA;
+    const int64_t tiles_n = (rows + QC_COLS - 1) / QC_COLS, tiles_k = L.kst / QC_ROWS;
+    const int64_t total = tiles_n * tiles_k;
+    const int64_t cap = (int64_t)sm_count() * ctas_per_sm;
+    const int grid = (int)(total < cap ? total : cap);
+    quant_col_tma<PLANES, LB, SR><<<grid, QC_THREADS, smem, st>>>(mX, mM0, mM1, p, exps, L.rs, L.nkb, K, rows, (int)tiles_n,
+                                                              (int)total, status);
+    return launch_status();
+}
+
 QParams make_params(const hbfp_format* f) {
     QParams p;
     p.m = f->mant_bits;
@@ -562,6 +733,18 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
             case 256: return launch_row_fast<32>(x, rows, K, ld, p, L, mant, exps, st);
             default: break;
         }
+    }
+    if (f->tile == 0 && axis == 0 && aligned && L.b == L.bp && L.b <= 128 && (p.rounding == 0 || rows % 8 == 0) &&
+        (reinterpret_cast<uintptr_t>(mant) & 127) == 0 && rows < (1ll << 29) && K < (1ll << 31) &&
+        ((rows + QC_COLS - 1) / QC_COLS) * (L.kst / QC_ROWS) < (1ll << 31)) {
+        // exponent padding bytes (lines >= rows) are documented as zero
+        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+#define HBFP_QCOL_TMA(PL, LBV) (p.rounding ? launch_col_tma<PL, LBV, true>(x, K, rows, ld, p, L, mant, exps, st) \
+                                           : launch_col_tma<PL, LBV, false>(x, K, rows, ld, p, L, mant, exps, st))
+        const int lb = L.b == 128 ? 0 : L.b == 64 ? 1 : 2;
+        if (L.planes == 1) return lb == 0 ? HBFP_QCOL_TMA(1, 0) : lb == 1 ? HBFP_QCOL_TMA(1, 1) : HBFP_QCOL_TMA(1, 2);
+        return lb == 0 ? HBFP_QCOL_TMA(2, 0) : lb == 1 ? HBFP_QCOL_TMA(2, 1) : HBFP_QCOL_TMA(2, 2);
+#undef HBFP_QCOL_TMA
     }
     if (f->tile == 0 && axis == 0 && L.b <= 128) {
         const int vec_ok = aligned && (rows % 4 == 0);

@@ -72,6 +72,41 @@ def test_column_blocks_transposed_output(hb, shape, law, fd):
     _check(hb, wl.draw(law, shape, seed=12), 0, fd)
 
 
+# The streaming column kernel (128 x 64 tiles through a TMA pipeline) takes b in {32, 64, 128} with a
+# 16-byte aligned pitch: several tiles per CTA, ragged last tiles in both directions, fewer rows than
+# one tile, both plane counts, both rounding modes, every blocks-per-tile variant.
+COL_STREAM_CASES = [
+    ((4096, 2048), "lognormal", F(8, 128)),                                 # 1024 tiles: the persistent loop wraps
+    ((3000, 1096), "grad", F(8, 64, rounding=1, seed=8, sid=1)),            # ragged K and N, N % 8 == 0
+    ((1111, 520), "outliers", F(12, 32, rounding=1, seed=2)),               # two planes, stochastic
+    ((90, 72), "normal", F(12, 128)),                                       # less than one tile
+    ((640, 4), "half_normal", F(8, 64)),                                    # four output rows
+    ((2048, 640), "lognormal", F(6, 32, rounding=1, seed=13, exp_mode=1)),
+]
+
+
+@pytest.mark.parametrize("shape,law,fd", COL_STREAM_CASES)
+def test_column_blocks_streaming_kernel(hb, shape, law, fd):
+    _check(hb, wl.draw(law, shape, seed=14), 0, fd)
+
+
+def test_column_blocks_of_a_pitched_view(hb):
+    # a 16-byte aligned column window of a wider matrix: the pitch differs from the logical width,
+    # and the stochastic stream follows the logical index of the window
+    base = wl.draw("lognormal", (700, 1024), seed=15)
+    xd = to_dev(base)
+    for sl in (np.s_[:, 256:896], np.s_[60:, 128:392]):
+        ref = np.ascontiguousarray(base[sl])
+        for fd in (F(8, 128, rounding=1, seed=3), F(12, 64)):
+            q_ref, s_ref = oracle.quantize(ref, 0, ofmt(fd))
+            p = hb.quantize(xd[sl], 0, gfmt(fd))
+            q, s = hb.unpack(p)
+            assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+            qd, sd = decode_packed(p, hb.packed_layout(p.rows, p.k, p.fmt))
+            assert np.array_equal(qd, q_ref) and np.array_equal(sd, s_ref)
+    assert hb.device_status() == 0
+
+
 def test_strided_and_unaligned_inputs(hb):
     import torch
     base = wl.draw("lognormal", (50, 203), seed=3)
