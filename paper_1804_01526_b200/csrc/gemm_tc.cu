@@ -45,15 +45,7 @@ namespace {
 #define HBFP_TC_PROBE 0
 #endif
 
-// 1: packed two-wide FP32 FMAs in the rescale; 0: scalar FMAs.
-#ifndef HBFP_TC_FFMA2
-#define HBFP_TC_FFMA2 1
-#endif
-
-#ifndef HBFP_TC_RWARPS
-#define HBFP_TC_RWARPS 8              // rescale warps: 8 (two per sub-partition) or 16 (four)
-#endif
-constexpr int RESCALE_WARPS = HBFP_TC_RWARPS;
+constexpr int RESCALE_WARPS = 8;                   // two per sub-partition
 constexpr int COL_GROUPS = RESCALE_WARPS / 4;      // warps sharing a lane quarter split the columns
 // The control warps take the lowest warp ids: the issue logic favours them over the rescale
 // warps of the same sub-partition, and a starved MMA issuer stalls the whole pipeline.
@@ -61,19 +53,11 @@ constexpr int CONTROL_WARPS = 4;      // one warpgroup: producer, MMA issuer, ta
 constexpr int PRODUCER_WARP = 0;
 constexpr int MMA_WARP = 1;
 constexpr int TABLE_WARP = 2;
-constexpr int THREADS = 32 * (4 + RESCALE_WARPS);
-#ifndef HBFP_TC_REGS_RESCALE
-#define HBFP_TC_REGS_RESCALE (HBFP_TC_RWARPS == 8 ? 208 : 104)
-#endif
-#ifndef HBFP_TC_CHUNK
-#define HBFP_TC_CHUNK 16          // columns per tensor-memory load in the fast rescale path (16 or 32)
-#endif
-// setmaxnreg totals must never exceed what the launch allocated (threads x registers at launch,
-// 384 x 168 or 640 x 96): a request the register file cannot satisfy blocks forever.
-constexpr int REGS_LAUNCH_TOTAL = RESCALE_WARPS == 8 ? 384 * 168 : 640 * 96;
-constexpr int REGS_RESCALE = HBFP_TC_REGS_RESCALE;
-constexpr int REGS_CONTROL = ((REGS_LAUNCH_TOTAL - 32 * RESCALE_WARPS * REGS_RESCALE) / 128) / 8 * 8;
-static_assert(REGS_CONTROL >= 24 && 128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= REGS_LAUNCH_TOTAL, "register split");
+constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
+// setmaxnreg totals must never exceed what the launch allocated (384 threads x 168 registers): a
+// request the register file cannot satisfy blocks forever.
+constexpr int REGS_RESCALE = 216, REGS_CONTROL = 72;
+static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= 384 * 168, "register split");
 
 template <int N_TILE, int PLANES>
 struct Cfg {
@@ -85,8 +69,8 @@ struct Cfg {
     static constexpr int MANT_STAGE = PLANES * (A_BYTES + B_BYTES);
     static constexpr int EXP_A = 4 * TILE_M, EXP_B = 4 * N_TILE;
     static constexpr int EXP_STAGE = EXP_A + EXP_B;
-    // scale tables: a ring of TABLE_SLOTS blocks, each [N_TILE column scales][128 row scales], 32-bit
-    static constexpr int TABLE_SLOTS = 4;
+    // scale tables: a ring of 2 * GROUPS blocks, each [N_TILE column scales][128 row scales], 32-bit
+    static constexpr int TABLE_SLOTS = 2 * GROUPS;
     static constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
     static constexpr int TABLE_BYTES = 4 * TABLE_SLOTS * TABLE_SLOT_WORDS;
     static constexpr int STAGES_RAW = (232448 - 2048 - TABLE_BYTES) / (MANT_STAGE + EXP_STAGE);
@@ -106,7 +90,6 @@ struct Problem {
     int tiles_m, tiles_n;
     int splits;
     int64_t kb_per_split;
-    int64_t rsA, rsB;       // exponent row strides (only for the dump path's bookkeeping)
     float* C;
     int64_t ldc;
     float* partial;         // [splits][M][ldp] when splits > 1
@@ -126,15 +109,15 @@ struct Problem {
 #endif
 
 struct Work {
-    int m0, n0, split;
-    int kb0;                // first K-block of this item
-    int step0, step1;       // K=32 steps [step0, step1), step0 % 4 == 0
+    int m0, nt, split;
+    int kb0, nblk;          // first K-block and number of K-blocks of this item
 };
 
-// 32-bit arithmetic only: this runs in warps that have given most of their registers away.
-__device__ __forceinline__ bool get_work(const Problem& p, int w, Work* out) {
+// 32-bit arithmetic only (this runs in warps that have given most of their registers away);
+// returned by value so that the fields stay in registers.
+__device__ __forceinline__ Work get_work(const Problem& p, int w) {
+    Work out;
     const int tiles = p.tiles_m * p.tiles_n;
-    if (w >= tiles * p.splits) return false;
     const int split = w / tiles;
     const int t = w - split * tiles;
     // groups of 16 tile rows share their B panels in L2 while a group sweeps across N
@@ -145,16 +128,145 @@ __device__ __forceinline__ bool get_work(const Problem& p, int w, Work* out) {
     const int gsize = min(G, p.tiles_m - first_m);
     const int within = t - group * per_group;
     const int nt = within / gsize;
-    out->m0 = (first_m + (within - nt * gsize)) * TILE_M;
-    out->n0 = nt;
-    out->split = split;
-    const int spb = p.bp / 32;
-    const int kb0 = split * (int)p.kb_per_split;
-    const int kb1 = min((int)p.nkb, kb0 + (int)p.kb_per_split);
-    out->kb0 = kb0;
-    out->step0 = kb0 * spb;
-    out->step1 = kb1 * spb;
-    return true;
+    out.m0 = (first_m + (within - nt * gsize)) * TILE_M;
+    out.nt = nt;
+    out.split = split;
+    out.kb0 = split * (int)p.kb_per_split;
+    out.nblk = min((int)p.nkb, out.kb0 + (int)p.kb_per_split) - out.kb0;
+    return out;
+}
+
+// How the K-blocks of an item map onto 128-byte stages: blocks of 32 or 64 bytes share a stage
+// (bps of them, spb MMA steps each); longer blocks span spk whole stages.
+struct Shape {
+    int lb, bps, spb, spk;  // log2(bps), blocks per stage, MMA steps per block inside a stage, stages per block
+    bool lng;
+};
+__device__ __forceinline__ Shape make_shape(int bp) {
+    Shape s;
+    s.lng = bp >= STAGE_K;
+    s.lb = bp == 32 ? 2 : bp == 64 ? 1 : 0;
+    s.bps = 1 << s.lb;
+    s.spb = 4 >> s.lb;
+    s.spk = s.lng ? bp / STAGE_K : 1;       // (once per kernel)
+    return s;
+}
+__device__ __forceinline__ int stages_of(const Shape& sh, int nblk) {
+    return sh.lng ? nblk * sh.spk : (nblk + sh.bps - 1) >> sh.lb;
+}
+
+// Advances a ring position (stage, accumulator group or table slot) and its phase bit.
+template <int N>
+__device__ __forceinline__ void ring_next(uint32_t& i, uint32_t& ph) {
+    if (++i == N) { i = 0; ph ^= 1u; }
+}
+
+// Non-blocking look at a barrier phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+
+// 2^e as binary32 bits (MAGIC) or the exponent shifted into the exponent field, e = signed byte i of
+// a packed word of exponents.
+__device__ __forceinline__ uint32_t exp_to_field(uint32_t packed, int i, int add) {
+    const int e = (int)(int8_t)(packed >> (8 * i));
+    return (uint32_t)(e + add) << 23;
+}
+
+// ------------------------------------------------------------------------------ MMA issuer
+
+struct MmaArgs {
+    uint32_t full_bar, empty_bar, tfull_bar, tempty_bar, done_bar, mant_base, tmem_base;
+    int total_work;
+    volatile int* abort_flag;
+};
+
+// The loop of the single MMA-issuing thread. LNG: blocks of 128 bytes or more (one block step set per
+// stage, SPB = 4); otherwise 128 / (32 SPB) blocks of SPB steps share a stage.
+template <int N_TILE, int PLANES, bool MAGIC, bool LNG, int SPB>
+__device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh, const MmaArgs& a) {
+    using C = Cfg<N_TILE, PLANES>;
+    constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
+    constexpr int BPS = LNG ? 1 : 4 / SPB;
+    constexpr uint32_t idesc = idesc_i8<N_TILE>();
+    uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
+    // The barriers the next MMAs will need are polled (without blocking) just before the last MMA
+    // step of a block or stage is issued, while earlier MMAs still occupy the tensor pipe; a
+    // barrier found complete then is not waited on again.
+    bool pre_full = false, pre_tempty = false;
+    bool ok = true;
+    for (int wi = blockIdx.x; ok && wi < a.total_work; wi += gridDim.x) {
+        const Work w = get_work(p, wi);
+        const int nst = stages_of(sh, w.nblk);
+        int left = w.nblk, sib = 0;
+        for (int si = 0; ok && si < nst; ++si, ++it) {
+            if (pre_full) pre_full = false;
+            else if (!mbar_wait(a.full_bar + 8 * s, ph, a.abort_flag, p.status, 201)) { ok = false; break; }
+            HBFP_TRACE(2, it);
+            tc_fence_after();
+            const uint32_t ms = a.mant_base + s * C::MANT_STAGE;
+            const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
+            const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
+            const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
+            const int nb = LNG ? 1 : min(BPS, left);          // blocks that have steps in this stage
+#pragma unroll
+            for (int jb = 0; jb < BPS; ++jb) {
+                if (jb < nb) {
+                    const bool first = !LNG || sib == 0;              // the block starts in this stage
+                    const bool last = !LNG || sib == sh.spk - 1;      // ... and ends in it
+                    if (first) {
+                        // the group was read (and, on the biased path, re-armed) by all rescale warps
+                        if (pre_tempty) pre_tempty = false;
+                        else if (!mbar_wait(a.tempty_bar + 8 * g, gph, a.abort_flag, p.status, 202)) { ok = false; break; }
+                        HBFP_TRACE(3, blk);
+                        tc_fence_after();
+                    }
+                    const uint32_t d = a.tmem_base + g * PARTS * N_TILE;
+#pragma unroll
+                    for (int q = 0; q < SPB; ++q) {
+                        if (q == SPB - 1) {
+                            // look ahead while the tensor pipe still has the earlier MMAs to run
+                            if (last) {
+                                uint32_t g2 = g, gph2 = gph;
+                                ring_next<GROUPS>(g2, gph2);
+                                pre_tempty = mbar_test_wait(a.tempty_bar + 8 * g2, gph2);
+                            }
+                            if (jb == nb - 1) {
+                                uint32_t s2 = s, ph2 = ph;
+                                ring_next<STAGES>(s2, ph2);
+                                pre_full = mbar_test_wait(a.full_bar + 8 * s2, ph2);
+                            }
+                        }
+                        const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));      // 32 bytes per step, in 16-byte units
+                        // biased path: always accumulate on top of the bias; else the first step of a block overwrites
+                        const uint32_t acc = MAGIC ? 1u : (uint32_t)!(first && q == 0);
+                        if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
+                        if (PLANES == 2 && !(HBFP_TC_PROBE & 2)) {
+                            tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
+                            tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc, 1u);
+                            tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_lo + ko, idesc, acc);
+                        }
+                    }
+                    if (last) {
+                        tc_commit(a.tfull_bar + 8 * g);
+                        ring_next<GROUPS>(g, gph);
+                        ++blk;
+                        sib = 0;
+                    } else {
+                        ++sib;
+                    }
+                }
+            }
+            left -= nb;
+            tc_commit(a.empty_bar + 8 * s);        // the stage is free once these MMAs have read it
+            HBFP_TRACE(4, it);
+            ring_next<STAGES>(s, ph);
+        }
+    }
+    tc_commit(a.done_bar);
+    mbar_wait(a.done_bar, 0, a.abort_flag, p.status, 203, false);
 }
 
 // ------------------------------------------------------------------------------ kernel
@@ -166,7 +278,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                const __grid_constant__ CUtensorMap mapEA, const __grid_constant__ CUtensorMap mapEB,
                const Problem p) {
     using C = Cfg<N_TILE, PLANES>;
-    constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
+    constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS, TSLOTS = C::TABLE_SLOTS;
     constexpr int COLS_PER_WARP = N_TILE / COL_GROUPS;  // warps that share a lane quarter split the columns
     static_assert(!(MAGIC && PLANES != 1), "the biased-accumulator path is for one-plane operands");
 
@@ -177,15 +289,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     const uint32_t exp_base = mant_base + STAGES * C::MANT_STAGE;           // STAGES x EXP_STAGE
     const uint32_t table_off = STAGES * (C::MANT_STAGE + C::EXP_STAGE);
     uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [slot][N_TILE column scales | 128 row scales]
-    constexpr int TSLOTS = C::TABLE_SLOTS;
     const uint32_t bar_off = table_off + C::TABLE_BYTES;
     const uint32_t bars = base + bar_off;
-    const uint32_t full_bar = bars, empty_bar = bars + 8 * STAGES;
-    const uint32_t tfull_bar = bars + 16 * STAGES, tempty_bar = tfull_bar + 8 * GROUPS;
+    const uint32_t full_bar = bars;                          // stage landed (mantissa tiles and exponent slices)
+    const uint32_t empty_bar = bars + 8 * STAGES;            // stage consumed (MMA commit + table warp)
+    const uint32_t tfull_bar = bars + 16 * STAGES;           // block sums complete (MMA commit) and scale table written
+    const uint32_t tempty_bar = tfull_bar + 8 * GROUPS;      // group read (and re-armed) by every rescale warp
     const uint32_t done_bar = tempty_bar + 8 * GROUPS;
-    const uint32_t tready_bar = done_bar + 8;              // table slot written (by the table warp)
-    const uint32_t tfree_bar = tready_bar + 8 * TSLOTS;    // table slot read by all rescale warps
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + 16 * STAGES + 16 * GROUPS + 8 + 16 * TSLOTS);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(base_ptr + bar_off + 16 * STAGES + 16 * GROUPS + 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -196,14 +307,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             mbar_init(empty_bar + 8 * s, 2);                 // MMA commit + table warp
         }
         for (int g = 0; g < GROUPS; ++g) {
-            mbar_init(tfull_bar + 8 * g, 1);
+            mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + table warp
             mbar_init(tempty_bar + 8 * g, RESCALE_WARPS);
         }
         mbar_init(done_bar, 1);
-        for (int i = 0; i < TSLOTS; ++i) {
-            mbar_init(tready_bar + 8 * i, 1);
-            mbar_init(tfree_bar + 8 * i, RESCALE_WARPS);
-        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -217,7 +324,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int spb = p.bp / 32;                      // K=32 steps per block
+    const Shape sh = make_shape(p.bp);
+    const int total_work = p.tiles_m * p.tiles_n * p.splits;
 
     if (warp < CONTROL_WARPS) {
         // the control warpgroup hands most of its registers to the rescale warps
@@ -225,19 +333,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         if (warp == PRODUCER_WARP) {
             // -------------------------------------------------------------- TMA producer
             if (lane == 0) {
-                uint32_t it = 0;
+                uint32_t s = 0, ph = 0, it = 0;
                 bool ok = true;
-                Work w;
-                for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-                    const int n0 = w.n0 * N_TILE;
-                    int pos = 0, kb = w.kb0;          // position inside the current block, its index
-                    for (int st0 = w.step0; st0 < w.step1; st0 += 4, ++it) {
-                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+                for (int wi = blockIdx.x; ok && wi < total_work; wi += gridDim.x) {
+                    const Work w = get_work(p, wi);
+                    const int n0 = w.nt * N_TILE;
+                    const int nst = stages_of(sh, w.nblk);
+                    int kb = w.kb0, sib = 0;              // first block touched by the stage; stage inside a long block
+                    int kbyte = w.kb0 * p.bp;
+                    for (int si = 0; si < nst; ++si, kbyte += STAGE_K, ++it) {
                         if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
                         HBFP_TRACE(0, it);
                         const uint32_t fb = full_bar + 8 * s;
                         mbar_expect_tx(fb, (HBFP_TC_PROBE & 4) ? (uint32_t)C::EXP_STAGE : C::TX_BYTES);
-                        const int kbyte = st0 * 32;
                         const uint32_t ms = mant_base + s * C::MANT_STAGE;
                         // A panels are re-used by every column tile of a group of 16 tile rows: ask L2 to keep
                         // them while the B panels stream past (marking B evict-first doubled the DRAM reads:
@@ -249,105 +357,82 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                             tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
                         }
                         const uint32_t es = exp_base + s * C::EXP_STAGE;
-                        tma_load_2d(es, &mapEA, w.m0, kb, fb);          // kb = first block touched by this stage
+                        tma_load_2d(es, &mapEA, w.m0, kb, fb);
                         tma_load_2d(es + C::EXP_A, &mapEB, n0, kb, fb);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            if (pos == spb - 1) { pos = 0; ++kb; } else { ++pos; }
-                        }
+                        if (sh.lng) { if (++sib == sh.spk) { sib = 0; ++kb; } } else { kb += sh.bps; }
+                        ring_next<STAGES>(s, ph);
                     }
                 }
                 // Drain: every issued copy must have landed before the CTA may exit. In a normal run
                 // the consumers already waited for all of them, so these return at once.
-                const uint32_t issued = it;
-                for (uint32_t k = issued > (uint32_t)STAGES ? issued - STAGES : 0; k < issued; ++k)
-                    mbar_wait(full_bar + 8 * (k % STAGES), (k / STAGES) & 1, abort_flag, p.status, 102, false);
+                const uint32_t back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+                for (uint32_t k = 0; k < back; ++k) {
+                    if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+                    mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 102, false);
+                }
             }
         } else if (warp == MMA_WARP) {
             // -------------------------------------------------------------- MMA issuer
             if (lane == 0) {
-                constexpr uint32_t idesc = idesc_i8<N_TILE>();
-                uint32_t it = 0, blk = 0;
-                bool ok = true;
-                Work w;
-                for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-                    int pos = 0;
-                    for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
-                        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
-                        if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 201)) { ok = false; break; }
-                        HBFP_TRACE(2, it);
-                        tc_fence_after();
-                        const uint32_t ms = mant_base + s * C::MANT_STAGE;
-                        const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
-                        const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
-                        const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
-                        for (int j = 0; j < 4; ++j) {
-                            if (st0 + j >= w.step1) break;
-                            const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
-                            if (pos == 0) {
-                                // the group was read (and, on the biased path, re-biased) by all rescale warps
-                                if (!mbar_wait(tempty_bar + 8 * g, gph, abort_flag, p.status, 202)) { ok = false; break; }
-                                HBFP_TRACE(3, blk);
-                                tc_fence_after();
-                            }
-                            const uint32_t d = tmem_base + g * PARTS * N_TILE;
-                            const uint64_t ko = (uint64_t)(2 * j);          // 32 bytes per step, in 16-byte units
-                            const uint32_t acc = MAGIC ? 1u : (uint32_t)(pos != 0);   // biased path: accumulate on top of the bias
-                            if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
-                            if (PLANES == 2 && !(HBFP_TC_PROBE & 2)) {
-                                tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, acc);
-                                tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc, 1u);
-                                tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_lo + ko, idesc, acc);
-                            }
-                            if (pos == spb - 1) {
-                                tc_commit(tfull_bar + 8 * g);
-                                ++blk;
-                                pos = 0;
-                            } else {
-                                ++pos;
-                            }
-                        }
-                        tc_commit(empty_bar + 8 * s);        // the stage is free once these MMAs have read it
-                        HBFP_TRACE(4, it);
-                    }
-                }
-                tc_commit(done_bar);
-                mbar_wait(done_bar, 0, abort_flag, p.status, 203, false);
+                const MmaArgs ma{full_bar, empty_bar, tfull_bar, tempty_bar, done_bar, mant_base, tmem_base, total_work, abort_flag};
+                if (sh.lng) mma_issue_loop<N_TILE, PLANES, MAGIC, true, 4>(p, sh, ma);
+                else if (sh.spb == 2) mma_issue_loop<N_TILE, PLANES, MAGIC, false, 2>(p, sh, ma);
+                else mma_issue_loop<N_TILE, PLANES, MAGIC, false, 1>(p, sh, ma);
             }
         } else if (warp == TABLE_WARP) {
             // -------------------------------------------------------------- scale-table builder
-            uint32_t it = 0, blk = 0;
+            // The table of block b goes to slot b % (2 GROUPS) and its arrival counts on tfull[b % GROUPS].
+            // It is written once the previous phase of that barrier (block b - GROUPS) is complete: the
+            // MMAs of that block were issued only after every rescale warp had finished block
+            // b - 2 GROUPS, the last reader of the slot, and the barrier is back in the phase that the
+            // arrival for b belongs to.
+            uint32_t s = 0, ph = 0, g = 0, gph = 0, slot = 0, it = 0, blk = 0;
             bool ok = true;
-            Work w;
-            for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-                int pos = 0;
-                for (int st0 = w.step0; ok && st0 < w.step1; st0 += 4, ++it) {
-                    const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
+            for (int wi = blockIdx.x; ok && wi < total_work; wi += gridDim.x) {
+                const Work w = get_work(p, wi);
+                const int nst = stages_of(sh, w.nblk);
+                int left = w.nblk, sib = 0;
+                for (int si = 0; ok && si < nst; ++si, ++it) {
                     if (!mbar_wait_warp(full_bar + 8 * s, ph, abort_flag, p.status, 401)) { ok = false; break; }
-                    const int8_t* eA = reinterpret_cast<const int8_t*>(base_ptr + (exp_base - base) + s * C::EXP_STAGE);
-                    const int8_t* eB = eA + C::EXP_A;
-                    int jb = 0;                    // row of the exponent slices: blocks that start in this stage
-                    for (int j = 0; j < 4; ++j) {
-                        if (st0 + j >= w.step1) break;
-                        if (pos == 0) {
-                            const uint32_t slot = blk % TSLOTS, sph = (blk / TSLOTS) & 1;
-                            if (!mbar_wait_warp(tfree_bar + 8 * slot, sph, abort_flag, p.status, 402)) { ok = false; break; }
-                            uint32_t* tb = tables + slot * C::TABLE_SLOT_WORDS;
-                            for (int c = lane; c < N_TILE; c += 32) {
-                                const int sb = (int)eB[jb * N_TILE + c];
-                                tb[c] = MAGIC ? (uint32_t)(sb + 127) << 23 : (uint32_t)(sb << 23);
-                            }
-                            for (int r = lane; r < TILE_M; r += 32)
-                                tb[N_TILE + r] = (uint32_t)((int)eA[jb * TILE_M + r] + 127) << 23;
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(tready_bar + 8 * slot);
-                            ++blk;
-                            ++jb;
+                    const unsigned char* eA = base_ptr + (exp_base - base) + s * C::EXP_STAGE;
+                    const unsigned char* eB = eA + C::EXP_A;
+                    const int nb = sh.lng ? (sib == 0 ? 1 : 0) : min(sh.bps, left);   // blocks that start in this stage
+                    for (int jb = 0; jb < nb; ++jb) {
+                        // this lane's N_TILE / 32 column exponents and 4 row exponents of the block
+                        constexpr int CPL = N_TILE / 32;      // 8, 4 or 2 column bytes per lane
+                        uint32_t cw[2] = {0u, 0u};
+                        if (CPL == 8) { const uint2 t = *reinterpret_cast<const uint2*>(eB + jb * N_TILE + 8 * lane); cw[0] = t.x; cw[1] = t.y; }
+                        else if (CPL == 4) cw[0] = *reinterpret_cast<const uint32_t*>(eB + jb * N_TILE + 4 * lane);
+                        else cw[0] = *reinterpret_cast<const uint16_t*>(eB + jb * N_TILE + 2 * lane);
+                        const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
+                        uint32_t cs[CPL];
+#pragma unroll
+                        for (int i = 0; i < CPL; ++i) cs[i] = exp_to_field(cw[i >> 2], i & 3, MAGIC ? 127 : 0);
+                        uint4 r0;
+                        r0.x = exp_to_field(ra, 0, 127); r0.y = exp_to_field(ra, 1, 127);
+                        r0.z = exp_to_field(ra, 2, 127); r0.w = exp_to_field(ra, 3, 127);
+                        if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 402)) { ok = false; break; }
+                        uint32_t* tb = tables + slot * C::TABLE_SLOT_WORDS;
+                        if (CPL == 8) {
+                            *reinterpret_cast<uint4*>(tb + 8 * lane) = make_uint4(cs[0], cs[1], cs[2], cs[3]);
+                            *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = make_uint4(cs[4 % CPL], cs[5 % CPL], cs[6 % CPL], cs[7 % CPL]);
+                        } else if (CPL == 4) {
+                            *reinterpret_cast<uint4*>(tb + 4 * lane) = make_uint4(cs[0], cs[1], cs[2 % CPL], cs[3 % CPL]);
+                        } else {
+                            *reinterpret_cast<uint2*>(tb + 2 * lane) = make_uint2(cs[0], cs[1]);
                         }
-                        pos = pos == spb - 1 ? 0 : pos + 1;
+                        *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
+                        ring_next<GROUPS>(g, gph);
+                        if (++slot == (uint32_t)TSLOTS) slot = 0;
+                        ++blk;
                     }
+                    if (sh.lng) { if (++sib == sh.spk) sib = 0; }
+                    left -= nb;
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_bar + 8 * s);      // the exponent slices are consumed
+                    ring_next<STAGES>(s, ph);
                 }
             }
         }
@@ -360,47 +445,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         const int col0 = half * COLS_PER_WARP;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
         uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
-#if !HBFP_TC_FFMA2
-        float accf[MAGIC ? COLS_PER_WARP : 1];
-#endif
-        uint32_t bias[8];
+        uint32_t bias16[MAGIC ? 16 : 1];
         if (MAGIC) {
+            {
+                uint32_t bias[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
-            for (int g = 0; g < GROUPS; ++g)
+                for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
+                for (int g = 0; g < GROUPS; ++g)
 #pragma unroll
-                for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
-            tc_wait_st();
+                    for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
+                tc_wait_st();
+            }
+            // Read the bias back as one sixteen-register tuple: a tuple that is born as such is passed
+            // to every re-arming store in place, while separately defined registers are copied into a
+            // fresh tuple for each store (one extra instruction per register and store).
+            tc_ld16(lane_addr, reinterpret_cast<uint32_t(&)[16]>(bias16));
+            tc_wait_ld();
         }
-        // every accumulator group and every table slot starts out free
+        // every accumulator group starts out free
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) {
+        if (lane == 0)
             for (int g = 0; g < GROUPS; ++g) mbar_arrive(tempty_bar + 8 * g);
-            for (int i = 0; i < TSLOTS; ++i) mbar_arrive(tfree_bar + 8 * i);
-        }
 
-        uint32_t blk = 0;
+        uint32_t g = 0, gph = 0, slot = 0, blk = 0;
         bool ok = true;
-        Work w;
-        for (int wi = blockIdx.x; ok && get_work(p, wi, &w); wi += gridDim.x) {
-            const int n0 = w.n0 * N_TILE;
+        for (int wi = blockIdx.x; ok && wi < total_work; wi += gridDim.x) {
+            const Work w = get_work(p, wi);
+            const int n0 = w.nt * N_TILE;
             const int64_t gi = w.m0 + row;
 #pragma unroll
             for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
-#if !HBFP_TC_FFMA2
-            if (MAGIC) {
-#pragma unroll
-                for (int c = 0; c < COLS_PER_WARP; ++c) accf[c] = 0.f;
-            }
-#endif
-            const int nblk = (w.step1 - w.step0) / spb;      // (once per tile; spb divides the range)
-            for (int kb = w.kb0; kb < w.kb0 + nblk; ++kb, ++blk) {
-                const uint32_t g = blk % GROUPS, gph = (blk / GROUPS) & 1;
-                const uint32_t slot = blk % TSLOTS, sph = (blk / TSLOTS) & 1;
-                if (!mbar_wait_warp(tready_bar + 8 * slot, sph, abort_flag, p.status, 303)) { ok = false; break; }
+            for (int kb = w.kb0; kb < w.kb0 + w.nblk; ++kb, ++blk) {
+                // one wait per block: the block sums are complete and the scale table is written
                 if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
-                if (threadIdx.x == CONTROL_WARPS * 32) HBFP_TRACE(7, blk);
                 if (lane == 0) HBFP_TRACE(17 + rwarp, blk);
                 tc_fence_after();
                 const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
@@ -414,17 +492,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     const float ca_f = -12582912.0f * sa_f;
                     const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
                     const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
-                    constexpr int CH = HBFP_TC_CHUNK;
+                    constexpr int CH = 16;
                     constexpr int NCHK = COLS_PER_WARP / CH;
-                    constexpr int NBUF = RESCALE_WARPS == 8 ? 2 : 1;   // four warps per sub-partition hide the load latency themselves
-                    uint32_t v[NBUF][CH];
-                    if (NBUF == 2) tc_ldn(taddr, v[0]);
+                    uint32_t v[2][CH];
+                    tc_ld16(taddr, v[0]);
 #pragma unroll
                     for (int ch = 0; ch < NCHK; ++ch) {
-                        if (NBUF == 1) tc_ldn(taddr + ch * CH, v[0]);
                         tc_wait_ld();
-                        if (NBUF == 2 && ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & (NBUF - 1)]);
-                        const uint32_t(&x)[CH] = v[ch & (NBUF - 1)];
+                        if (ch + 1 < NCHK) tc_ld16(taddr + (ch + 1) * CH, v[(ch + 1) & 1]);
+                        const uint32_t(&x)[CH] = v[ch & 1];
                         if (DUMP && p.P != nullptr && gi < p.M) {
 #pragma unroll
                             for (int c = 0; c < CH; ++c) {
@@ -432,33 +508,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                                 if (gj < p.N) p.P[(gi * p.N + gj) * p.nkb + kb] = (int32_t)(x[c] - BIAS_BITS);
                             }
                         }
-#if HBFP_TC_PROBE & 16
-                        acc2[ch] ^= pack2(x[0], x[CH - 1]);
-                        continue;
-#endif
 #pragma unroll
                         for (int q = 0; q < CH; q += 4) {
-#if HBFP_TC_PROBE & 1024
-                            const uint4 sb = make_uint4(sa_u, sa_u + q, sa_u, sa_u + ch);
-#else
                             const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CH + q);
-#endif
-#if HBFP_TC_FFMA2
                             const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
                             const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
                             acc2[(ch * CH + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
                             acc2[(ch * CH + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CH + q) / 2 + 1]);
-#else
-                            accf[ch * CH + q + 0] = fmaf(fmaf(__uint_as_float(x[q + 0]), sa_f, ca_f), __uint_as_float(sb.x), accf[ch * CH + q + 0]);
-                            accf[ch * CH + q + 1] = fmaf(fmaf(__uint_as_float(x[q + 1]), sa_f, ca_f), __uint_as_float(sb.y), accf[ch * CH + q + 1]);
-                            accf[ch * CH + q + 2] = fmaf(fmaf(__uint_as_float(x[q + 2]), sa_f, ca_f), __uint_as_float(sb.z), accf[ch * CH + q + 2]);
-                            accf[ch * CH + q + 3] = fmaf(fmaf(__uint_as_float(x[q + 3]), sa_f, ca_f), __uint_as_float(sb.w), accf[ch * CH + q + 3]);
-#endif
                         }
-#if !(HBFP_TC_PROBE & 2048)
-#pragma unroll
-                        for (int c8 = 0; c8 < CH / 8; ++c8) tc_st8(taddr + ch * CH + c8 * 8, bias);   // re-arm
-#endif
+                        tc_st16(taddr + ch * CH, reinterpret_cast<const uint32_t(&)[16]>(bias16));   // re-arm
                     }
                     tc_wait_st();
                 } else {
@@ -503,18 +561,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(tempty_bar + 8 * g);
-                    mbar_arrive(tfree_bar + 8 * slot);
+                    HBFP_TRACE(9 + rwarp, blk);
                 }
-                if (threadIdx.x == CONTROL_WARPS * 32) HBFP_TRACE(8, blk);
-                if (lane == 0) HBFP_TRACE(9 + rwarp, blk);
+                ring_next<GROUPS>(g, gph);
+                if (++slot == (uint32_t)TSLOTS) slot = 0;
             }
             if (!ok) break;
-#if !HBFP_TC_FFMA2
-            if (MAGIC) {
-#pragma unroll
-                for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = pack2(__float_as_uint(accf[2 * c]), __float_as_uint(accf[2 * c + 1]));
-            }
-#endif
             // ---- store the tile (or this split's partial tile)
             float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
             const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
@@ -656,8 +708,6 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     p.tiles_n = (int)((N + plan.n_tile - 1) / plan.n_tile);
     p.splits = P ? 1 : plan.splits;
     p.kb_per_split = P ? a.L.nkb : plan.kb_per_split;
-    p.rsA = a.L.rs;
-    p.rsB = b.L.rs;
     p.C = Cout;
     p.ldc = ldc;
     p.partial = static_cast<float*>(partial);
