@@ -7,9 +7,10 @@
 // rescale work as a 128 x 256 tile on one SM, but only half of the B panel crosses from L2 into
 // each SM, which is what limits the single-SM kernel on large problems.
 //
-// Roles per CTA (12 warps) as in the single-SM kernel: warp 0 TMA producer, warp 1 MMA issuer
+// Roles per CTA (16 warps) as in the single-SM kernel: warp 0 TMA producer, warp 1 MMA issuer
 // (only in the cluster's first CTA, the leader) and tensor-memory owner, warp 2 scale-table
-// builder, warps 4-11 rescale (Eq. 2 per block, blocks accumulated in FP32, Sec. 4).
+// builder, warps 4-15 rescale (Eq. 2 per block, blocks accumulated in FP32, Sec. 4): three per
+// lane quarter of tensor memory, which split the 256 columns 88 + 88 + 80.
 //
 // Barriers. Mantissa tiles of both CTAs complete on the leader's full[s]; exponent slices on a
 // local efull[s]; the leader's MMA thread commits to tfull[g] and empty[s] of both CTAs; the
@@ -31,13 +32,21 @@ namespace {
 constexpr int N_TILE = 256;            // columns of the pair tile = accumulator columns per CTA
 constexpr int PAIR_M = 2 * TILE_M;     // rows of the pair tile
 constexpr int B_HALF = N_TILE / 2;     // B rows staged in each CTA
-constexpr int RESCALE_WARPS = 8;
+// Rescale warps: 12 (three per sub-partition, 88 + 88 + 80 columns) or 8 (two, 128 columns each). The
+// rescale is bound by latencies, not by a pipe (FP32 pipe about half busy), so the third warp pays.
+#ifndef HBFP_TC2_RWARPS
+#define HBFP_TC2_RWARPS 12
+#endif
+constexpr int RESCALE_WARPS = HBFP_TC2_RWARPS;
 constexpr int CONTROL_WARPS = 4;
 constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = 2;
 constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
-// setmaxnreg totals must not exceed the launch allocation (384 threads x 168 registers)
-constexpr int REGS_RESCALE = 216, REGS_CONTROL = 72;
-static_assert(128 * REGS_CONTROL + 256 * REGS_RESCALE <= 384 * 168, "register split");
+// setmaxnreg totals must not exceed the launch allocation (384 threads x 168 or 512 x 128 registers)
+constexpr int REGS_RESCALE = RESCALE_WARPS == 8 ? 216 : 144;
+constexpr int REGS_CONTROL = RESCALE_WARPS == 8 ? 72 : 64;
+constexpr int REGS_LAUNCH = RESCALE_WARPS == 8 ? 168 : 128;
+static_assert(RESCALE_WARPS == 8 || RESCALE_WARPS == 12, "rescale warp count");
+static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= THREADS * REGS_LAUNCH - (RESCALE_WARPS == 8 ? 0 : 512), "register split");
 
 constexpr int GROUPS = TMEM_COLS / N_TILE;                  // 2 accumulator groups
 constexpr int A_BYTES = TILE_M * STAGE_K, B_BYTES = B_HALF * STAGE_K;
@@ -50,7 +59,6 @@ constexpr int TABLE_BYTES = 4 * TSLOTS * TABLE_SLOT_WORDS;
 constexpr int STAGES = 6;
 constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024;
 static_assert(SMEM <= 232448, "shared memory");
-constexpr int CH = 16;                                      // columns per tensor-memory load
 
 // Build-time probe for performance bisection (never set in the shipped library; results are wrong
 // when it is): 1 = rescale warps skip the tensor-memory traffic and the math, 2 = no MMA is issued,
@@ -209,13 +217,130 @@ __device__ __forceinline__ uint32_t exp_to_scale(uint32_t packed, int i) {
     return (uint32_t)(e + 127) << 23;
 }
 
-// ------------------------------------------------------------------------------ kernel
-
 // Advances a ring position (stage, accumulator group or table slot) and its phase bit.
 template <int N>
 __device__ __forceinline__ void ring_next(uint32_t& i, uint32_t& ph) {
     if (++i == N) { i = 0; ph ^= 1u; }
 }
+
+// ------------------------------------------------------------------------------ rescale warps
+
+struct RescaleArgs {
+    uint32_t tfull_bar, leader_tempty, tmem_base;
+    uint32_t* tables;
+    int total_work, cluster, nclusters;
+    uint32_t rank;
+    volatile int* abort_flag;
+};
+
+// The loop of one rescale warp: rows = its lane quarter of this CTA's half tile, columns
+// [col0, col0 + NCOLS) of every accumulator group, read in chunks of CHW columns.
+template <int NCOLS, int CHW>
+__device__ __forceinline__ void rescale_loop(const Problem& p, const RescaleArgs& a, int col0, int rwarp) {
+    constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : NCOLS / CHW;
+    static_assert(NCOLS % CHW == 0 && NCOLS % 8 == 0, "column split");
+    const int lane = threadIdx.x & 31, quarter = (threadIdx.x >> 5) & 3;   // tensor-memory lanes follow warp % 4
+    const int row = quarter * 32 + lane;                 // row of this CTA's half tile = tensor-memory lane
+    const uint32_t lane_addr = a.tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
+    const int cluster = a.cluster;
+    const uint32_t rank = a.rank;
+    (void)cluster; (void)rank; (void)rwarp;
+    uint64_t acc2[NCOLS / 2];                            // FP32 accumulators, two columns per entry
+    {
+        uint32_t bias[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
+        for (int g = 0; g < GROUPS; ++g)
+#pragma unroll
+            for (int c8 = 0; c8 < NCOLS / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
+        tc_wait_st();
+    }
+    // Read the bias back as one register tuple: a tuple that is born as such is passed to every
+    // re-arming store in place, while separately defined registers are copied into a fresh tuple
+    // for each store (one extra instruction per register and store).
+    uint32_t bias_t[CHW];
+    tc_ldn(lane_addr, bias_t);
+    tc_wait_ld();
+    // every accumulator group starts out free
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0)
+        for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(a.leader_tempty + 8 * g);
+
+    uint32_t g = 0, gph = 0, slot = 0, blk = 0;
+    bool ok = true;
+    for (int wi = a.cluster; ok && wi < a.total_work; wi += a.nclusters) {
+        const Work w = get_work(p, wi);
+        const int64_t gi = w.m0 + (int)a.rank * TILE_M + row;
+#pragma unroll
+        for (int c = 0; c < NCOLS / 2; ++c) acc2[c] = 0ull;
+        for (int kb = 0; kb < w.nblk; ++kb, ++blk) {
+            const uint32_t taddr = lane_addr + g * N_TILE;
+            uint32_t v[2][CHW];
+            // one wait per block: the block sums are complete and this CTA's scale table is written
+            if (!mbar_wait_warp(a.tfull_bar + 8 * g, gph, a.abort_flag, p.status, 312)) { ok = false; break; }
+            tc_fence_after();
+            if (NCHK) tc_ldn(taddr, v[0]);
+            if (lane == 0) TC2_TRACE(4 + (rwarp & 7), blk);
+            const uint32_t* tab = a.tables + slot * TABLE_SLOT_WORDS + col0;
+            // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
+            // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
+            const float sa_f = __uint_as_float(a.tables[slot * TABLE_SLOT_WORDS + N_TILE + row]);
+            const float ca_f = -12582912.0f * sa_f;
+            const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
+            const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
+#pragma unroll
+            for (int ch = 0; ch < NCHK; ++ch) {
+                tc_wait_ld();
+                if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CHW, v[(ch + 1) & 1]);
+                const uint32_t(&x)[CHW] = v[ch & 1];
+#pragma unroll
+                for (int q = 0; q < CHW; q += 4) {
+                    const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CHW + q);
+                    const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
+                    const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
+                    acc2[(ch * CHW + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CHW + q) / 2]);
+                    acc2[(ch * CHW + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CHW + q) / 2 + 1]);
+                }
+#if !(HBFP_TC2_PROBE & 16)
+                tc_stn(taddr + ch * CHW, bias_t);          // re-arm
+#endif
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_remote(a.leader_tempty + 8 * g);
+                TC2_TRACE(12 + (rwarp & 7), blk);
+            }
+            ring_next<GROUPS>(g, gph);
+            slot = (slot + 1) & (TSLOTS - 1);
+        }
+        if (!ok) break;
+        // ---- store this warp's part of the tile (or of this split's partial tile)
+        float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
+        const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
+        if (gi < p.M) {
+            float* rowp = dst + gi * ldd + w.n0 + col0;
+#pragma unroll
+            for (int c = 0; c < NCOLS; c += 4) {
+                const int64_t gj = w.n0 + col0 + c;
+                if (gj + 3 < p.N) {
+                    *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
+                } else {
+                    float e4[4];
+                    unpack2(acc2[c / 2], e4[0], e4[1]);
+                    unpack2(acc2[c / 2 + 1], e4[2], e4[3]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (gj + e < p.N) rowp[c + e] = e4[e];
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------ kernel
 
 // LB = log2(K-blocks per 128-byte stage): 0 for blocks of 128 bytes, 1 for 64, 2 for 32.
 template <int LB>
@@ -425,107 +550,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     } else {
         // ------------------------------------------------------------------ rescale warps (both CTAs)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
-        constexpr int COLS_PER_WARP = N_TILE / 2;            // two warps share a lane quarter and split the columns
-        constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : COLS_PER_WARP / CH;
-        const int rwarp = warp - CONTROL_WARPS;              // 0..7
-        const int quarter = warp & 3, half = rwarp >> 2;     // tensor-memory lanes follow warp % 4
-        const int row = quarter * 32 + lane;                 // row of this CTA's half tile = tensor-memory lane
-        const int col0 = half * COLS_PER_WARP;
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
-        const uint32_t leader_tempty = map_to_rank(tempty_bar, 0);
-        uint64_t acc2[COLS_PER_WARP / 2];                    // FP32 accumulators, two columns per entry
-        {
-            uint32_t bias[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
-            for (int g = 0; g < GROUPS; ++g)
-#pragma unroll
-                for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
-            tc_wait_st();
-        }
-        // Read the bias back as one sixteen-register tuple: a tuple that is born as such is passed to
-        // every re-arming store in place, while separately defined registers are copied into a fresh
-        // tuple for each store (one extra instruction per register and store).
-        uint32_t bias16[16];
-        tc_ld16(lane_addr, bias16);
-        tc_wait_ld();
-        // every accumulator group starts out free
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0)
-            for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(leader_tempty + 8 * g);
-
-        uint32_t g = 0, gph = 0, slot = 0, blk = 0;
-        bool ok = true;
-        for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
-            const Work w = get_work(p, wi);
-            const int64_t gi = w.m0 + (int)rank * TILE_M + row;
-#pragma unroll
-            for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
-            for (int kb = 0; kb < w.nblk; ++kb, ++blk) {
-                const uint32_t taddr = lane_addr + g * N_TILE;
-                uint32_t v[2][CH];
-                // one wait per block: the block sums are complete and this CTA's scale table is written
-                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 312)) { ok = false; break; }
-                tc_fence_after();
-                if (NCHK) tc_ldn(taddr, v[0]);
-                if (lane == 0) TC2_TRACE(4 + rwarp, blk);
-                const uint32_t* tab = tables + slot * TABLE_SLOT_WORDS + col0;
-                // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
-                // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
-                const float sa_f = __uint_as_float(tables[slot * TABLE_SLOT_WORDS + N_TILE + row]);
-                const float ca_f = -12582912.0f * sa_f;
-                const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
-                const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
-#pragma unroll
-                for (int ch = 0; ch < NCHK; ++ch) {
-                    tc_wait_ld();
-                    if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CH, v[(ch + 1) & 1]);
-                    const uint32_t(&x)[CH] = v[ch & 1];
-#pragma unroll
-                    for (int q = 0; q < CH; q += 4) {
-                        const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CH + q);
-                        const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
-                        const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
-                        acc2[(ch * CH + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
-                        acc2[(ch * CH + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CH + q) / 2 + 1]);
-                    }
-#if !(HBFP_TC2_PROBE & 16)
-                    tc_st16(taddr + ch * CH, bias16);          // re-arm
+        const RescaleArgs ra{tfull_bar, map_to_rank(tempty_bar, 0), tmem_base, tables, total_work, cluster, nclusters, rank, abort_flag};
+        const int rwarp = warp - CONTROL_WARPS, part = rwarp >> 2;     // warps that share a lane quarter split the columns
+#if HBFP_TC2_RWARPS == 12
+        if (part == 2) rescale_loop<80, 8>(p, ra, 176, rwarp);
+        else rescale_loop<88, 8>(p, ra, part * 88, rwarp);
+#else
+        rescale_loop<128, 16>(p, ra, part * 128, rwarp);
 #endif
-                }
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive_remote(leader_tempty + 8 * g);
-                    TC2_TRACE(12 + rwarp, blk);
-                }
-                ring_next<GROUPS>(g, gph);
-                slot = (slot + 1) & (TSLOTS - 1);
-            }
-            if (!ok) break;
-            // ---- store this CTA's 128 rows of the tile (or of this split's partial tile)
-            float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
-            const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
-            if (gi < p.M) {
-                float* rowp = dst + gi * ldd + w.n0 + col0;
-#pragma unroll
-                for (int c = 0; c < COLS_PER_WARP; c += 4) {
-                    const int64_t gj = w.n0 + col0 + c;
-                    if (gj + 3 < p.N) {
-                        *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
-                    } else {
-                        float e4[4];
-                        unpack2(acc2[c / 2], e4[0], e4[1]);
-                        unpack2(acc2[c / 2 + 1], e4[2], e4[3]);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            if (gj + e < p.N) rowp[c + e] = e4[e];
-                    }
-                }
-            }
-        }
     }
 
     // ------------------------------------------------------------------ teardown

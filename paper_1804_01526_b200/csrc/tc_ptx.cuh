@@ -141,6 +141,13 @@ __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
         ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
 }
 
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+        : "r"(taddr) : "memory");
+}
+
 // 16-column variants used by the fast rescale path.
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
     asm volatile(
@@ -179,6 +186,9 @@ __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
 
 __device__ __forceinline__ void tc_ldn(uint32_t taddr, uint32_t (&v)[32]) { tc_ld32(taddr, v); }
 __device__ __forceinline__ void tc_ldn(uint32_t taddr, uint32_t (&v)[16]) { tc_ld16(taddr, v); }
+__device__ __forceinline__ void tc_ldn(uint32_t taddr, uint32_t (&v)[8]) { tc_ld8(taddr, v); }
+__device__ __forceinline__ void tc_stn(uint32_t taddr, const uint32_t (&v)[16]) { tc_st16(taddr, v); }
+__device__ __forceinline__ void tc_stn(uint32_t taddr, const uint32_t (&v)[8]) { tc_st8(taddr, v); }
 
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
