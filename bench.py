@@ -36,7 +36,7 @@ INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio (4.5 : 2.
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) of one launch of the GEMM kernel at the default workload (n = 16384, m = 8,
 # b = 128), from the single-pass ncu capture summarised in profiles/bench_launch_list_n16384_m8_b128.md.
-GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 3885147648 + 1110151680}
+GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 3970740224 + 1068051712}
 
 
 def load_peaks():
@@ -288,7 +288,10 @@ def gpu_arm(args):
     int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
     gemm_tops = ops / (t_gemm * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tops, "peak": int8_burst,
+    # the library takes the paired-SM kernel for one-plane operands with blocks up to 128 and >= 74 tiles of 256 x 256
+    paired = args.mant_bits <= 8 and 0 < args.block <= 128 and ((n + 255) // 256) ** 2 >= 74
+    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel" if paired else "gemm_tc_kernel", "achieved": gemm_tops,
+                "peak": int8_burst,
                 "unit": "TOP/s", "frac": gemm_tops / int8_burst,
                 "traffic": GEMM_DRAM_TRAFFIC_BYTES.get((n, args.mant_bits, args.block)),
                 "algorithmic_bytes": 2 * n * n * ((1 if args.mant_bits <= 8 else 2) + 1.0 / args.block) + 4 * n * n,
