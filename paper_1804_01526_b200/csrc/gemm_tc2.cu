@@ -322,10 +322,16 @@ __device__ __forceinline__ void rescale_loop(const Problem& p, const RescaleArgs
         const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
         if (gi < p.M) {
             float* rowp = dst + gi * ldd + w.n0 + col0;
+            // full 32-byte sectors per lane where the row pitch allows it (each lane owns a row)
+            const bool wide = (ldd & 7) == 0 && (reinterpret_cast<uintptr_t>(dst) & 31) == 0;
 #pragma unroll
             for (int c = 0; c < NCOLS; c += 4) {
                 const int64_t gj = w.n0 + col0 + c;
-                if (gj + 3 < p.N) {
+                if (wide && (c & 7) == 0 && gj + 7 < p.N) {
+                    st_global_256(rowp + c, acc2[c / 2], acc2[c / 2 + 1], acc2[c / 2 + 2], acc2[c / 2 + 3]);
+                } else if (wide && (c & 7) == 4 && gj + 3 < p.N) {
+                    // second half of a sector already written above
+                } else if (gj + 3 < p.N) {
                     *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
                 } else {
                     float e4[4];

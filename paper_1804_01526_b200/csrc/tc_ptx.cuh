@@ -177,6 +177,10 @@ __device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi) {
     asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
     return d;
 }
+// One 32-byte store (a full sector) of eight FP32 values held as four pairs; p must be 32-byte aligned.
+__device__ __forceinline__ void st_global_256(float* p, uint64_t a, uint64_t b, uint64_t c, uint64_t d) {
+    asm volatile("st.global.v4.b64 [%0], {%1, %2, %3, %4};" ::"l"(p), "l"(a), "l"(b), "l"(c), "l"(d) : "memory");
+}
 __device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
     uint32_t a, b;
     asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
