@@ -7,6 +7,8 @@
 //                    thread (two 128-bit loads, one Philox call in stochastic mode), block
 //                    max by warp shuffles, exponents staged in shared memory so that the
 //                    [kb][row] exponent array is written in full 32-byte sectors.
+//   quant_row_flat   the same for row lengths that are not a multiple of 512 (K % b == 0): 8-element
+//                    groups numbered through the whole matrix, no ragged last tile.
 //   quant_col_tma    blocks down the columns, b in {32,64,128}, 16-byte aligned pitch: persistent
 //                    CTAs stream 128 x 64 FP32 tiles through a TMA pipeline and write the packed,
 //                    transposed tile with a swizzled TMA store (full lines in both directions).
@@ -508,6 +510,101 @@ __global__ void dequant_kernel(const int8_t* __restrict__ mant, const int8_t* __
     out[r * ld + kk] = ldexpf((float)v, (int)exps[kb * rs + r]);
 }
 
+// ------------------------------------------------------------------------------ quant_row_flat
+
+// Blocks along contiguous rows for row lengths that are not a multiple of the 512-column tile of
+// quant_row_fast (K % b == 0, e.g. im2col matrices with K = 576 or 1152): the packed rows, padding
+// included, are cut into 8-element groups that are numbered through the whole matrix, and a warp takes
+// 32 consecutive groups wherever the row boundaries fall, so no lane idles on a ragged last tile.
+// CTA: 256 threads x 8 groups each (2048 consecutive groups).
+template <int LPB, bool SR, int PLANES>
+__global__ void __launch_bounds__(256)
+quant_row_flat(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, QParams p,
+               int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
+               int8_t* __restrict__ exps, int64_t rs, uint32_t gpr, uint32_t total_groups) {
+    constexpr int B = 8 * LPB;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const uint32_t g0 = blockIdx.x * 2048u + tid;
+    // (row, group in row) of this thread's first group; the next ones are 256 groups further on each
+    uint32_t row = g0 / gpr, cg = g0 - row * gpr;
+    const uint32_t q256 = 256u / gpr, r256 = 256u - q256 * gpr;
+    float4 v[8][2];
+    uint32_t rw[8], cc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        rw[j] = row;
+        cc[j] = cg * 8;
+        const bool in = g0 + j * 256u < total_groups && cc[j] < K;
+        if (in) {
+            const float4* src = reinterpret_cast<const float4*>(x + (int64_t)row * ld + cc[j]);
+            v[j][0] = __ldcs(src);
+            v[j][1] = __ldcs(src + 1);
+        } else {
+            v[j][0] = make_float4(0.f, 0.f, 0.f, 0.f);
+            v[j][1] = v[j][0];
+        }
+        row += q256;
+        cg += r256;
+        if (cg >= gpr) { cg -= gpr; ++row; }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const bool live = g0 + j * 256u < total_groups;      // uniform over the LPB lanes of a block
+        const float e8[8] = {v[j][0].x, v[j][0].y, v[j][0].z, v[j][0].w, v[j][1].x, v[j][1].y, v[j][1].z, v[j][1].w};
+        uint32_t am = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) am = max(am, abs_bits(e8[i]));
+#pragma unroll
+        for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        const int s = block_exponent(am, p.m, p.exp_mode);
+        int q[8];
+        if (SR) {
+            const uint64_t L0 = (uint64_t)rw[j] * (uint64_t)K + cc[j];     // multiple of 8 on this path
+            const uint4 w = draws_of_group(p, L0 >> 3);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i) q[i] = round_sr(e8[i], s, p.qmax, (ww[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) q[i] = round_rne(e8[i], s, p.qmax);
+        }
+        if (live) {
+            int8_t* dst = mant + (int64_t)rw[j] * kst + cc[j];
+            if (PLANES == 1) {
+                uint2 o;
+                o.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
+                o.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | ((uint32_t)(q[7] & 0xff) << 24);
+                *reinterpret_cast<uint2*>(dst) = o;
+            } else {
+                uint2 hi, lo;
+                hi.x = ((q[0] >> 4) & 0xff) | (((q[1] >> 4) & 0xff) << 8) | (((q[2] >> 4) & 0xff) << 16) | ((uint32_t)((q[3] >> 4) & 0xff) << 24);
+                hi.y = ((q[4] >> 4) & 0xff) | (((q[5] >> 4) & 0xff) << 8) | (((q[6] >> 4) & 0xff) << 16) | ((uint32_t)((q[7] >> 4) & 0xff) << 24);
+                lo.x = (q[0] & 15) | ((q[1] & 15) << 8) | ((q[2] & 15) << 16) | ((uint32_t)(q[3] & 15) << 24);
+                lo.y = (q[4] & 15) | ((q[5] & 15) << 8) | ((q[6] & 15) << 16) | ((uint32_t)(q[7] & 15) << 24);
+                *reinterpret_cast<uint2*>(dst) = hi;
+                *reinterpret_cast<uint2*>(dst + plane_stride) = lo;
+            }
+            // blocks that lie in the padding beyond K have no exponent
+            if ((lane % LPB) == 0 && cc[j] < K) exps[(int64_t)(cc[j] / B) * rs + rw[j]] = (int8_t)s;
+        }
+    }
+}
+
+template <int LPB>
+int launch_row_flat(const float* x, int64_t rows, int64_t K, int64_t ld, const QParams& p, const Layout& L,
+                    int8_t* mant, int8_t* exps, cudaStream_t st) {
+    const uint32_t gpr = (uint32_t)(L.kst / 8), total = (uint32_t)(rows * (L.kst / 8));
+    const unsigned grid = (total + 2047u) / 2048u;
+    if (p.rounding == 1) {
+        if (L.planes == 1) quant_row_flat<LPB, true, 1><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, gpr, total);
+        else quant_row_flat<LPB, true, 2><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, gpr, total);
+    } else {
+        if (L.planes == 1) quant_row_flat<LPB, false, 1><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, gpr, total);
+        else quant_row_flat<LPB, false, 2><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, gpr, total);
+    }
+    return launch_status();
+}
+
 // ------------------------------------------------------------------------------ quant_col_tma
 
 // Blocks down the columns of x [K][R] for b in {32, 64, 128}, the layout of the B operand of a
@@ -724,6 +821,18 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
     const bool aligned = ((reinterpret_cast<uintptr_t>(x) & 15) == 0) && (ld % 4 == 0);
     if (rows * L.kst >= (int64_t)1 << 40) return HBFP_ERR_UNSUPPORTED;
 
+    // row lengths that the 512-column tiles of quant_row_fast would leave ragged
+    if (f->tile == 0 && axis == 1 && aligned && L.b == L.bp && L.b <= 128 && K % L.b == 0 && L.kst % 512 != 0 &&
+        rows * (L.kst / 8) < (1ll << 32) - 4096) {
+        // exponent padding bytes (rows .. rs of every block line) are documented as zero
+        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        switch (L.b) {
+            case 32: return launch_row_flat<4>(x, rows, K, ld, p, L, mant, exps, st);
+            case 64: return launch_row_flat<8>(x, rows, K, ld, p, L, mant, exps, st);
+            case 128: return launch_row_flat<16>(x, rows, K, ld, p, L, mant, exps, st);
+            default: break;
+        }
+    }
     if (f->tile == 0 && axis == 1 && aligned && d1 % 8 == 0 && L.b == L.bp && L.b <= 256 &&
         rows <= 32ll * 65535) {
         switch (L.b) {

@@ -55,6 +55,24 @@ def test_row_blocks(hb, shape, law, fd):
     _check(hb, wl.draw(law, shape, seed=11), 1, fd)
 
 
+# Row lengths that are not a multiple of 512 (the im2col widths 576 and 1152 among them) take the
+# kernel that numbers 8-element groups through the whole matrix: warps straddle row ends, the packed
+# rows carry padding up to the next multiple of 128, and the last CTA is ragged.
+ROW_FLAT_CASES = [
+    ((300, 576), "half_normal", F(8, 64)),
+    ((257, 1152), "lognormal", F(12, 64, rounding=1, seed=5, sid=2)),
+    ((64, 2176), "grad", F(8, 128, rounding=1, seed=6)),
+    ((1000, 96), "outliers", F(8, 32)),
+    ((3, 640), "normal", F(6, 128, exp_mode=1)),
+    ((4099, 192), "lognormal", F(8, 64, rounding=1, seed=8)),
+]
+
+
+@pytest.mark.parametrize("shape,law,fd", ROW_FLAT_CASES)
+def test_row_blocks_ragged_row_lengths(hb, shape, law, fd):
+    _check(hb, wl.draw(law, shape, seed=16), 1, fd)
+
+
 COL_CASES = [
     ((784, 128), "half_normal", F(8, 24, rounding=1, seed=1)),
     ((1000, 300), "lognormal", F(12, 64)),
