@@ -341,8 +341,9 @@ def gpu_arm(args):
     int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
     gemm_tops = ops / (t_gemm * 1e-3) / 1e12
-    # the library takes the paired-SM kernel for one-plane operands with blocks up to 128 and >= 74 tiles of 256 x 256
-    paired = args.mant_bits <= 8 and 0 < args.block <= 128 and ((n + 255) // 256) ** 2 >= 74
+    # the library takes the paired-SM kernel for one-plane operands with blocks up to 128, >= 74 tiles of
+    # 256 x 256 and at least 1 KiB of mantissas per row
+    paired = args.mant_bits <= 8 and 0 < args.block <= 128 and ((n + 255) // 256) ** 2 >= 74 and n >= 1024
     roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel" if paired else "gemm_tc_kernel", "achieved": gemm_tops,
                 "peak": int8_burst,
                 "unit": "TOP/s", "frac": gemm_tops / int8_burst,

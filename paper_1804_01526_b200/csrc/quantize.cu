@@ -53,6 +53,70 @@ __device__ __forceinline__ float pow2f(int e) {   // 2^e for e in [-126, 127]
 
 __device__ __forceinline__ int clampq(int q, int qmax) { return max(-qmax, min(qmax, q)); }
 
+// Bit pattern of max(m, |a|, |b|) for finite values, in one three-input instruction.
+__device__ __forceinline__ uint32_t max3_abs_bits(uint32_t m, float a, float b) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(__uint_as_float(m)), "f"(fabsf(a)), "f"(fabsf(b)));
+    return __float_as_uint(d);
+}
+
+// Stochastic rounding of two neighbours whose 16-bit draws are the halves of one word w: the
+// floors of (Y + r) / 2^16 are the upper halfwords of the two sums, clamped as a signed pair.
+// Returns the two mantissas as packed signed halfwords (element 0 in the low half).
+__device__ __forceinline__ uint32_t round_sr_pair(float x0, float x1, float scale, uint32_t w, uint32_t qmax2, uint32_t nqmax2) {
+    const int t0 = __float2int_rd(__fmul_rn(x0, scale)) + (int)(w & 0xFFFFu);
+    const int t1 = __float2int_rd(__fmul_rn(x1, scale)) + (int)(w >> 16);
+    const uint32_t h = __byte_perm((uint32_t)t0, (uint32_t)t1, 0x7632);
+    return __vmaxs2(__vmins2(h, qmax2), nqmax2);
+}
+
+// Nearest-even rounding of two values, clamped as a signed halfword pair (m <= 12: the unclamped
+// value, at most 2^(m-1) in magnitude, fits a halfword).
+__device__ __forceinline__ uint32_t round_rne_pair(float x0, float x1, float scale, uint32_t qmax2, uint32_t nqmax2) {
+    const int q0 = __float2int_rn(__fmul_rn(x0, scale)), q1 = __float2int_rn(__fmul_rn(x1, scale));
+    const uint32_t h = __byte_perm((uint32_t)q0, (uint32_t)q1, 0x5410);
+    return __vmaxs2(__vmins2(h, qmax2), nqmax2);
+}
+
+__device__ __forceinline__ uint32_t qmax_pair(int qmax) { return (uint32_t)qmax * 0x10001u; }
+__device__ __forceinline__ uint32_t neg_qmax_pair(int qmax) { return ((uint32_t)(-qmax) & 0xFFFFu) * 0x10001u; }
+
+// Bytes of the mantissa planes from two halfword pairs (four mantissas): the 8-bit plane, or for
+// two planes (q = 16 hi + lo) bits 4..11 and bits 0..3 of every halfword.
+template <int PLANES>
+__device__ __forceinline__ void pack4(uint32_t h01, uint32_t h23, uint32_t& hi, uint32_t& lo) {
+    if (PLANES == 1) {
+        hi = __byte_perm(h01, h23, 0x6420);
+        lo = 0;
+    } else {
+        hi = __byte_perm((h01 >> 4) & 0x00FF00FFu, (h23 >> 4) & 0x00FF00FFu, 0x6420);
+        lo = __byte_perm(h01 & 0x000F000Fu, h23 & 0x000F000Fu, 0x6420);
+    }
+}
+
+// Largest |x| of eight values, as a bit pattern.
+__device__ __forceinline__ uint32_t amax8_bits(const float (&e8)[8]) {
+    uint32_t am = 0;
+#pragma unroll
+    for (int j = 0; j < 8; j += 2) am = max3_abs_bits(am, e8[j], e8[j + 1]);
+    return am;
+}
+
+// Rounds eight consecutive values that share the exponent s (w: their eight 16-bit draws in
+// stochastic mode) and packs the plane(s), eight bytes each.
+template <bool SR, int PLANES>
+__device__ __forceinline__ void quantize_pack8(const float (&e8)[8], int s, const QParams& p, uint4 w, uint2& hi, uint2& lo) {
+    const uint32_t qm = qmax_pair(p.qmax), nqm = neg_qmax_pair(p.qmax);
+    const float sc = pow2f(SR ? 16 - s : -s);
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    uint32_t h[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        h[j] = SR ? round_sr_pair(e8[2 * j], e8[2 * j + 1], sc, ww[j], qm, nqm) : round_rne_pair(e8[2 * j], e8[2 * j + 1], sc, qm, nqm);
+    pack4<PLANES>(h[0], h[1], hi.x, lo.x);
+    pack4<PLANES>(h[2], h[3], hi.y, lo.y);
+}
+
 // round-half-even( x * 2^-s ), saturated
 __device__ __forceinline__ int round_rne(float x, int s, int qmax) {
     float y = __fmul_rn(x, pow2f(-s));           // s >= -63 and s <= 126 for finite input, m >= 3
@@ -140,39 +204,17 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
             const int64_t r = r0 + warp * 4 + i;
             const float e8[8] = {v[i][0].x, v[i][0].y, v[i][0].z, v[i][0].w,
                                  v[i][1].x, v[i][1].y, v[i][1].z, v[i][1].w};
-            uint32_t am = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) am = max(am, abs_bits(e8[j]));
+            uint32_t am = amax8_bits(e8);
 #pragma unroll
             for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
             const int s = block_exponent(am, p.m, p.exp_mode);
-            int q[8];
-            if (SR) {
-                const uint64_t L0 = (uint64_t)(r * K + col);     // multiple of 8 on this path
-                const uint4 w = draws_of_group(p, L0 >> 3);
-                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    q[j] = round_sr(e8[j], s, p.qmax, (ww[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) q[j] = round_rne(e8[j], s, p.qmax);
-            }
+            uint4 w = make_uint4(0u, 0u, 0u, 0u);
+            if (SR) w = draws_of_group(p, (uint64_t)(r * K + col) >> 3);     // r * K + col is a multiple of 8 on this path
+            uint2 hi, lo;
+            quantize_pack8<SR, PLANES>(e8, s, p, w, hi, lo);
             if (r < rows && col < kst) {
-                if (PLANES == 1) {
-                    uint2 o;
-                    o.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
-                    o.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | ((uint32_t)(q[7] & 0xff) << 24);
-                    *reinterpret_cast<uint2*>(mant + r * kst + col) = o;
-                } else {
-                    uint2 hi, lo;
-                    hi.x = ((q[0] >> 4) & 0xff) | (((q[1] >> 4) & 0xff) << 8) | (((q[2] >> 4) & 0xff) << 16) | ((uint32_t)((q[3] >> 4) & 0xff) << 24);
-                    hi.y = ((q[4] >> 4) & 0xff) | (((q[5] >> 4) & 0xff) << 8) | (((q[6] >> 4) & 0xff) << 16) | ((uint32_t)((q[7] >> 4) & 0xff) << 24);
-                    lo.x = (q[0] & 15) | ((q[1] & 15) << 8) | ((q[2] & 15) << 16) | ((uint32_t)(q[3] & 15) << 24);
-                    lo.y = (q[4] & 15) | ((q[5] & 15) << 8) | ((q[6] & 15) << 16) | ((uint32_t)(q[7] & 15) << 24);
-                    *reinterpret_cast<uint2*>(mant + r * kst + col) = hi;
-                    *reinterpret_cast<uint2*>(mant + plane_stride + r * kst + col) = lo;
-                }
+                *reinterpret_cast<uint2*>(mant + r * kst + col) = hi;
+                if (PLANES == 2) *reinterpret_cast<uint2*>(mant + plane_stride + r * kst + col) = lo;
             }
             if ((lane % LPB) == 0 && r < rows && col < K)
                 s_exps[span * KB_PER_SPAN + lane / LPB][warp * 4 + i] = (int8_t)s;
@@ -551,39 +593,18 @@ quant_row_flat(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
     for (int j = 0; j < 8; ++j) {
         const bool live = g0 + j * 256u < total_groups;      // uniform over the LPB lanes of a block
         const float e8[8] = {v[j][0].x, v[j][0].y, v[j][0].z, v[j][0].w, v[j][1].x, v[j][1].y, v[j][1].z, v[j][1].w};
-        uint32_t am = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) am = max(am, abs_bits(e8[i]));
+        uint32_t am = amax8_bits(e8);
 #pragma unroll
         for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
         const int s = block_exponent(am, p.m, p.exp_mode);
-        int q[8];
-        if (SR) {
-            const uint64_t L0 = (uint64_t)rw[j] * (uint64_t)K + cc[j];     // multiple of 8 on this path
-            const uint4 w = draws_of_group(p, L0 >> 3);
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i) q[i] = round_sr(e8[i], s, p.qmax, (ww[i >> 1] >> (16 * (i & 1))) & 0xFFFFu);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) q[i] = round_rne(e8[i], s, p.qmax);
-        }
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (SR) w = draws_of_group(p, ((uint64_t)rw[j] * (uint64_t)K + cc[j]) >> 3);     // a multiple of 8 on this path
+        uint2 hi, lo;
+        quantize_pack8<SR, PLANES>(e8, s, p, w, hi, lo);
         if (live) {
             int8_t* dst = mant + (int64_t)rw[j] * kst + cc[j];
-            if (PLANES == 1) {
-                uint2 o;
-                o.x = (q[0] & 0xff) | ((q[1] & 0xff) << 8) | ((q[2] & 0xff) << 16) | ((uint32_t)(q[3] & 0xff) << 24);
-                o.y = (q[4] & 0xff) | ((q[5] & 0xff) << 8) | ((q[6] & 0xff) << 16) | ((uint32_t)(q[7] & 0xff) << 24);
-                *reinterpret_cast<uint2*>(dst) = o;
-            } else {
-                uint2 hi, lo;
-                hi.x = ((q[0] >> 4) & 0xff) | (((q[1] >> 4) & 0xff) << 8) | (((q[2] >> 4) & 0xff) << 16) | ((uint32_t)((q[3] >> 4) & 0xff) << 24);
-                hi.y = ((q[4] >> 4) & 0xff) | (((q[5] >> 4) & 0xff) << 8) | (((q[6] >> 4) & 0xff) << 16) | ((uint32_t)((q[7] >> 4) & 0xff) << 24);
-                lo.x = (q[0] & 15) | ((q[1] & 15) << 8) | ((q[2] & 15) << 16) | ((uint32_t)(q[3] & 15) << 24);
-                lo.y = (q[4] & 15) | ((q[5] & 15) << 8) | ((q[6] & 15) << 16) | ((uint32_t)(q[7] & 15) << 24);
-                *reinterpret_cast<uint2*>(dst) = hi;
-                *reinterpret_cast<uint2*>(dst + plane_stride) = lo;
-            }
+            *reinterpret_cast<uint2*>(dst) = hi;
+            if (PLANES == 2) *reinterpret_cast<uint2*>(dst + plane_stride) = lo;
             // blocks that lie in the padding beyond K have no exponent
             if ((lane % LPB) == 0 && cc[j] < K) exps[(int64_t)(cc[j] / B) * rs + rw[j]] = (int8_t)s;
         }
@@ -677,9 +698,10 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
         float v[32];
         uint32_t am = 0;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < 32; j += 2) {
             v[j] = tile[(q * 32 + j) * QC_COLS + n];
-            am = max(am, abs_bits(v[j]));
+            v[j + 1] = tile[(q * 32 + j + 1) * QC_COLS + n];
+            am = max3_abs_bits(am, v[j], v[j + 1]);
         }
         if (LB < 2) pmax[q * QC_COLS + n] = am;
         // the packed tile of the previous iteration must have left shared memory before it is rewritten
@@ -700,20 +722,24 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
         if ((q & ((4 >> LB) - 1)) == 0 && kb < nkb && col < R) exps[kb * rs + col] = (int8_t)sexp;
 
         uint32_t hi[8], lo[8];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { hi[w] = 0; lo[w] = 0; }
         const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
+        const uint32_t qm = qmax_pair(p.qmax), nqm = neg_qmax_pair(p.qmax);
+        const float sc = pow2f(SR ? 16 - sexp : -sexp);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            int qv;
-            if (SR) qv = round_sr(v[j], sexp, p.qmax, rnd16[(q * 32 + j) * QC_COLS + n]);
-            else qv = round_rne(v[j], sexp, p.qmax);
-            if (PLANES == 1) {
-                hi[j >> 2] |= (uint32_t)(qv & 0xff) << (8 * (j & 3));
-            } else {
-                hi[j >> 2] |= (uint32_t)((qv >> 4) & 0xff) << (8 * (j & 3));
-                lo[j >> 2] |= (uint32_t)(qv & 15) << (8 * (j & 3));
+        for (int w = 0; w < 8; ++w) {
+            uint32_t h[2];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int j = 4 * w + 2 * k;
+                if (SR) {
+                    // the draws of two vertical neighbours belong to different rows: two table entries
+                    const uint32_t r01 = (uint32_t)rnd16[(q * 32 + j) * QC_COLS + n] | ((uint32_t)rnd16[(q * 32 + j + 1) * QC_COLS + n] << 16);
+                    h[k] = round_sr_pair(v[j], v[j + 1], sc, r01, qm, nqm);
+                } else {
+                    h[k] = round_rne_pair(v[j], v[j + 1], sc, qm, nqm);
+                }
             }
+            pack4<PLANES>(h[0], h[1], hi[w], lo[w]);
         }
         // 128B swizzle of the store tile: 16-byte chunk c of row n sits at chunk position c ^ (n % 8)
         unsigned char* orow = base_ptr + (n >> 3) * 1024 + (n & 7) * 128;

@@ -4,7 +4,9 @@ For every GEMM of the benchmark configurations (single 256-cube, MLP step, ResNe
 convolutions, transformer layer, large sweep) it times, with CUDA events on the current stream,
 the conversion of each FP32 operand to block floating point and the BFP GEMM on already-packed
 operands, and prints one markdown table row per GEMM. Weights in shared tiles are converted once
-per layer (both views) and re-used by forward and backward-data, as in training.
+per layer (both views) and re-used by forward and backward-data, as in training. Calls shorter
+than 0.3 ms are timed as the per-call device time of 20 calls captured in one CUDA graph (their
+operands then sit in L2), since one event-timed call would measure the binding's host time.
 """
 from __future__ import annotations
 
@@ -33,6 +35,49 @@ def _time(fn, iters=10, warm=3):
     return statistics.median(ts)
 
 
+GRAPH_BELOW_MS = 0.3      # calls shorter than this are timed as a CUDA-graph replay
+GRAPH_CALLS = 20
+
+
+def _time_graph(fn, calls=GRAPH_CALLS, iters=10):
+    """Device time per call of ``calls`` back-to-back calls captured in one CUDA graph. For calls of
+    a few microseconds this leaves out the host time the Python binding spends per launch, which a
+    single event-timed call would measure instead of the kernels."""
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(calls):
+            fn()
+    return _time(g.replay, iters=iters) / calls
+
+
+def _time_auto(fn):
+    t = _time(fn)
+    return _time_graph(fn) if t < GRAPH_BELOW_MS else t
+
+
+def mlp_step_lines():
+    """The nine GEMMs of the MLP step, each with its conversions, as one captured graph."""
+    specs = wl.config_mlp()
+    t = wl.materialize(specs, seed=1)
+    dev = {k: torch.from_numpy(v).cuda() for k, v in t.items()}
+    outs = [torch.empty((sp.M, sp.N), dtype=torch.float32, device="cuda") for sp in specs]
+    fmts = [(hb.Format(**sp.fmt_a), hb.Format(**sp.fmt_b)) for sp in specs]
+    wss = [torch.empty(max(hb.gemm_workspace(sp.transA, sp.transB, sp.M, sp.N, sp.K, fa, fb), 1), dtype=torch.int8,
+                       device="cuda") for sp, (fa, fb) in zip(specs, fmts)]
+
+    def step():
+        for sp, (fa, fb), C, ws in zip(specs, fmts, outs, wss):
+            hb.gemm(sp.transA, sp.transB, dev[sp.a_key], dev[sp.b_key], fa, fb, out=C, workspace=ws)
+
+    t_eager = _time(step)
+    t_graph = _time_graph(step, calls=1)
+    ops = sum(sp.ops for sp in specs)
+    return [f"MLP step, 9 x hbfp_gemm (27 launches + memsets): {t_eager*1e3:.1f} us issued call by call from Python, "
+            f"{t_graph*1e3:.1f} us as one CUDA-graph replay ({ops/(t_graph*1e-3)/1e12:.2f} TOPS)"]
+
+
 def rows_for(specs, tensors_np, peak_tops, hbm_gbs):
     dev = {k: torch.from_numpy(v).cuda() for k, v in tensors_np.items()}
     out = []
@@ -42,17 +87,17 @@ def rows_for(specs, tensors_np, peak_tops, hbm_gbs):
         a_axis = 0 if sp.transA else 1           # contraction axis of the stored A
         b_axis = 1 if sp.transB else 0
         pa = hb.quantize(A, a_axis, fa)
-        t_qa = _time(lambda: hb.quantize(A, a_axis, fa, out=pa))
+        t_qa = _time_auto(lambda: hb.quantize(A, a_axis, fa, out=pa))
         if fb.tile > 0:
             c0, c1, _ = hb.quantize_tiles(B, fb)
-            t_qb = _time(lambda: hb.quantize_tiles(B, fb, out=(c0, c1), want_grid=False))
+            t_qb = _time_auto(lambda: hb.quantize_tiles(B, fb, out=(c0, c1), want_grid=False))
             pb = c1 if sp.transB else c0
         else:
             pb = hb.quantize(B, b_axis, fb)
-            t_qb = _time(lambda: hb.quantize(B, b_axis, fb, out=pb))
+            t_qb = _time_auto(lambda: hb.quantize(B, b_axis, fb, out=pb))
         C = torch.empty((sp.M, sp.N), dtype=torch.float32, device="cuda")
         ws = torch.empty(max(hb.gemm_q_workspace(sp.M, sp.N, sp.K, pa, pb), 1), dtype=torch.int8, device="cuda")
-        t_g = _time(lambda: hb.gemm_q(sp.M, sp.N, sp.K, pa, pb, out=C, workspace=ws))
+        t_g = _time_auto(lambda: hb.gemm_q(sp.M, sp.N, sp.K, pa, pb, out=C, workspace=ws))
         ops = sp.ops
         planes = 1 if fa.mant_bits <= 8 else 2
         qa_bytes = A.numel() * (4 + planes + 1.0 / max(fa.block, 1))
@@ -74,19 +119,27 @@ def main():
     ap.add_argument("--peak-tops", type=float, default=3266.6, help="int8 dense peak used for the % column")
     ap.add_argument("--hbm-gbs", type=float, default=6550.1)
     ap.add_argument("--sweep", type=int, nargs="*", default=[4096, 8192, 16384])
+    ap.add_argument("--only", default=None, help="time only the GEMMs whose name contains this text (e.g. for a profiler)")
     args = ap.parse_args()
     hb.lib()
     lines = ["| GEMM | M x N x K | format | quantise A µs | quantise B µs | GEMM µs | quantise A GB/s (% HBM) | GEMM-only TOPS | "
              "quantise+GEMM TOPS (% of measured int8 proxy / % of nominal 4500) |", "|---|---|---|---|---|---|---|---|---|"]
     for name, specs, seed in (("single", wl.config_single_256(), 0), ("mlp", wl.config_mlp(), 1),
                               ("resnet", wl.config_resnet_im2col(), 2), ("transformer", wl.config_transformer(), 7)):
-        lines += rows_for(specs, wl.materialize(specs, seed=seed), args.peak_tops, args.hbm_gbs)
+        if args.only:
+            specs = [sp for sp in specs if args.only in sp.name]
+        if specs:
+            lines += rows_for(specs, wl.materialize(specs, seed=seed), args.peak_tops, args.hbm_gbs)
     for n in args.sweep:
         for (m, b, r) in ((8, 128, 0), (8, 64, 0), (8, 32, 0), (8, 128, 1), (12, 64, 1)):
             specs = wl.config_sweep(n, m, b, r)
+            if args.only and args.only not in specs[0].name:
+                continue
             t = {specs[0].a_key: wl.draw("lognormal", (n, n), seed=3, salt=0),
                  specs[0].b_key: wl.draw("lognormal", (n, n), seed=3, salt=1)}
             lines += rows_for(specs, t, args.peak_tops, args.hbm_gbs)
+    if not args.only:
+        lines += [""] + mlp_step_lines()
     text = "\n".join(lines) + "\n"
     if args.out:
         with open(args.out, "w") as f:

@@ -185,3 +185,46 @@ def test_paired_sm_kernel_refuses_what_it_cannot_run(hb):
     with pytest.raises(hb.HbfpError) as e:           # two mantissa planes
         hb.gemm(0, 1, big, big, gfmt(f12), gfmt(f12), flags=hb.GEMM_FORCE_TENSOR_2SM)
     assert e.value.code == hb.ERR_UNSUPPORTED
+
+
+def test_mlp_step_captured_in_a_cuda_graph_replays_on_new_data(hb):
+    """The calls are stream-ordered and allocate nothing when given their buffers, so a whole
+    training step's GEMMs (stochastic rounding included: the draws depend on seed, stream id and
+    element index only) can be captured once and replayed on new contents of the same tensors."""
+    import torch
+    specs = wl.config_mlp()
+    t = wl.materialize(specs, seed=1)
+    dev = {k: to_dev(v) for k, v in t.items()}
+    outs = [torch.empty((sp.M, sp.N), dtype=torch.float32, device="cuda") for sp in specs]
+    wss = [torch.empty(max(hb.gemm_workspace(sp.transA, sp.transB, sp.M, sp.N, sp.K, gfmt(sp.fmt_a), gfmt(sp.fmt_b)), 1),
+                       dtype=torch.int8, device="cuda") for sp in specs]
+
+    def step():
+        for sp, C, ws in zip(specs, outs, wss):
+            hb.gemm(sp.transA, sp.transB, dev[sp.a_key], dev[sp.b_key], gfmt(sp.fmt_a), gfmt(sp.fmt_b),
+                    out=C, workspace=ws)
+
+    step()                                   # eager: also sets the kernels' attributes once
+    torch.cuda.synchronize()
+    eager = [C.clone() for C in outs]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for C in outs:
+        C.fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert hb.device_status() == 0
+    for sp, C, E in zip(specs, outs, eager):
+        assert torch.equal(C, E), sp.name
+    # new contents, same buffers: the replay must compute on them
+    t2 = wl.materialize(specs, seed=5)
+    for k, v in t2.items():
+        dev[k].copy_(to_dev(v))
+    graph.replay()
+    torch.cuda.synchronize()
+    assert hb.device_status() == 0
+    for sp, C in zip(specs, outs):
+        ref = oracle.hbfp_gemm(sp.transA, sp.transB, t2[sp.a_key], t2[sp.b_key], ofmt(sp.fmt_a), ofmt(sp.fmt_b))
+        err = np.abs(C.cpu().numpy().astype(np.float64) - ref["c_ref"].astype(np.float64))
+        assert (err <= TOL * ref["a_mag"]).all(), sp.name
