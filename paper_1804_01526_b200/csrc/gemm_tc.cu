@@ -14,8 +14,8 @@
 // int32 accumulator group in tensor memory. Groups form a ring, so the MMA of the next block
 // overlaps the rescale of the previous one. 12-bit mantissas (two int8 planes, q = 16 hi + lo): the
 // hi and lo planes of the B tile lie back to back in a stage, so each A plane is multiplied by both
-// in one MMA of width 2 N_TILE; two MMAs per step fill four accumulators (hi*hi | hi*lo, lo*hi |
-// lo*lo) that the rescale warps combine exactly in int32.
+// in one MMA of width 2 N_TILE, the two results overlapping in the middle: three accumulators
+// (hi*hi | hi*lo + lo*hi | lo*lo) that the rescale warps combine exactly in int32.
 //
 // Fast rescale (8-bit mantissas, blocks up to 256, so |P| < 2^22): integer-to-float conversion
 // runs on a slow pipe and an integer add per element would land on the FP32 pipe, so the
@@ -62,8 +62,8 @@ static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= 384 * 16
 
 template <int N_TILE, int PLANES>
 struct Cfg {
-    // accumulator parts per group; two planes: [hi.hi | hi.lo | lo.hi | lo.lo], each N_TILE columns
-    static constexpr int PARTS = PLANES == 1 ? 1 : 4;
+    // accumulator parts per group; two planes: [hi.hi | hi.lo + lo.hi | lo.lo], each N_TILE columns
+    static constexpr int PARTS = PLANES == 1 ? 1 : 3;
     static constexpr int GROUPS_RAW = TMEM_COLS / (N_TILE * PARTS);
     static constexpr int GROUPS = GROUPS_RAW > 4 ? 4 : GROUPS_RAW;
     static constexpr int A_BYTES = TILE_M * STAGE_K;              // per plane
@@ -193,8 +193,11 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
     constexpr int BPS = LNG ? 1 : 4 / SPB;
     // Two planes: the hi and lo planes of B lie back to back in a stage, so one MMA of twice the width
-    // multiplies an A plane by both (half as many MMAs, each A tile read from shared memory once).
-    constexpr uint32_t idesc = idesc_i8<PLANES * N_TILE>();
+    // (idesc2) multiplies an A plane by both: A_hi gives [hi.hi | hi.lo] from column 0 of the group,
+    // A_lo gives [lo.hi | lo.lo] from column N_TILE, so that the two cross terms add up in the middle
+    // part. Only the first step of a block, which must overwrite hi.hi and lo.lo but accumulate the
+    // second cross term, takes three MMAs.
+    constexpr uint32_t idesc = idesc_i8<N_TILE>(), idesc2 = idesc_i8<2 * N_TILE>();
     uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
     // The barriers the next MMAs will need are polled (without blocking) just before the last MMA
     // step of a block or stage is issued, while earlier MMAs still occupy the tensor pipe; a
@@ -213,6 +216,7 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
             const uint32_t ms = a.mant_base + s * C::MANT_STAGE;
             const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
             const uint64_t a_lo = smem_desc_sw128(ms + C::A_BYTES);
+            const uint64_t b_lo = smem_desc_sw128(ms + 2 * C::A_BYTES + C::B_BYTES);
             const int nb = LNG ? 1 : min(BPS, left);          // blocks that have steps in this stage
 #pragma unroll
             for (int jb = 0; jb < BPS; ++jb) {
@@ -245,8 +249,18 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
                         const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));      // 32 bytes per step, in 16-byte units
                         // biased path: always accumulate on top of the bias; else the first step of a block overwrites
                         const uint32_t acc = MAGIC ? 1u : (uint32_t)!(first && q == 0);
-                        if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
-                        if (PLANES == 2 && !(HBFP_TC_PROBE & 2)) tc_mma_i8(d + 2 * N_TILE, a_lo + ko, b_hi + ko, idesc, acc);
+                        if (PLANES == 1) {
+                            if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
+                        } else if (!(HBFP_TC_PROBE & 2)) {
+                            if (acc == 0u) {
+                                tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc2, 0u);
+                                tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, 0u);
+                                tc_mma_i8(d + N_TILE, a_hi + ko, b_lo + ko, idesc, 1u);
+                            } else {
+                                tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc2, 1u);
+                                tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc2, 1u);
+                            }
+                        }
                     }
                     if (last) {
                         tc_commit(a.tfull_bar + 8 * g);
@@ -526,13 +540,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         tc_ld16(taddr + ch * 16, v);
                         if (PLANES == 2) {
                             // mantissa = 16 hi + lo:  P = 256 hi.hi + 16 (hi.lo + lo.hi) + lo.lo
-                            uint32_t hl[16], lh[16], ll[16];
-                            tc_ld16(taddr + N_TILE + ch * 16, hl);
-                            tc_ld16(taddr + 2 * N_TILE + ch * 16, lh);
-                            tc_ld16(taddr + 3 * N_TILE + ch * 16, ll);
+                            uint32_t mid[16], ll[16];
+                            tc_ld16(taddr + N_TILE + ch * 16, mid);
+                            tc_ld16(taddr + 2 * N_TILE + ch * 16, ll);
                             tc_wait_ld();
 #pragma unroll
-                            for (int c = 0; c < 16; ++c) v[c] = (v[c] << 8) + ((hl[c] + lh[c]) << 4) + ll[c];
+                            for (int c = 0; c < 16; ++c) v[c] = (v[c] << 8) + (mid[c] << 4) + ll[c];
                         } else {
                             tc_wait_ld();
                         }
