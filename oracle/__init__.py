@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_quantize.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p]
         L.oracle_gemm.restype = ctypes.c_int
         L.oracle_gemm.argtypes = [i64, i64, i64, i64, p, p, p, p, p, p, p, p, ctypes.c_int]
+        L.oracle_wide_narrow.restype = ctypes.c_int
+        L.oracle_wide_narrow.argtypes = [p, p, i64, i64, ctypes.c_int, p, p]
+        L.oracle_wide_update.restype = ctypes.c_int
+        L.oracle_wide_update.argtypes = [p, p, p, i64, i64, i64, p]
         L.oracle_hbfp_gemm.restype = ctypes.c_int
         L.oracle_hbfp_gemm.argtypes = [ctypes.c_int, ctypes.c_int, i64, i64, i64, p, i64, p, i64,
                                        p, p, p, p, p]
@@ -207,3 +211,35 @@ def hbfp_gemm(transA: int, transB: int, A: np.ndarray, B: np.ndarray, fmtA: Form
     if rc:
         raise ValueError(f"oracle_hbfp_gemm failed: {rc}")
     return {"c_ref": c_ref, "a_mag": a_mag, "c_seq": c_seq}
+
+
+def wide_quantize(w: np.ndarray, fmt: Format):
+    """Wide weight storage of a stored weight matrix ``w [d0][d1]``: 16-bit mantissas ``q16 [d0][d1]``
+    and canonical exponents ``s16 [d0][ceil(d1/t)]``, one exponent per ``t x t`` tile (``fmt.tile``)."""
+    f16 = Format(**{**fmt.__dict__, "mant_bits": 16})
+    return quantize(w, 1, f16)
+
+
+def wide_narrow(q16: np.ndarray, s16: np.ndarray, mant_bits: int):
+    """The narrow copy the passes read: the ``mant_bits`` most significant bits of every mantissa."""
+    q16 = np.ascontiguousarray(q16, dtype=np.int16)
+    s16 = np.ascontiguousarray(s16, dtype=np.int8)
+    qm, sm = np.zeros_like(q16), np.zeros_like(s16)
+    rc = lib().oracle_wide_narrow(_ptr(q16), _ptr(s16), q16.size, s16.size, int(mant_bits), _ptr(qm), _ptr(sm))
+    if rc:
+        raise ValueError(f"oracle_wide_narrow failed: {rc}")
+    return qm, sm
+
+
+def wide_update(q16: np.ndarray, s16: np.ndarray, delta: np.ndarray, fmt: Format):
+    """``w = float32(q16 * 2^s16 + delta)`` re-quantised to wide storage; returns new ``(q16, s16)``."""
+    assert delta.dtype == np.float32 and delta.shape == q16.shape
+    q = np.ascontiguousarray(q16, dtype=np.int16).copy()
+    s = np.ascontiguousarray(s16, dtype=np.int8).copy()
+    delta = np.ascontiguousarray(delta)
+    d0, d1 = q.shape
+    cf = fmt._c()
+    rc = lib().oracle_wide_update(_ptr(q), _ptr(s), _ptr(delta), d1, d0, d1, ctypes.byref(cf))
+    if rc:
+        raise ValueError(f"oracle_wide_update failed: {rc}")
+    return q, s

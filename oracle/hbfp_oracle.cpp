@@ -15,14 +15,17 @@
 //   * dot product       : Eq. 2 (integer dot product of mantissas, scaled by 2^(ea+eb))
 //   * tiled product     : Sec. 4 after Eq. 2 and Sec. 4.2 "Tiling" (tile products in fixed
 //                         point, tiles accumulated in floating point)
+//   * wide weight storage: Sec. 4.2 (16-bit long-lived mantissas, the passes read the top bits)
 // Arithmetic is double / int64 throughout; nothing is blocked, fused or reordered.
 //
 // Pins (tests/test_oracle_*.py): exact-rational brute force of exponent + nearest rounding,
 // a float64 numpy restatement, idempotence, exact pass-through, power-of-two equivariance,
 // sign symmetry, half-ULP / one-ULP error bounds, exhaustive stochastic-rounding mean,
 // published Philox4x32-10 known answers, Eq. 2 against a float64 matmul of de-quantised
-// operands, exact-rational sums on tiny shapes and closed forms. No function here is
-// "parity unpinned".
+// operands, exact-rational sums on tiny shapes and closed forms; wide storage: the floor
+// bracket in exact rationals, agreement with direct quantisation on narrow-representable
+// weights, idempotence of the zero update, a binary32 numpy restatement of the update and
+// exact integer steps. No function here is "parity unpinned".
 
 #include <cmath>
 #include <cstdint>
@@ -305,6 +308,55 @@ int oracle_hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K,
     if (rc) return rc;
     return oracle_gemm(M, N, K, bA, qA.data(), sA.data(), qB.data(), sB.data(),
                        c_ref, a_mag, c_seq, nullptr, 0);
+}
+
+// ---------------------------------------------------------------------------------------
+// Wide weight storage (Sec. 4.2): the long-lived copy of a weight matrix keeps 16-bit
+// mantissas (one exponent per t x t tile); forward and backward passes read only the m most
+// significant bits of each mantissa. In canonical arrays:
+//   narrow mantissa = floor(q16 / 2^(16-m))     (the top m bits of the two's-complement word)
+//   narrow exponent = s16 + (16 - m)            (the weight of the narrow LSB)
+// so the narrow value never exceeds the wide one and lies less than one narrow ULP below it.
+// n_q mantissas, n_s exponents. Returns 0; -2 for m outside [2, 16].
+// ---------------------------------------------------------------------------------------
+int oracle_wide_narrow(const int16_t* q16, const int8_t* s16, int64_t n_q, int64_t n_s, int m,
+                       int16_t* qm, int8_t* sm) {
+    if (!q16 || !s16 || !qm || !sm || n_q < 0 || n_s < 0) return -1;
+    if (m < 2 || m > 16) return -2;
+    const int64_t d = (int64_t)1 << (16 - m);
+    for (int64_t i = 0; i < n_q; ++i) {
+        int64_t v = q16[i];
+        int64_t fl = v >= 0 ? v / d : -((-v + d - 1) / d);      // floor division
+        qm[i] = (int16_t)fl;
+    }
+    for (int64_t i = 0; i < n_s; ++i) sm[i] = (int8_t)(s16[i] + (16 - m));
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------
+// Weight update on wide storage (Sec. 4.2 "only weight updates use the wider mantissa";
+// Sec. 5.1: the update itself is computed in FP32, then the weights are converted back):
+//   w[i][j] = binary32( q16[i][j] * 2^s16 + delta[i][j] )      (q16 * 2^s16 is exact in binary32)
+//   (q16, s16) = 16-bit quantisation of w with one exponent per t x t tile of the stored matrix
+// q16 is [d0][d1], s16 is canonical [d0][ceil(d1/t)] (each row repeats its tile's exponent),
+// delta is [d0][d1] with row stride ldd. f gives tile (= block), rounding, exponent rule and
+// random stream; f->mant_bits is ignored (the wide width is 16). Returns what oracle_quantize returns.
+// ---------------------------------------------------------------------------------------
+int oracle_wide_update(int16_t* q16, int8_t* s16, const float* delta, int64_t ldd, int64_t d0, int64_t d1,
+                       const oracle_format* f) {
+    if (!q16 || !s16 || !delta || !f || d0 < 0 || d1 < 0 || ldd < d1) return -1;
+    if (f->tile <= 0 || f->block != f->tile) return -2;
+    const int64_t t = f->tile, nkb = (d1 + t - 1) / t;
+    std::vector<float> w((size_t)(d0 * d1));
+    for (int64_t i = 0; i < d0; ++i)
+        for (int64_t j = 0; j < d1; ++j) {
+            volatile float dq = std::ldexp((float)q16[i * d1 + j], (int)s16[i * nkb + j / t]);
+            volatile float sum = dq + delta[i * ldd + j];       // one binary32 rounding
+            w[(size_t)(i * d1 + j)] = sum;
+        }
+    oracle_format f16 = *f;
+    f16.mant_bits = 16;
+    return oracle_quantize(w.data(), d0, d1, d1, 1, &f16, q16, s16);
 }
 
 }  // extern "C"
