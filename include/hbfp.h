@@ -131,6 +131,36 @@ HBFP_API int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t
                                  const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0,
                                  void* mant_c1, int8_t* exps_c1, int8_t* tile_exps, void* stream);
 
+/* Wide weight storage (Sec. 4.2 "Wide weight storage": weights are kept with wider mantissas, only
+ * weight updates use them, and the forward and backward passes read only the most significant bits).
+ * The long-lived copy of w [d0][d1] is `wide`: int16 mantissas, row-major with pitch d1 (device,
+ * 2-byte aligned, d0 * d1 elements), and `wide_exps`: one int8 exponent (of the 16-bit LSB) per
+ * tile x tile square, [ceil(d0/t)][ceil(d1/t)] (device). fmt->tile == fmt->block = t in 1..128;
+ * fmt->rounding, seed, stream_id and exp_mode govern the conversion to 16 bits (stochastic rounding
+ * draws by the element's row-major index in w); fmt->mant_bits = m in 3..12 is the width of the narrow
+ * copy: its mantissas are the top m bits of the wide ones (floor(q16 / 2^(16-m)), which can reach
+ * -2^(m-1)) under the exponent s16 + 16 - m. The narrow copy is written as the two packed views of
+ * hbfp_quantize_tiles (`*_c0`: rows = d1, k = d0; `*_c1`: rows = d0, k = d1; buffers of the sizes
+ * hbfp_packed_sizes returns, fully overwritten); both mant_c0 and mant_c1 may be NULL to skip it, one
+ * of them alone may not.
+ *   hbfp_wide_quantize  w (FP32, pitch ld >= d1) -> wide storage (+ narrow views)
+ *   hbfp_wide_update    wide <- 16-bit quantisation of fl32(wide * 2^s16 + delta) with fresh tile
+ *                       exponents, in place; delta: FP32 [d0][d1], pitch ldd >= d1 (the update the
+ *                       optimiser computed in FP32, Sec. 5.1) (+ narrow views of the new weights)
+ *   hbfp_wide_narrow    wide storage -> narrow views only (reads 2 bytes per weight)
+ * One launch, one CTA per tile; asynchronous on `stream`. Errors: HBFP_ERR_INVALID_ARG (null or
+ * inconsistent arguments, tile != block), HBFP_ERR_UNSUPPORTED (tile > 128, m outside 3..12),
+ * HBFP_ERR_ALIGNMENT (view buffers as for hbfp_quantize). */
+HBFP_API int hbfp_wide_quantize(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* fmt,
+                                int16_t* wide, int8_t* wide_exps, void* mant_c0, int8_t* exps_c0,
+                                void* mant_c1, int8_t* exps_c1, void* stream);
+HBFP_API int hbfp_wide_update(int16_t* wide, int8_t* wide_exps, const float* delta, int64_t d0, int64_t d1,
+                              int64_t ldd, const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0,
+                              void* mant_c1, int8_t* exps_c1, void* stream);
+HBFP_API int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1,
+                              const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1,
+                              int8_t* exps_c1, void* stream);
+
 /* Packed -> canonical arrays for inspection: q [rows][k] int16 mantissas and s [rows][nkb]
  * int8 exponents (either may be NULL). */
 HBFP_API int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k,

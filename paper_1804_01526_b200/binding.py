@@ -27,7 +27,7 @@ EXPORTS = [
     "hbfp_status_string", "hbfp_packed_layout", "hbfp_packed_sizes", "hbfp_quantize",
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
-    "hbfp_device_status", "hbfp_gemm_static",
+    "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
 ]
 
 
@@ -89,6 +89,9 @@ def lib() -> ctypes.CDLL:
         L.hbfp_packed_sizes.argtypes = [i64, i64, p, p, p]
         L.hbfp_quantize.argtypes = [p, i64, i64, i64, i32, p, p, p, p]
         L.hbfp_quantize_tiles.argtypes = [p, i64, i64, i64, p, p, p, p, p, p, p]
+        L.hbfp_wide_quantize.argtypes = [p, i64, i64, i64, p, p, p, p, p, p, p, p]
+        L.hbfp_wide_update.argtypes = [p, p, p, i64, i64, i64, p, p, p, p, p, p]
+        L.hbfp_wide_narrow.argtypes = [p, p, i64, i64, p, p, p, p, p, p]
         L.hbfp_unpack.argtypes = [p, p, i64, i64, p, p, p, p]
         L.hbfp_dequantize.argtypes = [p, p, i64, i64, p, p, i64, p]
         L.hbfp_gemm_workspace.argtypes = [i32, i32, i64, i64, i64, p, p, p]
@@ -192,6 +195,69 @@ def quantize_tiles(w: torch.Tensor, fmt: Format, out: Optional[Tuple[Packed, Pac
                                      _dptr(c1.mant), _dptr(c1.exps), _dptr(grid), _stream()),
            "hbfp_quantize_tiles")
     return c0, c1, grid
+
+
+class Wide:
+    """Wide weight storage of ``w [d0][d1]``: int16 mantissas ``[d0][d1]`` and int8 tile exponents
+    ``[ceil(d0/t)][ceil(d1/t)]`` (device tensors)."""
+
+    def __init__(self, mant: torch.Tensor, exps: torch.Tensor, tile: int):
+        self.mant, self.exps, self.tile = mant, exps, tile
+
+
+def _alloc_views(d0: int, d1: int, fmt: Format, device) -> Tuple[Packed, Packed]:
+    return alloc_packed(d1, d0, fmt, device), alloc_packed(d0, d1, fmt, device)
+
+
+def _view_args(views: Optional[Tuple[Packed, Packed]]):
+    if views is None:
+        return [ctypes.c_void_p(0)] * 4
+    c0, c1 = views
+    return [_dptr(c0.mant), _dptr(c0.exps), _dptr(c1.mant), _dptr(c1.exps)]
+
+
+def wide_quantize(w: torch.Tensor, fmt: Format, out: Optional[Wide] = None, views: Optional[Tuple[Packed, Packed]] = None,
+                  want_views: bool = True):
+    """hbfp_wide_quantize: FP32 weights -> wide storage and (unless ``want_views`` is false) the two
+    packed narrow views of ``fmt.mant_bits`` bits. Returns ``(wide, (c0, c1) or None)``."""
+    _check_f32(w, "w")
+    d0, d1 = w.shape
+    t = fmt.tile
+    if out is None:
+        out = Wide(torch.empty((d0, d1), dtype=torch.int16, device=w.device),
+                   torch.empty((-(-d0 // t), -(-d1 // t)), dtype=torch.int8, device=w.device), t)
+    if views is None and want_views:
+        views = _alloc_views(d0, d1, fmt, w.device)
+    f = fmt.c()
+    _check(lib().hbfp_wide_quantize(_dptr(w), d0, d1, _ld(w), ctypes.byref(f), _dptr(out.mant), _dptr(out.exps),
+                                    *_view_args(views), _stream()), "hbfp_wide_quantize")
+    return out, views
+
+
+def wide_update(wide: Wide, delta: torch.Tensor, fmt: Format, views: Optional[Tuple[Packed, Packed]] = None,
+                want_views: bool = True):
+    """hbfp_wide_update: ``wide <- Q16(float32(wide + delta))`` in place; returns the narrow views."""
+    _check_f32(delta, "delta")
+    d0, d1 = wide.mant.shape
+    if tuple(delta.shape) != (d0, d1):
+        raise ValueError("delta must have the shape of the weights")
+    if views is None and want_views:
+        views = _alloc_views(d0, d1, fmt, delta.device)
+    f = fmt.c()
+    _check(lib().hbfp_wide_update(_dptr(wide.mant), _dptr(wide.exps), _dptr(delta), d0, d1, _ld(delta), ctypes.byref(f),
+                                  *_view_args(views), _stream()), "hbfp_wide_update")
+    return views
+
+
+def wide_narrow(wide: Wide, fmt: Format, views: Optional[Tuple[Packed, Packed]] = None) -> Tuple[Packed, Packed]:
+    """hbfp_wide_narrow: the two packed views of the top ``fmt.mant_bits`` bits of the wide mantissas."""
+    d0, d1 = wide.mant.shape
+    if views is None:
+        views = _alloc_views(d0, d1, fmt, wide.mant.device)
+    f = fmt.c()
+    _check(lib().hbfp_wide_narrow(_dptr(wide.mant), _dptr(wide.exps), d0, d1, ctypes.byref(f), *_view_args(views),
+                                  _stream()), "hbfp_wide_narrow")
+    return views
 
 
 def unpack(p: Packed) -> Tuple[torch.Tensor, torch.Tensor]:

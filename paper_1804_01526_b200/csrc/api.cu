@@ -205,6 +205,46 @@ int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, cons
                                  static_cast<cudaStream_t>(stream));
 }
 
+static int wide_views_ok(void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1) {
+    if (!mant_c0 && !mant_c1 && !exps_c0 && !exps_c1) return HBFP_OK;        // wide storage only
+    if (!mant_c0 || !exps_c0 || !mant_c1 || !exps_c1) return HBFP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mant_c0) & 255) || (reinterpret_cast<uintptr_t>(mant_c1) & 255) ||
+        (reinterpret_cast<uintptr_t>(exps_c0) & 127) || (reinterpret_cast<uintptr_t>(exps_c1) & 127))
+        return HBFP_ERR_ALIGNMENT;
+    return HBFP_OK;
+}
+
+int hbfp_wide_quantize(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* fmt, int16_t* wide,
+                       int8_t* wide_exps, void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
+    if (d0 < 0 || d1 < 0 || ld < d1 || !fmt) return HBFP_ERR_INVALID_ARG;
+    if ((!w && d0 * d1 > 0) || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
+    if (rc) return rc;
+    return launch_wide(0, w, ld, d0, d1, fmt, wide, wide_exps, static_cast<int8_t*>(mant_c0), exps_c0,
+                       static_cast<int8_t*>(mant_c1), exps_c1, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_wide_update(int16_t* wide, int8_t* wide_exps, const float* delta, int64_t d0, int64_t d1, int64_t ldd,
+                     const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
+    if (d0 < 0 || d1 < 0 || ldd < d1 || !fmt) return HBFP_ERR_INVALID_ARG;
+    if ((!delta && d0 * d1 > 0) || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
+    if (rc) return rc;
+    return launch_wide(1, delta, ldd, d0, d1, fmt, wide, wide_exps, static_cast<int8_t*>(mant_c0), exps_c0,
+                       static_cast<int8_t*>(mant_c1), exps_c1, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1, const hbfp_format* fmt,
+                     void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
+    if (d0 < 0 || d1 < 0 || !fmt || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    if (!mant_c0 || !mant_c1) return HBFP_ERR_INVALID_ARG;
+    int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
+    if (rc) return rc;
+    return launch_wide(2, nullptr, d1, d0, d1, fmt, const_cast<int16_t*>(wide), const_cast<int8_t*>(wide_exps),
+                       static_cast<int8_t*>(mant_c0), exps_c0, static_cast<int8_t*>(mant_c1), exps_c1,
+                       static_cast<cudaStream_t>(stream));
+}
+
 int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k, const hbfp_format* fmt,
                 int16_t* q, int8_t* s, void* stream) {
     Packed p;

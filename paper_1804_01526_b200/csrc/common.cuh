@@ -69,6 +69,11 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int cont
 int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* f,
                           int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
                           int8_t* tile_exps, cudaStream_t st);
+// Wide weight storage: mode 0 quantise FP32 weights, 1 apply an FP32 update in place, 2 read only; in every
+// mode the packed narrow views are written when their pointers are given.
+int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,
+                int16_t* wide, int8_t* wide_exps, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                cudaStream_t st);
 int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st);
 int launch_dequantize(const Packed& p, float* out, int64_t ld, cudaStream_t st);
 

@@ -346,6 +346,68 @@ quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, in
 
 // ------------------------------------------------------------------------------ quant_tiles
 
+// Writes one quantised t x t tile (qt: [tp][tp] int16, zero padded) into both packed views, with the
+// tile's exponent s replicated over its rows and columns, and zeroes the row tails beyond the last tile.
+// (u, v) = tile row / tile column; the tile covers hi x wj elements from (i0, j0).
+struct TileViews {
+    int8_t* mant_c0; int64_t kst0, ps0; int8_t* exps_c0; int64_t rs0, nkb0;
+    int8_t* mant_c1; int64_t kst1, ps1; int8_t* exps_c1; int64_t rs1, nkb1;
+};
+
+template <int PLANES>
+__device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int hi, int wj, int64_t i0, int64_t j0,
+                                                 int64_t u, int64_t v, int s, const TileViews& tv, int tid) {
+    int8_t* const mant_c0 = tv.mant_c0; int8_t* const mant_c1 = tv.mant_c1;
+    int8_t* const exps_c0 = tv.exps_c0; int8_t* const exps_c1 = tv.exps_c1;
+    const int64_t kst0 = tv.kst0, ps0 = tv.ps0, rs0 = tv.rs0, nkb0 = tv.nkb0;
+    const int64_t kst1 = tv.kst1, ps1 = tv.ps1, rs1 = tv.rs1, nkb1 = tv.nkb1;
+    // view c1: row i0+ii gets bytes [v*tp, v*tp+tp) = qt[ii][0..tp)
+    if (mant_c1) for (int e = tid; e < hi * (tp / 4); e += 256) {
+        const int ii = e / (tp / 4), g = (e % (tp / 4)) * 4;
+        uint32_t h = 0, l = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = qt[ii * tp + g + j];
+            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
+            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+        }
+        int8_t* dst = mant_c1 + (i0 + ii) * kst1 + v * tp + g;
+        *reinterpret_cast<uint32_t*>(dst) = h;
+        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps1) = l;
+    }
+    // view c0: row j0+jj gets bytes [u*tp, u*tp+tp) = qt[0..tp)[jj]
+    if (mant_c0) for (int e = tid; e < wj * (tp / 4); e += 256) {
+        const int jj = e % wj, g = (e / wj) * 4;
+        uint32_t h = 0, l = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int q = qt[(g + j) * tp + jj];
+            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
+            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+        }
+        int8_t* dst = mant_c0 + (j0 + jj) * kst0 + u * tp + g;
+        *reinterpret_cast<uint32_t*>(dst) = h;
+        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps0) = l;
+    }
+    // replicated exponents: exps_c1[v][i0+ii], exps_c0[u][j0+jj]
+    if (exps_c1) for (int e = tid; e < hi; e += 256) exps_c1[v * rs1 + i0 + e] = (int8_t)s;
+    if (exps_c0) for (int e = tid; e < wj; e += 256) exps_c0[u * rs0 + j0 + e] = (int8_t)s;
+    // row tails beyond the last tile: zero them (last tile column / last tile row only)
+    if (mant_c1 && v == nkb1 - 1)
+        for (int64_t e = tid; e < (int64_t)hi * ((kst1 - nkb1 * tp) / 4); e += 256) {
+            const int64_t per = (kst1 - nkb1 * tp) / 4, ii = e / per, o = nkb1 * tp + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(mant_c1 + (i0 + ii) * kst1 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c1 + ps1 + (i0 + ii) * kst1 + o) = 0;
+        }
+    if (mant_c0 && u == nkb0 - 1)
+        for (int64_t e = tid; e < (int64_t)wj * ((kst0 - nkb0 * tp) / 4); e += 256) {
+            const int64_t per = (kst0 - nkb0 * tp) / 4, jj = e / per, o = nkb0 * tp + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(mant_c0 + (j0 + jj) * kst0 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c0 + ps0 + (j0 + jj) * kst0 + o) = 0;
+        }
+}
+
+
 // One CTA per t x t tile of w [d0][d1] (t <= 128), 256 threads.
 //   view c1: rows = d0, contraction along d1 (the stored orientation)
 //   view c0: rows = d1, contraction along d0 (the transpose)
@@ -392,50 +454,87 @@ quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int
         qt[ii * tp + jj] = (int16_t)quantize_one(tile[ii * (t + 1) + jj], s, p, L);
     }
     __syncthreads();
-    // view c1: row i0+ii gets bytes [v*tp, v*tp+tp) = qt[ii][0..tp)
-    if (mant_c1) for (int e = tid; e < hi * (tp / 4); e += 256) {
-        const int ii = e / (tp / 4), g = (e % (tp / 4)) * 4;
-        uint32_t h = 0, l = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int q = qt[ii * tp + g + j];
-            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
-            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
+    const TileViews tv{mant_c0, kst0, ps0, exps_c0, rs0, nkb0, mant_c1, kst1, ps1, exps_c1, rs1, nkb1};
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s, tv, tid);
+}
+
+// ------------------------------------------------------------------------------ wide weight storage
+
+// Stochastic rounding to 16 bits: x * 2^(16-s) reaches 2^31, so the floor form runs in 64 bits.
+__device__ __forceinline__ int round_sr_wide(float x, int s, uint32_t r) {
+    const long long Y = __float2ll_rd(__fmul_rn(x, pow2f(16 - s)));
+    const long long q = (Y + (long long)r) >> 16;
+    return (int)max(-32767ll, min(32767ll, q));
+}
+
+// Wide weight storage (Sec. 4.2): w [d0][d1] lives as int16 mantissas (row-major, pitch d1) with one
+// exponent per t x t tile in grid [tiles along d0][tiles along d1]. One CTA per tile, 256 threads.
+//   MODE 0  quantise FP32 weights src [d0][d1] (pitch ld) to wide storage
+//   MODE 1  update: w = fl32(wide * 2^s + src) with src the FP32 update, re-quantised in place
+//   MODE 2  read wide storage only
+// and, in every mode, when view pointers are given: the two packed narrow views of the tile, whose
+// mantissas are the top narrow_m bits of the wide ones (an arithmetic shift) under the exponent
+// s + 16 - narrow_m.
+template <int MODE, int PLANES>
+__global__ void __launch_bounds__(256)
+wide_tiles(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, int t, int tp, QParams p, int narrow_m,
+           int16_t* __restrict__ wide, int8_t* __restrict__ grid, int64_t grid_ld, TileViews tv) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* tile = reinterpret_cast<float*>(smem_raw);                      // [t][t+1]
+    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp] zero padded
+    __shared__ uint32_t s_am[8];
+    __shared__ int s_exp;
+
+    const int tid = threadIdx.x;
+    const int64_t u = blockIdx.y, v = blockIdx.x;
+    const int64_t i0 = u * t, j0 = v * t;
+    const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
+    for (int e = tid; e < tp * tp; e += 256) qt[e] = 0;
+    int s;
+    if (MODE == 2) {
+        __syncthreads();
+        s = grid[u * grid_ld + v];
+        for (int e = tid; e < hi * wj; e += 256) {
+            const int ii = e / wj, jj = e % wj;
+            qt[ii * tp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
         }
-        int8_t* dst = mant_c1 + (i0 + ii) * kst1 + v * tp + g;
-        *reinterpret_cast<uint32_t*>(dst) = h;
-        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps1) = l;
+    } else {
+        const float old_scale = MODE == 1 ? pow2f(grid[u * grid_ld + v]) : 0.f;
+        uint32_t am = 0;
+        for (int e = tid; e < hi * wj; e += 256) {
+            const int ii = e / wj, jj = e % wj;
+            float val = src[(i0 + ii) * ld + j0 + jj];
+            if (MODE == 1) val = __fadd_rn(__fmul_rn((float)wide[(i0 + ii) * d1 + j0 + jj], old_scale), val);
+            tile[ii * (t + 1) + jj] = val;
+            am = max(am, abs_bits(val));
+        }
+        for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        if ((tid & 31) == 0) s_am[tid >> 5] = am;
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t a = 0;
+            for (int i = 0; i < 8; ++i) a = max(a, s_am[i]);
+            s_exp = block_exponent(a, 16, p.exp_mode);
+            grid[u * grid_ld + v] = (int8_t)s_exp;
+        }
+        __syncthreads();
+        s = s_exp;
+        for (int e = tid; e < hi * wj; e += 256) {
+            const int ii = e / wj, jj = e % wj;
+            const float val = tile[ii * (t + 1) + jj];
+            int q;
+            if (p.rounding == 0) q = round_rne(val, s, 32767);
+            else q = round_sr_wide(val, s, draw_of_element(p, (uint64_t)((i0 + ii) * d1 + j0 + jj)));
+            qt[ii * tp + jj] = (int16_t)q;
+            wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
+        }
     }
-    // view c0: row j0+jj gets bytes [u*tp, u*tp+tp) = qt[0..tp)[jj]
-    if (mant_c0) for (int e = tid; e < wj * (tp / 4); e += 256) {
-        const int jj = e % wj, g = (e / wj) * 4;
-        uint32_t h = 0, l = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int q = qt[(g + j) * tp + jj];
-            if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
-            else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
-        }
-        int8_t* dst = mant_c0 + (j0 + jj) * kst0 + u * tp + g;
-        *reinterpret_cast<uint32_t*>(dst) = h;
-        if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps0) = l;
-    }
-    // replicated exponents: exps_c1[v][i0+ii], exps_c0[u][j0+jj]
-    if (exps_c1) for (int e = tid; e < hi; e += 256) exps_c1[v * rs1 + i0 + e] = (int8_t)s;
-    if (exps_c0) for (int e = tid; e < wj; e += 256) exps_c0[u * rs0 + j0 + e] = (int8_t)s;
-    // row tails beyond the last tile: zero them (last tile column / last tile row only)
-    if (mant_c1 && v == nkb1 - 1)
-        for (int64_t e = tid; e < (int64_t)hi * ((kst1 - nkb1 * tp) / 4); e += 256) {
-            const int64_t per = (kst1 - nkb1 * tp) / 4, ii = e / per, o = nkb1 * tp + (e % per) * 4;
-            *reinterpret_cast<uint32_t*>(mant_c1 + (i0 + ii) * kst1 + o) = 0;
-            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c1 + ps1 + (i0 + ii) * kst1 + o) = 0;
-        }
-    if (mant_c0 && u == nkb0 - 1)
-        for (int64_t e = tid; e < (int64_t)wj * ((kst0 - nkb0 * tp) / 4); e += 256) {
-            const int64_t per = (kst0 - nkb0 * tp) / 4, jj = e / per, o = nkb0 * tp + (e % per) * 4;
-            *reinterpret_cast<uint32_t*>(mant_c0 + (j0 + jj) * kst0 + o) = 0;
-            if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant_c0 + ps0 + (j0 + jj) * kst0 + o) = 0;
-        }
+    if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
+    __syncthreads();
+    const int sh = 16 - narrow_m;
+    for (int e = tid; e < hi * tp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
+    __syncthreads();
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, tv, tid);
 }
 
 // ------------------------------------------------------------------------------ generic two-pass path
@@ -956,6 +1055,40 @@ int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, co
         quant_tiles<2><<<grid, 256, smem, st>>>(w, d0, d1, ld, t, tp, p, mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb,
                                                mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb, tile_exps, nv);
     }
+    return launch_status();
+}
+
+int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,
+                int16_t* wide, int8_t* wide_exps, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                cudaStream_t st) {
+    if (f->tile <= 0 || f->tile != f->block) return HBFP_ERR_INVALID_ARG;
+    if (f->tile > 128) return HBFP_ERR_UNSUPPORTED;
+    Layout L0, L1;
+    int rc = make_layout(d1, d0, f, &L0);     // view c0: rows = d1, k = d0
+    if (rc) return rc;
+    rc = make_layout(d0, d1, f, &L1);         // view c1: rows = d0, k = d1
+    if (rc) return rc;
+    if (d0 == 0 || d1 == 0) return HBFP_OK;
+    const QParams p = make_params(f);         // rounding, exponent rule and random stream (the wide width is 16)
+    const int t = f->tile, tp = (int)L0.bp;
+    const int64_t nu = L0.nkb, nv = L1.nkb;   // tiles along d0, along d1
+    if (nu > 65535) return HBFP_ERR_UNSUPPORTED;
+    if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
+    if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
+    const TileViews tv{mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb, mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb};
+    const size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * tp * sizeof(int16_t);
+    const dim3 grid((unsigned)nv, (unsigned)nu);
+#define HBFP_WIDE_LAUNCH(MODE, PLANES)                                                                                  \
+    do {                                                                                                                \
+        HBFP_CUDA_OK(cudaFuncSetAttribute(wide_tiles<MODE, PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        wide_tiles<MODE, PLANES><<<grid, 256, smem, st>>>(src, ld, d0, d1, t, tp, p, f->mant_bits, wide, wide_exps, nv, tv);  \
+    } while (0)
+    if (L0.planes == 1) {
+        if (mode == 0) HBFP_WIDE_LAUNCH(0, 1); else if (mode == 1) HBFP_WIDE_LAUNCH(1, 1); else HBFP_WIDE_LAUNCH(2, 1);
+    } else {
+        if (mode == 0) HBFP_WIDE_LAUNCH(0, 2); else if (mode == 1) HBFP_WIDE_LAUNCH(1, 2); else HBFP_WIDE_LAUNCH(2, 2);
+    }
+#undef HBFP_WIDE_LAUNCH
     return launch_status();
 }
 
