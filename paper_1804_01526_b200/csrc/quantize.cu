@@ -354,20 +354,23 @@ struct TileViews {
     int8_t* mant_c1; int64_t kst1, ps1; int8_t* exps_c1; int64_t rs1, nkb1;
 };
 
+// qt rows have a pitch of tp + 2 halfwords, so that the column reads of view c0 spread over the banks.
 template <int PLANES>
 __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int hi, int wj, int64_t i0, int64_t j0,
                                                  int64_t u, int64_t v, int s, const TileViews& tv, int tid) {
+    const int qp = tp + 2;
+    const int lg = 31 - __clz(tp >> 2), gmask = (tp >> 2) - 1;       // tp is 32, 64 or 128
     int8_t* const mant_c0 = tv.mant_c0; int8_t* const mant_c1 = tv.mant_c1;
     int8_t* const exps_c0 = tv.exps_c0; int8_t* const exps_c1 = tv.exps_c1;
     const int64_t kst0 = tv.kst0, ps0 = tv.ps0, rs0 = tv.rs0, nkb0 = tv.nkb0;
     const int64_t kst1 = tv.kst1, ps1 = tv.ps1, rs1 = tv.rs1, nkb1 = tv.nkb1;
     // view c1: row i0+ii gets bytes [v*tp, v*tp+tp) = qt[ii][0..tp)
     if (mant_c1) for (int e = tid; e < hi * (tp / 4); e += 256) {
-        const int ii = e / (tp / 4), g = (e % (tp / 4)) * 4;
+        const int ii = e >> lg, g = (e & gmask) * 4;
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[ii * tp + g + j];
+            const int q = qt[ii * qp + g + j];
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -376,12 +379,13 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + ps1) = l;
     }
     // view c0: row j0+jj gets bytes [u*tp, u*tp+tp) = qt[0..tp)[jj]
+    // (neighbouring threads write neighbouring words of one output row)
     if (mant_c0) for (int e = tid; e < wj * (tp / 4); e += 256) {
-        const int jj = e % wj, g = (e / wj) * 4;
+        const int jj = e >> lg, g = (e & gmask) * 4;
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[(g + j) * tp + jj];
+            const int q = qt[(g + j) * qp + jj];
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -419,7 +423,7 @@ quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int
             int8_t* __restrict__ grid, int64_t grid_ld) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* tile = reinterpret_cast<float*>(smem_raw);                  // [t][t+1]
-    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp] zero padded
+    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp + 2] zero padded
     __shared__ uint32_t s_am[8];
     __shared__ int s_exp;
 
@@ -428,17 +432,17 @@ quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int
     const int64_t i0 = u * t, j0 = v * t;
     const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
 
+    const int lane = tid & 31, wrow = tid >> 5, qp = tp + 2;
     uint32_t am = 0;
-    for (int e = tid; e < hi * t; e += 256) {
-        const int ii = e / t, jj = e % t;
-        float val = 0.f;
-        if (jj < wj) val = w[(i0 + ii) * ld + j0 + jj];
-        tile[ii * (t + 1) + jj] = val;
-        am = max(am, abs_bits(val));
-    }
-    for (int e = tid; e < tp * tp; e += 256) qt[e] = 0;
+    for (int ii = wrow; ii < hi; ii += 8)
+        for (int jj = lane; jj < wj; jj += 32) {
+            const float val = w[(i0 + ii) * ld + j0 + jj];
+            tile[ii * (t + 1) + jj] = val;
+            am = max(am, abs_bits(val));
+        }
+    for (int e = tid; e < tp * qp; e += 256) qt[e] = 0;
     for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
-    if ((tid & 31) == 0) s_am[tid >> 5] = am;
+    if (lane == 0) s_am[wrow] = am;
     __syncthreads();
     if (tid == 0) {
         uint32_t a = 0;
@@ -448,11 +452,11 @@ quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int
     }
     __syncthreads();
     const int s = s_exp;
-    for (int e = tid; e < hi * wj; e += 256) {
-        const int ii = e / wj, jj = e % wj;
-        const uint64_t L = (uint64_t)((i0 + ii) * d1 + j0 + jj);
-        qt[ii * tp + jj] = (int16_t)quantize_one(tile[ii * (t + 1) + jj], s, p, L);
-    }
+    for (int ii = wrow; ii < hi; ii += 8)
+        for (int jj = lane; jj < wj; jj += 32) {
+            const uint64_t L = (uint64_t)((i0 + ii) * d1 + j0 + jj);
+            qt[ii * qp + jj] = (int16_t)quantize_one(tile[ii * (t + 1) + jj], s, p, L);
+        }
     __syncthreads();
     const TileViews tv{mant_c0, kst0, ps0, exps_c0, rs0, nkb0, mant_c1, kst1, ps1, exps_c1, rs1, nkb1};
     write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s, tv, tid);
@@ -481,7 +485,7 @@ wide_tiles(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, in
            int16_t* __restrict__ wide, int8_t* __restrict__ grid, int64_t grid_ld, TileViews tv) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* tile = reinterpret_cast<float*>(smem_raw);                      // [t][t+1]
-    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp] zero padded
+    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp + 2] zero padded
     __shared__ uint32_t s_am[8];
     __shared__ int s_exp;
 
@@ -489,27 +493,26 @@ wide_tiles(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, in
     const int64_t u = blockIdx.y, v = blockIdx.x;
     const int64_t i0 = u * t, j0 = v * t;
     const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
-    for (int e = tid; e < tp * tp; e += 256) qt[e] = 0;
+    const int lane = tid & 31, wrow = tid >> 5, qp = tp + 2;
+    for (int e = tid; e < tp * qp; e += 256) qt[e] = 0;
     int s;
     if (MODE == 2) {
         __syncthreads();
         s = grid[u * grid_ld + v];
-        for (int e = tid; e < hi * wj; e += 256) {
-            const int ii = e / wj, jj = e % wj;
-            qt[ii * tp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
-        }
+        for (int ii = wrow; ii < hi; ii += 8)
+            for (int jj = lane; jj < wj; jj += 32) qt[ii * qp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
     } else {
         const float old_scale = MODE == 1 ? pow2f(grid[u * grid_ld + v]) : 0.f;
         uint32_t am = 0;
-        for (int e = tid; e < hi * wj; e += 256) {
-            const int ii = e / wj, jj = e % wj;
-            float val = src[(i0 + ii) * ld + j0 + jj];
-            if (MODE == 1) val = __fadd_rn(__fmul_rn((float)wide[(i0 + ii) * d1 + j0 + jj], old_scale), val);
-            tile[ii * (t + 1) + jj] = val;
-            am = max(am, abs_bits(val));
-        }
+        for (int ii = wrow; ii < hi; ii += 8)
+            for (int jj = lane; jj < wj; jj += 32) {
+                float val = src[(i0 + ii) * ld + j0 + jj];
+                if (MODE == 1) val = __fadd_rn(__fmul_rn((float)wide[(i0 + ii) * d1 + j0 + jj], old_scale), val);
+                tile[ii * (t + 1) + jj] = val;
+                am = max(am, abs_bits(val));
+            }
         for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
-        if ((tid & 31) == 0) s_am[tid >> 5] = am;
+        if (lane == 0) s_am[wrow] = am;
         __syncthreads();
         if (tid == 0) {
             uint32_t a = 0;
@@ -519,20 +522,20 @@ wide_tiles(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, in
         }
         __syncthreads();
         s = s_exp;
-        for (int e = tid; e < hi * wj; e += 256) {
-            const int ii = e / wj, jj = e % wj;
-            const float val = tile[ii * (t + 1) + jj];
-            int q;
-            if (p.rounding == 0) q = round_rne(val, s, 32767);
-            else q = round_sr_wide(val, s, draw_of_element(p, (uint64_t)((i0 + ii) * d1 + j0 + jj)));
-            qt[ii * tp + jj] = (int16_t)q;
-            wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
-        }
+        for (int ii = wrow; ii < hi; ii += 8)
+            for (int jj = lane; jj < wj; jj += 32) {
+                const float val = tile[ii * (t + 1) + jj];
+                int q;
+                if (p.rounding == 0) q = round_rne(val, s, 32767);
+                else q = round_sr_wide(val, s, draw_of_element(p, (uint64_t)((i0 + ii) * d1 + j0 + jj)));
+                qt[ii * qp + jj] = (int16_t)q;
+                wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
+            }
     }
     if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
     __syncthreads();
     const int sh = 16 - narrow_m;
-    for (int e = tid; e < hi * tp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
+    for (int e = tid; e < hi * qp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
     __syncthreads();
     write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, tv, tid);
 }
@@ -1044,7 +1047,7 @@ int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, co
     if (nu > 65535) return HBFP_ERR_UNSUPPORTED;
     if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
     if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
-    size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * tp * sizeof(int16_t);
+    size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
     dim3 grid((unsigned)nv, (unsigned)nu);
     if (L0.planes == 1) {
         HBFP_CUDA_OK(cudaFuncSetAttribute(quant_tiles<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -1076,7 +1079,7 @@ int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, 
     if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
     if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
     const TileViews tv{mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb, mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb};
-    const size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * tp * sizeof(int16_t);
+    const size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
     const dim3 grid((unsigned)nv, (unsigned)nu);
 #define HBFP_WIDE_LAUNCH(MODE, PLANES)                                                                                  \
     do {                                                                                                                \

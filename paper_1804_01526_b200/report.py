@@ -78,6 +78,35 @@ def mlp_step_lines():
             f"{t_graph*1e3:.1f} us as one CUDA-graph replay ({ops/(t_graph*1e-3)/1e12:.2f} TOPS)"]
 
 
+def wide_lines(hbm_gbs):
+    """Wide weight storage on the weight matrices of the configurations: first conversion, in-place
+    FP32 update (with the narrow views of the new weights) and the narrow views alone."""
+    out = ["", "| weights | format | wide quantise µs | wide update + views µs (GB/s, % HBM) | narrow views only µs | FP32 -> views (`hbfp_quantize_tiles`) µs |",
+           "|---|---|---|---|---|---|"]
+    for name, shape, fd in (("c1.l1.W", (1024, 1024), dict(mant_bits=8, block=24, tile=24, rounding=1, seed=1)),
+                            ("c3.up.W", (1024, 4096), dict(mant_bits=12, block=64, tile=64, rounding=1, seed=7)),
+                            ("8192 x 8192", (8192, 8192), dict(mant_bits=8, block=64, tile=64, rounding=0)),
+                            ("16384 x 16384", (16384, 16384), dict(mant_bits=8, block=128, tile=128, rounding=0))):
+        fmt = hb.Format(**fd)
+        w = torch.from_numpy(wl.draw("he_weight", shape, seed=3, fan_in=shape[0])).cuda()
+        dw = torch.from_numpy(wl.draw("grad", shape, seed=4)).cuda()
+        wide, views = hb.wide_quantize(w, fmt)
+        t_q = _time_auto(lambda: hb.wide_quantize(w, fmt, out=wide, views=views))
+        t_u = _time_auto(lambda: hb.wide_update(wide, dw, fmt, views=views))
+        t_n = _time_auto(lambda: hb.wide_narrow(wide, fmt, views=views))
+        t_t = _time_auto(lambda: hb.quantize_tiles(w, fmt, out=views, want_grid=False))
+        planes = 1 if fd["mant_bits"] <= 8 else 2
+        n = shape[0] * shape[1]
+        bytes_u = n * (2 + 4 + 2 + 2 * planes)          # read wide + delta, write wide + both views
+        gbs = bytes_u / (t_u * 1e-3) / 1e9
+        f = f"m{fd['mant_bits']} t{fd['tile']}" + (" SR" if fd["rounding"] else " RNE")
+        out.append(f"| {name} {shape[0]}x{shape[1]} | {f} | {t_q*1e3:.1f} | {t_u*1e3:.1f} ({gbs:.0f}, {100*gbs/hbm_gbs:.0f} %) | "
+                   f"{t_n*1e3:.1f} | {t_t*1e3:.1f} |")
+        del w, dw, wide, views
+    torch.cuda.empty_cache()
+    return out
+
+
 def rows_for(specs, tensors_np, peak_tops, hbm_gbs):
     dev = {k: torch.from_numpy(v).cuda() for k, v in tensors_np.items()}
     out = []
@@ -140,6 +169,8 @@ def main():
             lines += rows_for(specs, t, args.peak_tops, args.hbm_gbs)
     if not args.only:
         lines += [""] + mlp_step_lines()
+    if not args.only or args.only == "wide":
+        lines += wide_lines(args.hbm_gbs)
     text = "\n".join(lines) + "\n"
     if args.out:
         with open(args.out, "w") as f:
