@@ -15,7 +15,7 @@
 //   quant_col_fast   blocks down the columns, any b <= 128 and any pitch: a (<=128) x 32 FP32
 //                    panel is read with coalesced row loads into shared memory, reduced down the
 //                    columns by four threads per column and written transposed.
-//   quant_tiles      t x t weight tiles (t <= 128): one pass writes both packed views and
+//   tile_kernel      t x t weight tiles (t <= 128): one pass writes both packed views and
 //                    the tile exponent grid.
 //   exps_* / mant_generic   two-pass path for every other geometry (any b, any alignment).
 #include "common.cuh"
@@ -344,7 +344,7 @@ quant_col_fast(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, in
     }
 }
 
-// ------------------------------------------------------------------------------ quant_tiles
+// ------------------------------------------------------------------------------ weight tiles
 
 // Writes one quantised t x t tile (qt: [tp][tp] int16, zero padded) into both packed views, with the
 // tile's exponent s replicated over its rows and columns, and zeroes the row tails beyond the last tile.
@@ -412,58 +412,6 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
 }
 
 
-// One CTA per t x t tile of w [d0][d1] (t <= 128), 256 threads.
-//   view c1: rows = d0, contraction along d1 (the stored orientation)
-//   view c0: rows = d1, contraction along d0 (the transpose)
-template <int PLANES>
-__global__ void __launch_bounds__(256)
-quant_tiles(const float* __restrict__ w, int64_t d0, int64_t d1, int64_t ld, int t, int tp, QParams p,
-            int8_t* __restrict__ mant_c0, int64_t kst0, int64_t ps0, int8_t* __restrict__ exps_c0, int64_t rs0, int64_t nkb0,
-            int8_t* __restrict__ mant_c1, int64_t kst1, int64_t ps1, int8_t* __restrict__ exps_c1, int64_t rs1, int64_t nkb1,
-            int8_t* __restrict__ grid, int64_t grid_ld) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* tile = reinterpret_cast<float*>(smem_raw);                  // [t][t+1]
-    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp + 2] zero padded
-    __shared__ uint32_t s_am[8];
-    __shared__ int s_exp;
-
-    const int tid = threadIdx.x;
-    const int64_t u = blockIdx.y, v = blockIdx.x;       // tile row (along d0), tile column (along d1)
-    const int64_t i0 = u * t, j0 = v * t;
-    const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
-
-    const int lane = tid & 31, wrow = tid >> 5, qp = tp + 2;
-    uint32_t am = 0;
-    for (int ii = wrow; ii < hi; ii += 8)
-        for (int jj = lane; jj < wj; jj += 32) {
-            const float val = w[(i0 + ii) * ld + j0 + jj];
-            tile[ii * (t + 1) + jj] = val;
-            am = max(am, abs_bits(val));
-        }
-    for (int e = tid; e < tp * qp; e += 256) qt[e] = 0;
-    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
-    if (lane == 0) s_am[wrow] = am;
-    __syncthreads();
-    if (tid == 0) {
-        uint32_t a = 0;
-        for (int i = 0; i < 8; ++i) a = max(a, s_am[i]);
-        s_exp = block_exponent(a, p.m, p.exp_mode);
-        if (grid) grid[u * grid_ld + v] = (int8_t)s_exp;
-    }
-    __syncthreads();
-    const int s = s_exp;
-    for (int ii = wrow; ii < hi; ii += 8)
-        for (int jj = lane; jj < wj; jj += 32) {
-            const uint64_t L = (uint64_t)((i0 + ii) * d1 + j0 + jj);
-            qt[ii * qp + jj] = (int16_t)quantize_one(tile[ii * (t + 1) + jj], s, p, L);
-        }
-    __syncthreads();
-    const TileViews tv{mant_c0, kst0, ps0, exps_c0, rs0, nkb0, mant_c1, kst1, ps1, exps_c1, rs1, nkb1};
-    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s, tv, tid);
-}
-
-// ------------------------------------------------------------------------------ wide weight storage
-
 // Stochastic rounding to 16 bits: x * 2^(16-s) reaches 2^31, so the floor form runs in 64 bits.
 __device__ __forceinline__ int round_sr_wide(float x, int s, uint32_t r) {
     const long long Y = __float2ll_rd(__fmul_rn(x, pow2f(16 - s)));
@@ -471,73 +419,156 @@ __device__ __forceinline__ int round_sr_wide(float x, int s, uint32_t r) {
     return (int)max(-32767ll, min(32767ll, q));
 }
 
-// Wide weight storage (Sec. 4.2): w [d0][d1] lives as int16 mantissas (row-major, pitch d1) with one
-// exponent per t x t tile in grid [tiles along d0][tiles along d1]. One CTA per tile, 256 threads.
-//   MODE 0  quantise FP32 weights src [d0][d1] (pitch ld) to wide storage
-//   MODE 1  update: w = fl32(wide * 2^s + src) with src the FP32 update, re-quantised in place
+// Weight matrices with one exponent per t x t tile (Sec. 4.2 "Tiling", t <= 128) and their wide storage
+// (Sec. 4.2 "Wide weight storage"): one CTA per tile of w [d0][d1], 256 threads.
+//   MODE 3  quantise FP32 weights src (pitch ld) straight to p.m bits (no wide copy)
+//   MODE 0  quantise FP32 weights src to wide storage: int16 mantissas `wide` (row-major, pitch d1) and
+//           one exponent per tile in grid [tiles along d0][tiles along d1]
+//   MODE 1  update: w = fl32(wide * 2^s + src) with src the FP32 update, re-quantised to 16 bits in place
 //   MODE 2  read wide storage only
-// and, in every mode, when view pointers are given: the two packed narrow views of the tile, whose
-// mantissas are the top narrow_m bits of the wide ones (an arithmetic shift) under the exponent
-// s + 16 - narrow_m.
-template <int MODE, int PLANES>
+// In every mode, when view pointers are given, the tile goes to the two packed views
+//   c1: rows = d0, contraction along d1 (the stored orientation);  c0: rows = d1, contraction along d0
+// with, for the wide modes, the top p.m bits of the 16-bit mantissas (an arithmetic shift) under the
+// exponent s + 16 - p.m.
+// FAST: t, d1 multiples of 8, pitches and bases 16-byte aligned: a thread handles eight consecutive
+// weights of a row at a time (two 128-bit loads, one Philox call, 128-bit store of the int16 mantissas).
+template <int MODE, int PLANES, bool FAST>
 __global__ void __launch_bounds__(256)
-wide_tiles(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, int t, int tp, QParams p, int narrow_m,
-           int16_t* __restrict__ wide, int8_t* __restrict__ grid, int64_t grid_ld, TileViews tv) {
+tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, int t, int tp, QParams p,
+            int16_t* __restrict__ wide, int8_t* __restrict__ grid, int64_t grid_ld, TileViews tv) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* tile = reinterpret_cast<float*>(smem_raw);                      // [t][t+1]
-    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * (t + 1));  // [tp][tp + 2] zero padded
+    const int fp = FAST ? t + 4 : t + 1;                                   // pitch of the FP32 tile
+    float* tile = reinterpret_cast<float*>(smem_raw);                      // [t][fp]
+    const int qp = tp + 2;
+    int16_t* qt = reinterpret_cast<int16_t*>(tile + (size_t)t * fp);       // [tp][tp + 2], zero padded
     __shared__ uint32_t s_am[8];
     __shared__ int s_exp;
 
-    const int tid = threadIdx.x;
-    const int64_t u = blockIdx.y, v = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, wrow = tid >> 5;
+    const int64_t u = blockIdx.y, v = blockIdx.x;       // tile row (along d0), tile column (along d1)
     const int64_t i0 = u * t, j0 = v * t;
     const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
-    const int lane = tid & 31, wrow = tid >> 5, qp = tp + 2;
-    for (int e = tid; e < tp * qp; e += 256) qt[e] = 0;
+    const int G = wj >> 3;                              // FAST: groups of eight per tile row
+    const int wbits = MODE == 3 ? p.m : 16, wqmax = MODE == 3 ? p.qmax : 32767;
+    for (int e = tid; e < tp * qp / 2; e += 256) reinterpret_cast<uint32_t*>(qt)[e] = 0;
     int s;
     if (MODE == 2) {
         __syncthreads();
         s = grid[u * grid_ld + v];
-        for (int ii = wrow; ii < hi; ii += 8)
-            for (int jj = lane; jj < wj; jj += 32) qt[ii * qp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
+        if (FAST) {
+            for (int item = tid; item < hi * G; item += 256) {
+                const int ii = item / G, gj = item - ii * G;
+                const uint4 q8 = *reinterpret_cast<const uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj);
+                uint32_t* dst = reinterpret_cast<uint32_t*>(qt + ii * qp + 8 * gj);
+                dst[0] = q8.x; dst[1] = q8.y; dst[2] = q8.z; dst[3] = q8.w;
+            }
+        } else {
+            for (int ii = wrow; ii < hi; ii += 8)
+                for (int jj = lane; jj < wj; jj += 32) qt[ii * qp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
+        }
     } else {
         const float old_scale = MODE == 1 ? pow2f(grid[u * grid_ld + v]) : 0.f;
         uint32_t am = 0;
-        for (int ii = wrow; ii < hi; ii += 8)
-            for (int jj = lane; jj < wj; jj += 32) {
-                float val = src[(i0 + ii) * ld + j0 + jj];
-                if (MODE == 1) val = __fadd_rn(__fmul_rn((float)wide[(i0 + ii) * d1 + j0 + jj], old_scale), val);
-                tile[ii * (t + 1) + jj] = val;
-                am = max(am, abs_bits(val));
+        if (FAST) {
+            for (int item = tid; item < hi * G; item += 256) {
+                const int ii = item / G, gj = item - ii * G;
+                const float4* sp = reinterpret_cast<const float4*>(src + (i0 + ii) * ld + j0 + 8 * gj);
+                float4 a = __ldcs(sp), b = __ldcs(sp + 1);
+                if (MODE == 1) {
+                    const uint4 q8 = *reinterpret_cast<const uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj);
+                    a.x = __fadd_rn(__fmul_rn((float)(int16_t)(q8.x & 0xFFFFu), old_scale), a.x);
+                    a.y = __fadd_rn(__fmul_rn((float)(int16_t)(q8.x >> 16), old_scale), a.y);
+                    a.z = __fadd_rn(__fmul_rn((float)(int16_t)(q8.y & 0xFFFFu), old_scale), a.z);
+                    a.w = __fadd_rn(__fmul_rn((float)(int16_t)(q8.y >> 16), old_scale), a.w);
+                    b.x = __fadd_rn(__fmul_rn((float)(int16_t)(q8.z & 0xFFFFu), old_scale), b.x);
+                    b.y = __fadd_rn(__fmul_rn((float)(int16_t)(q8.z >> 16), old_scale), b.y);
+                    b.z = __fadd_rn(__fmul_rn((float)(int16_t)(q8.w & 0xFFFFu), old_scale), b.z);
+                    b.w = __fadd_rn(__fmul_rn((float)(int16_t)(q8.w >> 16), old_scale), b.w);
+                }
+                float4* tp4 = reinterpret_cast<float4*>(tile + ii * fp + 8 * gj);
+                tp4[0] = a; tp4[1] = b;
+                const float e8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                am = max(am, amax8_bits(e8));
             }
+        } else {
+            for (int ii = wrow; ii < hi; ii += 8)
+                for (int jj = lane; jj < wj; jj += 32) {
+                    float val = src[(i0 + ii) * ld + j0 + jj];
+                    if (MODE == 1) val = __fadd_rn(__fmul_rn((float)wide[(i0 + ii) * d1 + j0 + jj], old_scale), val);
+                    tile[ii * fp + jj] = val;
+                    am = max(am, abs_bits(val));
+                }
+        }
         for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
         if (lane == 0) s_am[wrow] = am;
         __syncthreads();
         if (tid == 0) {
             uint32_t a = 0;
             for (int i = 0; i < 8; ++i) a = max(a, s_am[i]);
-            s_exp = block_exponent(a, 16, p.exp_mode);
-            grid[u * grid_ld + v] = (int8_t)s_exp;
+            s_exp = block_exponent(a, wbits, p.exp_mode);
+            if (grid) grid[u * grid_ld + v] = (int8_t)s_exp;
         }
         __syncthreads();
         s = s_exp;
-        for (int ii = wrow; ii < hi; ii += 8)
-            for (int jj = lane; jj < wj; jj += 32) {
-                const float val = tile[ii * (t + 1) + jj];
-                int q;
-                if (p.rounding == 0) q = round_rne(val, s, 32767);
-                else q = round_sr_wide(val, s, draw_of_element(p, (uint64_t)((i0 + ii) * d1 + j0 + jj)));
-                qt[ii * qp + jj] = (int16_t)q;
-                wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
+        if (FAST) {
+            const uint32_t qm = qmax_pair(wqmax), nqm = neg_qmax_pair(wqmax);
+            for (int item = tid; item < hi * G; item += 256) {
+                const int ii = item / G, gj = item - ii * G;
+                const float4* tp4 = reinterpret_cast<const float4*>(tile + ii * fp + 8 * gj);
+                const float4 a = tp4[0], b = tp4[1];
+                const float e8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                if (p.rounding == 1) w = draws_of_group(p, (uint64_t)((i0 + ii) * d1 + j0 + 8 * gj) >> 3);
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                uint32_t h[4];
+                if (MODE == 3) {
+                    // at most 12 bits: the packed halfword forms
+                    const float sc = pow2f(p.rounding == 1 ? 16 - s : -s);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        h[j] = p.rounding == 1 ? round_sr_pair(e8[2 * j], e8[2 * j + 1], sc, ww[j], qm, nqm)
+                                               : round_rne_pair(e8[2 * j], e8[2 * j + 1], sc, qm, nqm);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        int q0, q1;
+                        if (p.rounding == 0) {
+                            q0 = round_rne(e8[2 * j], s, 32767);
+                            q1 = round_rne(e8[2 * j + 1], s, 32767);
+                        } else {
+                            q0 = round_sr_wide(e8[2 * j], s, ww[j] & 0xFFFFu);
+                            q1 = round_sr_wide(e8[2 * j + 1], s, ww[j] >> 16);
+                        }
+                        h[j] = ((uint32_t)q0 & 0xFFFFu) | ((uint32_t)q1 << 16);
+                    }
+                }
+                uint32_t* dst = reinterpret_cast<uint32_t*>(qt + ii * qp + 8 * gj);
+                dst[0] = h[0]; dst[1] = h[1]; dst[2] = h[2]; dst[3] = h[3];
+                if (MODE != 3) *reinterpret_cast<uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj) = make_uint4(h[0], h[1], h[2], h[3]);
             }
+        } else {
+            for (int ii = wrow; ii < hi; ii += 8)
+                for (int jj = lane; jj < wj; jj += 32) {
+                    const float val = tile[ii * fp + jj];
+                    const uint64_t L = (uint64_t)((i0 + ii) * d1 + j0 + jj);
+                    int q;
+                    if (MODE == 3) q = quantize_one(val, s, p, L);
+                    else if (p.rounding == 0) q = round_rne(val, s, 32767);
+                    else q = round_sr_wide(val, s, draw_of_element(p, L));
+                    qt[ii * qp + jj] = (int16_t)q;
+                    if (MODE != 3) wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
+                }
+        }
     }
     if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
     __syncthreads();
-    const int sh = 16 - narrow_m;
-    for (int e = tid; e < hi * qp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
-    __syncthreads();
-    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, tv, tid);
+    if (MODE != 3) {
+        const int sh = 16 - p.m;
+        for (int e = tid; e < hi * qp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
+        __syncthreads();
+        s += sh;
+    }
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s, tv, tid);
 }
 
 // ------------------------------------------------------------------------------ generic two-pass path
@@ -1030,9 +1061,11 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
     return launch_status();
 }
 
-int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* f,
-                          int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
-                          int8_t* tile_exps, cudaStream_t st) {
+namespace {
+
+template <int MODE>
+int launch_tiles(const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f, int16_t* wide,
+                 int8_t* grid, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1, cudaStream_t st) {
     if (f->tile <= 0 || f->tile != f->block) return HBFP_ERR_INVALID_ARG;
     if (f->tile > 128) return HBFP_ERR_UNSUPPORTED;
     Layout L0, L1;
@@ -1047,52 +1080,40 @@ int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, co
     if (nu > 65535) return HBFP_ERR_UNSUPPORTED;
     if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
     if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
-    size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
-    dim3 grid((unsigned)nv, (unsigned)nu);
+    const TileViews tv{mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb, mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb};
+    const bool fast = (t % 8) == 0 && (d1 % 8) == 0 &&
+                      (MODE == 2 || ((ld % 4) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0)) &&
+                      (MODE == 3 || (reinterpret_cast<uintptr_t>(wide) & 15) == 0);
+    const size_t smem = (size_t)t * (t + 4) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
+    const dim3 grid_dim((unsigned)nv, (unsigned)nu);
+#define HBFP_TILE_LAUNCH(PLANES, FAST)                                                                                       \
+    do {                                                                                                                     \
+        HBFP_CUDA_OK(cudaFuncSetAttribute(tile_kernel<MODE, PLANES, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        tile_kernel<MODE, PLANES, FAST><<<grid_dim, 256, smem, st>>>(src, ld, d0, d1, t, tp, p, wide, grid, nv, tv);         \
+    } while (0)
     if (L0.planes == 1) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(quant_tiles<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_tiles<1><<<grid, 256, smem, st>>>(w, d0, d1, ld, t, tp, p, mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb,
-                                               mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb, tile_exps, nv);
+        if (fast) HBFP_TILE_LAUNCH(1, true); else HBFP_TILE_LAUNCH(1, false);
     } else {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(quant_tiles<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        quant_tiles<2><<<grid, 256, smem, st>>>(w, d0, d1, ld, t, tp, p, mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb,
-                                               mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb, tile_exps, nv);
+        if (fast) HBFP_TILE_LAUNCH(2, true); else HBFP_TILE_LAUNCH(2, false);
     }
+#undef HBFP_TILE_LAUNCH
     return launch_status();
+}
+
+}  // namespace
+
+int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* f,
+                          int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                          int8_t* tile_exps, cudaStream_t st) {
+    return launch_tiles<3>(w, ld, d0, d1, f, nullptr, tile_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
 }
 
 int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,
                 int16_t* wide, int8_t* wide_exps, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
                 cudaStream_t st) {
-    if (f->tile <= 0 || f->tile != f->block) return HBFP_ERR_INVALID_ARG;
-    if (f->tile > 128) return HBFP_ERR_UNSUPPORTED;
-    Layout L0, L1;
-    int rc = make_layout(d1, d0, f, &L0);     // view c0: rows = d1, k = d0
-    if (rc) return rc;
-    rc = make_layout(d0, d1, f, &L1);         // view c1: rows = d0, k = d1
-    if (rc) return rc;
-    if (d0 == 0 || d1 == 0) return HBFP_OK;
-    const QParams p = make_params(f);         // rounding, exponent rule and random stream (the wide width is 16)
-    const int t = f->tile, tp = (int)L0.bp;
-    const int64_t nu = L0.nkb, nv = L1.nkb;   // tiles along d0, along d1
-    if (nu > 65535) return HBFP_ERR_UNSUPPORTED;
-    if (exps_c0 && L0.rs != d1) HBFP_CUDA_OK(cudaMemsetAsync(exps_c0, 0, (size_t)L0.exp_bytes, st));
-    if (exps_c1 && L1.rs != d0) HBFP_CUDA_OK(cudaMemsetAsync(exps_c1, 0, (size_t)L1.exp_bytes, st));
-    const TileViews tv{mant_c0, L0.kst, L0.plane_stride, exps_c0, L0.rs, L0.nkb, mant_c1, L1.kst, L1.plane_stride, exps_c1, L1.rs, L1.nkb};
-    const size_t smem = (size_t)t * (t + 1) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
-    const dim3 grid((unsigned)nv, (unsigned)nu);
-#define HBFP_WIDE_LAUNCH(MODE, PLANES)                                                                                  \
-    do {                                                                                                                \
-        HBFP_CUDA_OK(cudaFuncSetAttribute(wide_tiles<MODE, PLANES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        wide_tiles<MODE, PLANES><<<grid, 256, smem, st>>>(src, ld, d0, d1, t, tp, p, f->mant_bits, wide, wide_exps, nv, tv);  \
-    } while (0)
-    if (L0.planes == 1) {
-        if (mode == 0) HBFP_WIDE_LAUNCH(0, 1); else if (mode == 1) HBFP_WIDE_LAUNCH(1, 1); else HBFP_WIDE_LAUNCH(2, 1);
-    } else {
-        if (mode == 0) HBFP_WIDE_LAUNCH(0, 2); else if (mode == 1) HBFP_WIDE_LAUNCH(1, 2); else HBFP_WIDE_LAUNCH(2, 2);
-    }
-#undef HBFP_WIDE_LAUNCH
-    return launch_status();
+    if (mode == 0) return launch_tiles<0>(src, ld, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
+    if (mode == 1) return launch_tiles<1>(src, ld, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
+    return launch_tiles<2>(nullptr, d1, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
 }
 
 int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st) {
