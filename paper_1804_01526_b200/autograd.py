@@ -1,0 +1,94 @@
+"""A dense layer whose three GEMMs run in block floating point (Sec. 4.1, Sec. 5.1).
+
+The paper simulates HBFP by redefining PyTorch's linear module with ``autograd.Function``: the
+forward product ``Y = X W``, the backward-data product ``dX = dY W^T`` and the backward-weight
+product ``dW = X^T dY`` take BFP operands, every other operation (bias, activations, loss, the
+optimiser's arithmetic) stays FP32. This module is that wrapper over the library's calls; it holds
+no arithmetic of its own:
+
+* the weights live in wide storage (16-bit mantissas per tile, ``hbfp_wide_quantize``); the two
+  packed narrow views the GEMMs read are the top ``mant_bits`` bits (Sec. 4.2);
+* forward and backward-data read those views (``hbfp_gemm_q``), so the backward pass converts no
+  weights; activations and gradients are converted by the GEMM call with 1-D blocks along the
+  contraction axis; backward-weight is ``hbfp_gemm`` with ``transA = 1``;
+* ``apply_update(delta)`` hands the optimiser's FP32 update to ``hbfp_wide_update`` and refreshes the
+  views in the same launch.
+
+Stochastic rounding draws are keyed by (seed + step, stream id, element index): a layer takes three
+consecutive stream ids (X, W, dY) from ``stream_id``.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as hb
+
+
+class _HbfpLinearFn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, weight, bias, layer):
+        ctx.layer = layer
+        ctx.save_for_backward(x)
+        batch = x.shape[0]
+        y = hb.gemm_q(batch, layer.fout, layer.fin, x.contiguous(), layer.views[0], fmtA=layer.fmt_act(0))
+        return y + bias if bias is not None else y
+
+    @staticmethod
+    def backward(ctx, dy):
+        layer = ctx.layer
+        (x,) = ctx.saved_tensors
+        dy = dy.contiguous()
+        batch = x.shape[0]
+        dx = dw = db = None
+        if ctx.needs_input_grad[0]:
+            dx = hb.gemm_q(batch, layer.fin, layer.fout, dy, layer.views[1], fmtA=layer.fmt_act(2))
+        if ctx.needs_input_grad[1]:
+            # contraction over the batch axis: 1-D blocks down the columns of X and dY
+            dw = hb.gemm(1, 0, x.contiguous(), dy, layer.fmt_act(0, batch_axis=True), layer.fmt_act(2, batch_axis=True))
+        if ctx.needs_input_grad[2]:
+            db = dy.sum(dim=0)
+        return dx, dw, db, None
+
+
+class HbfpLinear(torch.nn.Module):
+    """``y = x W + b`` with W ``[fin][fout]`` in wide storage; see the module docstring."""
+
+    def __init__(self, fin: int, fout: int, mant_bits: int = 8, tile: int = 24, rounding: int = 1, seed: int = 0,
+                 stream_id: int = 0, batch_block: int = 32, bias: bool = True, device="cuda"):
+        super().__init__()
+        self.fin, self.fout = fin, fout
+        self.mant_bits, self.tile, self.rounding, self.seed, self.stream_id = mant_bits, tile, rounding, seed, stream_id
+        self.batch_block = batch_block
+        self.steps = 0
+        w = torch.randn(fin, fout, device=device) * (2.0 / fin) ** 0.5
+        self.weight = torch.nn.Parameter(w)
+        self.bias = torch.nn.Parameter(torch.zeros(fout, device=device)) if bias else None
+        self.wide, self.views = hb.wide_quantize(self.weight.data, self.fmt_weight())
+        self._refresh_fp32_copy()
+
+    # ---- formats
+    def fmt_weight(self) -> hb.Format:
+        return hb.Format(mant_bits=self.mant_bits, block=self.tile, tile=self.tile, rounding=self.rounding,
+                         seed=self.seed + self.steps, stream_id=self.stream_id + 1)
+
+    def fmt_act(self, which: int, batch_axis: bool = False) -> hb.Format:
+        """Format of X (which = 0) or dY (which = 2); blocks of ``tile`` along a feature axis, of
+        ``batch_block`` along the batch axis (backward-weight)."""
+        return hb.Format(mant_bits=self.mant_bits, block=self.batch_block if batch_axis else self.tile,
+                         rounding=self.rounding, seed=self.seed + self.steps, stream_id=self.stream_id + which)
+
+    # ---- weights
+    def _refresh_fp32_copy(self) -> None:
+        """The FP32 tensor autograd sees is the value of the wide copy (plain torch bookkeeping)."""
+        t = self.tile
+        scale = torch.exp2(self.wide.exps.float()).repeat_interleave(t, 0).repeat_interleave(t, 1)
+        self.weight.data = self.wide.mant.float() * scale[: self.fin, : self.fout]
+
+    def apply_update(self, delta: torch.Tensor) -> None:
+        """``W <- Q16(float32(W + delta))`` in wide storage, views refreshed by the same launch."""
+        self.steps += 1
+        hb.wide_update(self.wide, delta.contiguous(), self.fmt_weight(), views=self.views)
+        self._refresh_fp32_copy()
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        return _HbfpLinearFn.apply(x, self.weight, self.bias, self)

@@ -355,9 +355,10 @@ struct TileViews {
 };
 
 // qt rows have a pitch of tp + 2 halfwords, so that the column reads of view c0 spread over the banks.
+// sh: the views take the mantissas shifted down by sh bits (arithmetic: the top bits of wide storage).
 template <int PLANES>
 __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int hi, int wj, int64_t i0, int64_t j0,
-                                                 int64_t u, int64_t v, int s, const TileViews& tv, int tid) {
+                                                 int64_t u, int64_t v, int s, int sh, const TileViews& tv, int tid) {
     const int qp = tp + 2;
     const int lg = 31 - __clz(tp >> 2), gmask = (tp >> 2) - 1;       // tp is 32, 64 or 128
     int8_t* const mant_c0 = tv.mant_c0; int8_t* const mant_c1 = tv.mant_c1;
@@ -370,7 +371,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[ii * qp + g + j];
+            const int q = qt[ii * qp + g + j] >> sh;
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -385,7 +386,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[(g + j) * qp + jj];
+            const int q = qt[(g + j) * qp + jj] >> sh;
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -562,13 +563,8 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
     }
     if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
     __syncthreads();
-    if (MODE != 3) {
-        const int sh = 16 - p.m;
-        for (int e = tid; e < hi * qp; e += 256) qt[e] = (int16_t)(qt[e] >> sh);       // top bits: arithmetic shift
-        __syncthreads();
-        s += sh;
-    }
-    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s, tv, tid);
+    const int sh = MODE == 3 ? 0 : 16 - p.m;                  // wide modes: the views hold the top p.m bits
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, tv, tid);
 }
 
 // ------------------------------------------------------------------------------ generic two-pass path
