@@ -99,8 +99,8 @@ def test_small_classifier_trains_like_fp32(env):
         with torch.no_grad():
             for p in (w1, b1, w2, b2):
                 p -= lr * p.grad
-        hist_h.append(float(loss_h))
-        hist_f.append(float(loss_f))
+        hist_h.append(float(loss_h.detach()))
+        hist_f.append(float(loss_f.detach()))
     assert hb.device_status() == 0
     first, last_h, last_f = np.mean(hist_h[:5]), np.mean(hist_h[-10:]), np.mean(hist_f[-10:])
     assert last_h < 0.5 * first, (first, last_h)                     # it learns
