@@ -228,3 +228,18 @@ def test_mlp_step_captured_in_a_cuda_graph_replays_on_new_data(hb):
         ref = oracle.hbfp_gemm(sp.transA, sp.transB, t2[sp.a_key], t2[sp.b_key], ofmt(sp.fmt_a), ofmt(sp.fmt_b))
         err = np.abs(C.cpu().numpy().astype(np.float64) - ref["c_ref"].astype(np.float64))
         assert (err <= TOL * ref["a_mag"]).all(), sp.name
+
+
+@pytest.mark.parametrize("m,M,N,K", [(8, 128, 1024, 784), (8, 384, 512, 1024), (4, 200, 136, 1000), (12, 256, 256, 320)])
+def test_one_exponent_per_row_no_blocks_no_tiles(hb, m, M, N, K):
+    # "HBFP without tiles": block = 0, the whole contraction axis shares one exponent (one K-block per GEMM)
+    A = wl.draw("half_normal", (M, K), seed=51)
+    B = wl.draw("he_weight", (K, N), seed=52, fan_in=K)
+    fd = dict(mant_bits=m, block=0, rounding=0, seed=0)
+    ref = oracle.hbfp_gemm(0, 0, A, B, ofmt(fd), ofmt(fd))
+    for flags in (hb.GEMM_FORCE_SIMT, hb.GEMM_AUTO):
+        C = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), flags=flags).cpu().numpy()
+        assert hb.device_status() == 0
+        err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
+        assert (err <= TOL * ref["a_mag"]).all()
+        assert np.array_equal(C, ref["c_seq"])          # a single block: one product, one rounding
