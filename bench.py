@@ -337,6 +337,28 @@ def gpu_arm(args):
             quant[f"m{m}_b{b}_{'sr' if r else 'rne'}"] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9}
             del p
 
+    # ---- wide weight storage: in-place FP32 update of an 8192 x 8192 weight matrix (tile 64), with its
+    # narrow views; algorithmic bytes per weight: 2 + 4 read, 2 + 2 written
+    wide = {}
+    if n * n * 4 >= 2 ** 30 or args.quantize_line:
+        nw = 8192
+        fw = hb.Format(8, 64, 64, 0, 0, 3, 0)
+        Wm = A[:nw, :nw].contiguous()
+        dW = (B[:nw, :nw] * 1e-3).contiguous()
+        wst, views = hb.wide_quantize(Wm, fw)
+        for _ in range(3):
+            hb.wide_update(wst, dW, fw, views=views)
+        torch.cuda.synchronize()
+        s4, e4 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s4.record()
+        for _ in range(10):
+            hb.wide_update(wst, dW, fw, views=views)
+        e4.record()
+        torch.cuda.synchronize()
+        ms = s4.elapsed_time(e4) / 10
+        wide["update_8192x8192_m8_t64_rne"] = {"ms": ms, "gbs": nw * nw * 10 / (ms * 1e-3) / 1e9}
+        del Wm, dW, wst, views
+
     peaks, peaks_kind = load_peaks()
     int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
@@ -378,7 +400,7 @@ def gpu_arm(args):
                            "per panel) on 3 streams: copy-in, compute and copy-out overlap") if panels > 1
                           else "one hbfp_gemm call between the copies"},
            "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
-           "breakdown": breakdown, "quantize_standalone": quant}
+           "breakdown": breakdown, "quantize_standalone": quant, "wide_storage": wide}
     print(json.dumps(out), flush=True)
     replicas.shutdown(rep)
     return 0
