@@ -125,13 +125,14 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
     if (rc) return rc;
     rc = resolve_operand(b, false, N, K, g.lb, ws, g.off_bm, g.off_be, &pb, st);
     if (rc) return rc;
+    const bool quad_rows = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc % 4) == 0;
     const bool want_tensor = flags != HBFP_GEMM_FORCE_SIMT && g.tp.supported &&
-                             (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc % 4) == 0;
+                             (reinterpret_cast<uintptr_t>(C) & 3) == 0;
     if (want_tensor) {
         // With a short contraction (under 1 KiB of mantissas per row) a tile is bound by the write of
         // its C part, and the single-SM kernel, whose warps own wider row segments, is ~10 % faster.
         const bool long_k = g.la.nkb * g.la.bp >= 1024;
-        const bool pair_ok = !P && flags != HBFP_GEMM_FORCE_TENSOR_1SM && pair_gemm_eligible(M, N, pa, pb, g.tp) &&
+        const bool pair_ok = !P && quad_rows && flags != HBFP_GEMM_FORCE_TENSOR_1SM && pair_gemm_eligible(M, N, pa, pb, g.tp) &&
                              (long_k || flags == HBFP_GEMM_FORCE_TENSOR_2SM);
         if (pair_ok) return launch_gemm_tensor_pair(M, N, pa, pb, C, ldc, g.tp, ws ? ws + g.off_partial : nullptr, st);
         if (flags == HBFP_GEMM_FORCE_TENSOR_2SM) return HBFP_ERR_UNSUPPORTED;

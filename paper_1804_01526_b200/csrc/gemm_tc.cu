@@ -588,6 +588,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 float* rowp = dst + gi * ldd + n0 + col0;
                 // full 32-byte sectors per lane where the row pitch allows it (each lane owns a row)
                 const bool wide = (ldd & 7) == 0 && (reinterpret_cast<uintptr_t>(dst) & 31) == 0;
+                // 16-byte stores need a pitch of whole quads; any other pitch (an output ten columns wide) goes element by element
+                const bool quad = (ldd & 3) == 0 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0;
 #pragma unroll
                 for (int c = 0; c < COLS_PER_WARP; c += 4) {
                     const int64_t gj = n0 + col0 + c;
@@ -595,7 +597,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         st_global_256(rowp + c, acc2[c / 2], acc2[c / 2 + 1], acc2[c / 2 + 2], acc2[c / 2 + 3]);
                     } else if (wide && (c & 7) == 4 && gj + 3 < p.N) {
                         // second half of a sector already written above
-                    } else if (gj + 3 < p.N) {
+                    } else if (quad && gj + 3 < p.N) {
                         *reinterpret_cast<ulonglong2*>(rowp + c) = make_ulonglong2(acc2[c / 2], acc2[c / 2 + 1]);
                     } else {
                         float e4[4];

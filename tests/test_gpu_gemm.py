@@ -243,3 +243,23 @@ def test_one_exponent_per_row_no_blocks_no_tiles(hb, m, M, N, K):
         err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
         assert (err <= TOL * ref["a_mag"]).all()
         assert np.array_equal(C, ref["c_seq"])          # a single block: one product, one rounding
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 10, 1024), (1024, 10, 128), (200, 137, 256), (300, 66, 96)])
+def test_tensor_core_kernel_writes_outputs_of_any_width(hb, M, N, K):
+    # an output whose row pitch is not a multiple of four floats (the MLP's ten-class layer) cannot take
+    # 16-byte stores; the tensor-core kernel then stores element by element
+    A = wl.draw("half_normal", (M, K), seed=61)
+    B = wl.draw("he_weight", (K, N), seed=62, fan_in=K)
+    fd = dict(mant_bits=8, block=32, rounding=0, seed=0)
+    ref = oracle.hbfp_gemm(0, 0, A, B, ofmt(fd), ofmt(fd))
+    C = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), flags=hb.GEMM_FORCE_TENSOR).cpu().numpy()
+    assert hb.device_status() == 0
+    err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+    # a view into a wider buffer with an odd pitch and an odd column offset
+    import torch
+    buf = torch.full((M, N + 7), -1.0, device="cuda")
+    hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), out=buf[:, 3:3 + N], flags=hb.GEMM_FORCE_TENSOR)
+    out = buf.cpu().numpy()
+    assert np.array_equal(out[:, 3:3 + N], C) and (out[:, :3] == -1).all() and (out[:, 3 + N:] == -1).all()
