@@ -70,6 +70,14 @@ __device__ __forceinline__ uint32_t round_sr_pair(float x0, float x1, float scal
     return __vmaxs2(__vmins2(h, qmax2), nqmax2);
 }
 
+// The same for two values whose draws r0, r1 (16 bits each) come from different places.
+__device__ __forceinline__ uint32_t round_sr_pair2(float x0, float x1, float scale, uint32_t r0, uint32_t r1, uint32_t qmax2, uint32_t nqmax2) {
+    const int t0 = __float2int_rd(__fmul_rn(x0, scale)) + (int)r0;
+    const int t1 = __float2int_rd(__fmul_rn(x1, scale)) + (int)r1;
+    const uint32_t h = __byte_perm((uint32_t)t0, (uint32_t)t1, 0x7632);
+    return __vmaxs2(__vmins2(h, qmax2), nqmax2);
+}
+
 // Nearest-even rounding of two values, clamped as a signed halfword pair (m <= 12: the unclamped
 // value, at most 2^(m-1) in magnitude, fits a halfword).
 __device__ __forceinline__ uint32_t round_rne_pair(float x0, float x1, float scale, uint32_t qmax2, uint32_t nqmax2) {
@@ -814,16 +822,18 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
     for (int t = first; t < total_tiles; t += step) {
         const int nt = t % tiles_n, kt = t / tiles_n;
         const int64_t col = (int64_t)nt * QC_COLS + n;
-        // (uniform verdict: a wait that gave up in some threads only would split the CTA barriers below)
-        if (!__syncthreads_and(mbar_wait(full_bar + 8 * s, ph, abort_flag, status, 601))) break;
-        const float* tile = in + (size_t)s * (QC_IN_BYTES / 4);
         if (SR) {
-            // one Philox call per eight consecutive source elements of a row (R % 8 == 0 here)
+            // one Philox call per eight consecutive source elements of a row (R % 8 == 0 here); the draws
+            // do not depend on the data, so they are made while the tile may still be in flight (the
+            // previous tile's readers of the table are past the barrier that precedes its store)
             for (int i = tid; i < QC_ROWS * (QC_COLS / 8); i += QC_THREADS) {
                 const uint64_t L = (uint64_t)((int64_t)kt * QC_ROWS + (i >> 3)) * (uint64_t)R + (uint64_t)(nt * QC_COLS + (i & 7) * 8);
                 rnd[i] = draws_of_group(p, L >> 3);
             }
         }
+        // (uniform verdict: a wait that gave up in some threads only would split the CTA barriers below)
+        if (!__syncthreads_and(mbar_wait(full_bar + 8 * s, ph, abort_flag, status, 601))) break;
+        const float* tile = in + (size_t)s * (QC_IN_BYTES / 4);
         float v[32];
         uint32_t am = 0;
 #pragma unroll
@@ -862,8 +872,7 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
                 const int j = 4 * w + 2 * k;
                 if (SR) {
                     // the draws of two vertical neighbours belong to different rows: two table entries
-                    const uint32_t r01 = (uint32_t)rnd16[(q * 32 + j) * QC_COLS + n] | ((uint32_t)rnd16[(q * 32 + j + 1) * QC_COLS + n] << 16);
-                    h[k] = round_sr_pair(v[j], v[j + 1], sc, r01, qm, nqm);
+                    h[k] = round_sr_pair2(v[j], v[j + 1], sc, rnd16[(q * 32 + j) * QC_COLS + n], rnd16[(q * 32 + j + 1) * QC_COLS + n], qm, nqm);
                 } else {
                     h[k] = round_rne_pair(v[j], v[j + 1], sc, qm, nqm);
                 }
