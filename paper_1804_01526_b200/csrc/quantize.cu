@@ -207,6 +207,13 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
                 v[i][1] = v[i][0];
             }
         }
+        // the draws do not depend on the data: they are made while the loads are in flight
+        uint4 wd[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            wd[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (SR) wd[i] = draws_of_group(p, (uint64_t)((r0 + warp * 4 + i) * K + col) >> 3);   // a multiple of 8 on this path
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int64_t r = r0 + warp * 4 + i;
@@ -216,8 +223,7 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
 #pragma unroll
             for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
             const int s = block_exponent(am, p.m, p.exp_mode);
-            uint4 w = make_uint4(0u, 0u, 0u, 0u);
-            if (SR) w = draws_of_group(p, (uint64_t)(r * K + col) >> 3);     // r * K + col is a multiple of 8 on this path
+            const uint4 w = wd[i];
             uint2 hi, lo;
             quantize_pack8<SR, PLANES>(e8, s, p, w, hi, lo);
             if (r < rows && col < kst) {
@@ -726,6 +732,13 @@ quant_row_flat(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
         cg += r256;
         if (cg >= gpr) { cg -= gpr; ++row; }
     }
+    // the draws do not depend on the data: they are made while the loads are in flight
+    uint4 wd[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        wd[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (SR) wd[j] = draws_of_group(p, ((uint64_t)rw[j] * (uint64_t)K + cc[j]) >> 3);     // a multiple of 8 on this path
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const bool live = g0 + j * 256u < total_groups;      // uniform over the LPB lanes of a block
@@ -734,8 +747,7 @@ quant_row_flat(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
 #pragma unroll
         for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
         const int s = block_exponent(am, p.m, p.exp_mode);
-        uint4 w = make_uint4(0u, 0u, 0u, 0u);
-        if (SR) w = draws_of_group(p, ((uint64_t)rw[j] * (uint64_t)K + cc[j]) >> 3);     // a multiple of 8 on this path
+        const uint4 w = wd[j];
         uint2 hi, lo;
         quantize_pack8<SR, PLANES>(e8, s, p, w, hi, lo);
         if (live) {
