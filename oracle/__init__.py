@@ -243,3 +243,25 @@ def wide_update(q16: np.ndarray, s16: np.ndarray, delta: np.ndarray, fmt: Format
     if rc:
         raise ValueError(f"oracle_wide_update failed: {rc}")
     return q, s
+
+
+def im2col(x: np.ndarray, kh: int, kw: int, pad: int) -> np.ndarray:
+    """Convolution as a matrix product (the paper runs convolutions through the same BFP dot products,
+    Sec. 5.1): ``x [n][h][w][c]`` -> ``[n*ho*wo][kh*kw*c]`` with ``ho = h + 2 pad - kh + 1`` (stride 1),
+    row = output pixel, columns ordered tap-major ``(i, j, channel)``, zeros outside the image. With a
+    block of ``c`` along the columns every block is the channel vector of one input pixel."""
+    assert x.ndim == 4
+    n, h, w, c = x.shape
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    out = np.zeros((n, ho, wo, kh, kw, c), dtype=x.dtype)
+    for i in range(kh):
+        for j in range(kw):
+            for oy in range(ho):
+                iy = oy + i - pad
+                if iy < 0 or iy >= h:
+                    continue
+                for ox in range(wo):
+                    ix = ox + j - pad
+                    if 0 <= ix < w:
+                        out[:, oy, ox, i, j, :] = x[:, iy, ix, :]
+    return out.reshape(n * ho * wo, kh * kw * c)

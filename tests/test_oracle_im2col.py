@@ -1,0 +1,53 @@
+"""Pins of the oracle's convolution-as-matrix-product gather: against a direct evaluation of the
+convolution sum, and the block structure the packed gather on the GPU relies on."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import Format
+
+
+@pytest.mark.parametrize("n,h,w,c,kh,kw,pad,f", [(2, 5, 6, 3, 3, 3, 1, 4), (1, 4, 4, 2, 1, 1, 0, 3), (2, 6, 5, 4, 3, 3, 0, 2),
+                                               (1, 5, 5, 2, 5, 3, 2, 3)])
+def test_matrix_product_of_the_gather_is_the_convolution_sum(n, h, w, c, kh, kw, pad, f):
+    rng = np.random.default_rng(n * 100 + h)
+    x = rng.integers(-4, 5, size=(n, h, w, c)).astype(np.float64)
+    wt = rng.integers(-3, 4, size=(kh, kw, c, f)).astype(np.float64)
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    direct = np.zeros((n, ho, wo, f))
+    for b in range(n):
+        for oy in range(ho):
+            for ox in range(wo):
+                for i in range(kh):
+                    for j in range(kw):
+                        iy, ix = oy + i - pad, ox + j - pad
+                        if 0 <= iy < h and 0 <= ix < w:
+                            direct[b, oy, ox] += x[b, iy, ix] @ wt[i, j]
+    cols = oracle.im2col(x, kh, kw, pad)
+    assert cols.shape == (n * ho * wo, kh * kw * c)
+    assert np.array_equal((cols @ wt.reshape(kh * kw * c, f)).reshape(n, ho, wo, f), direct)
+
+
+def test_blocks_of_the_gathered_matrix_are_blocks_of_the_pixels():
+    # with a block of c along the columns, quantising the gathered matrix gives, block by block, the
+    # quantised channel vector of the pixel the block was gathered from (and an all-zero block outside)
+    rng = np.random.default_rng(3)
+    n, h, w, c = 2, 6, 7, 16
+    x = (rng.standard_normal((n, h, w, c)) * np.exp(rng.standard_normal((n, h, w, 1)) * 2)).astype(np.float32)
+    f = Format(mant_bits=8, block=c)
+    qp, sp = oracle.quantize(x.reshape(n * h * w, c), 1, f)
+    cols = oracle.im2col(x, 3, 3, 1)
+    qc, sc = oracle.quantize(cols, 1, f)
+    qc = qc.reshape(n, h, w, 3, 3, c)
+    sc = sc.reshape(n, h, w, 3, 3)
+    qp = qp.reshape(n, h, w, c)
+    sp = sp.reshape(n, h, w)
+    for i in range(3):
+        for j in range(3):
+            for oy in range(h):
+                for ox in range(w):
+                    iy, ix = oy + i - 1, ox + j - 1
+                    if 0 <= iy < h and 0 <= ix < w:
+                        assert np.array_equal(qc[:, oy, ox, i, j], qp[:, iy, ix]) and np.array_equal(sc[:, oy, ox, i, j], sp[:, iy, ix])
+                    else:
+                        assert not qc[:, oy, ox, i, j].any() and (sc[:, oy, ox, i, j] == -63).all()
