@@ -161,6 +161,23 @@ HBFP_API int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int6
                               const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1,
                               int8_t* exps_c1, void* stream);
 
+/* Convolution operand without the FP32 im2col matrix (the paper runs convolutions through the same
+ * BFP dot products, Sec. 5.1). x is an activation tensor [n][h][w][c] (channels last) that was
+ * converted once with hbfp_quantize(x as [n*h*w][c], contract_axis 1, block = c): one block, hence
+ * one exponent, per pixel. The convolution with a kh x kw filter, stride 1 and `pad` zeros around the
+ * image is the GEMM [n*ho*wo][kh*kw*c] x [kh*kw*c][filters], ho = h + 2 pad - kh + 1, columns ordered
+ * (filter row, filter column, channel); each block of c columns of a row is the channel vector of one
+ * input pixel, so the packed A operand is a gather of the packed pixels: this call writes it (rows =
+ * n*ho*wo, k = kh*kw*c, format fmt with fmt->block == c, fmt->tile == 0, c <= 128; positions outside
+ * the image hold zero mantissas and the exponent -63 of an all-zero block). It is bit-identical to
+ * hbfp_quantize of the FP32 im2col matrix under nearest-even rounding (under stochastic rounding the
+ * draws were keyed by the element's index in x, not in the im2col matrix). mant_x / exps_x: the
+ * packed pixels; mant_out / exps_out: buffers of the sizes hbfp_packed_sizes(n*ho*wo, kh*kw*c)
+ * returns, fully overwritten. All device pointers; asynchronous on `stream`. */
+HBFP_API int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_t n, int64_t h, int64_t w,
+                                int64_t c, int kh, int kw, int pad, const hbfp_format* fmt, void* mant_out,
+                                int8_t* exps_out, void* stream);
+
 /* Packed -> canonical arrays for inspection: q [rows][k] int16 mantissas and s [rows][nkb]
  * int8 exponents (either may be NULL). */
 HBFP_API int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k,

@@ -28,6 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
+    "hbfp_im2col_packed",
 ]
 
 
@@ -92,6 +93,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_wide_quantize.argtypes = [p, i64, i64, i64, p, p, p, p, p, p, p, p]
         L.hbfp_wide_update.argtypes = [p, p, p, i64, i64, i64, p, p, p, p, p, p]
         L.hbfp_wide_narrow.argtypes = [p, p, i64, i64, p, p, p, p, p, p]
+        L.hbfp_im2col_packed.argtypes = [p, p, i64, i64, i64, i64, i32, i32, i32, p, p, p, p]
         L.hbfp_unpack.argtypes = [p, p, i64, i64, p, p, p, p]
         L.hbfp_dequantize.argtypes = [p, p, i64, i64, p, p, i64, p]
         L.hbfp_gemm_workspace.argtypes = [i32, i32, i64, i64, i64, p, p, p]
@@ -258,6 +260,19 @@ def wide_narrow(wide: Wide, fmt: Format, views: Optional[Tuple[Packed, Packed]] 
     _check(lib().hbfp_wide_narrow(_dptr(wide.mant), _dptr(wide.exps), d0, d1, ctypes.byref(f), *_view_args(views),
                                   _stream()), "hbfp_wide_narrow")
     return views
+
+
+def im2col_packed(px: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, pad: int,
+                  out: Optional[Packed] = None) -> Packed:
+    """hbfp_im2col_packed: the packed convolution operand ``[n*ho*wo][kh*kw*c]`` gathered from the
+    packed pixels ``px`` (``quantize(x.view(n*h*w, c), 1, fmt)`` with ``fmt.block == c``)."""
+    ho, wo = h + 2 * pad - kh + 1, w + 2 * pad - kw + 1
+    if out is None:
+        out = alloc_packed(n * ho * wo, kh * kw * c, px.fmt, px.mant.device)
+    f = px.fmt.c()
+    _check(lib().hbfp_im2col_packed(_dptr(px.mant), _dptr(px.exps), n, h, w, c, kh, kw, pad, ctypes.byref(f),
+                                    _dptr(out.mant), _dptr(out.exps), _stream()), "hbfp_im2col_packed")
+    return out
 
 
 def unpack(p: Packed) -> Tuple[torch.Tensor, torch.Tensor]:

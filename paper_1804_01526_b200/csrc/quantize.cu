@@ -666,6 +666,38 @@ __global__ void mant_generic(const float* __restrict__ x, int64_t d1, int64_t ro
     if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant + plane_stride + r * kst + o) = l;
 }
 
+// ------------------------------------------------------------------------------ packed im2col gather
+
+// Convolution operand without the FP32 im2col matrix: with a block of c channels along the contraction
+// (taps ordered (i, j, channel)) every block of an im2col row is the quantised channel vector of one input
+// pixel, so the packed operand [n ho wo][kh kw c] is a gather of the packed per-pixel operand [n h w][c]:
+// bp bytes of mantissas and one exponent per tap, zeros (exponent -63, as an all-zero block has) outside the
+// image. One thread per 16 bytes of an output row (row tails beyond the last tap are zeroed too).
+__global__ void im2col_gather(const int8_t* __restrict__ xm, const int8_t* __restrict__ xe, int64_t kst_x, int64_t ps_x,
+                              int h, int w, int ho, int wo, int kh, int kw, int pad, int bp, int planes,
+                              int64_t rows_out, int64_t kst_out, int64_t ps_out, int64_t rs_out,
+                              int8_t* __restrict__ om, int8_t* __restrict__ oe) {
+    const int64_t chunks = kst_out >> 4;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows_out * chunks) return;
+    const int64_t r = i / chunks;
+    const int o = (int)(i - r * chunks) << 4;              // byte offset in the output row
+    const int tap = o / bp, within = o - tap * bp;
+    const int ox = (int)(r % wo), oy = (int)((r / wo) % ho);
+    const int64_t img = r / ((int64_t)wo * ho);
+    int64_t src = -1;
+    if (tap < kh * kw) {
+        const int iy = oy + tap / kw - pad, ix = ox + tap % kw - pad;
+        if (iy >= 0 && iy < h && ix >= 0 && ix < w) src = (img * h + iy) * w + ix;
+    }
+    for (int pl = 0; pl < planes; ++pl) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (src >= 0) v = *reinterpret_cast<const uint4*>(xm + pl * ps_x + src * kst_x + within);
+        *reinterpret_cast<uint4*>(om + pl * ps_out + r * kst_out + o) = v;
+    }
+    if (within == 0 && tap < kh * kw) oe[(int64_t)tap * rs_out + r] = src >= 0 ? xe[src] : (int8_t)-63;
+}
+
 // ------------------------------------------------------------------------------ inverse helpers
 
 __global__ void unpack_kernel(const int8_t* __restrict__ mant, const int8_t* __restrict__ exps, int64_t rows,
@@ -1131,6 +1163,26 @@ int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, 
     if (mode == 0) return launch_tiles<0>(src, ld, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
     if (mode == 1) return launch_tiles<1>(src, ld, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
     return launch_tiles<2>(nullptr, d1, d0, d1, f, wide, wide_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
+}
+
+int launch_im2col_packed(const int8_t* xm, const int8_t* xe, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
+                         int pad, const hbfp_format* f, int8_t* om, int8_t* oe, cudaStream_t st) {
+    if (f->tile != 0 || f->block != c) return HBFP_ERR_INVALID_ARG;      // one block per pixel
+    if (c > 128) return HBFP_ERR_UNSUPPORTED;
+    const int64_t ho = h + 2 * pad - kh + 1, wo = w + 2 * pad - kw + 1;
+    if (ho <= 0 || wo <= 0) return HBFP_ERR_INVALID_ARG;
+    Layout Lx, Lo;
+    int rc = make_layout(n * h * w, c, f, &Lx);
+    if (rc) return rc;
+    rc = make_layout(n * ho * wo, (int64_t)kh * kw * c, f, &Lo);
+    if (rc) return rc;
+    if (h > (1 << 20) || w > (1 << 20) || Lo.kst > (1ll << 30)) return HBFP_ERR_UNSUPPORTED;
+    if (n == 0) return HBFP_OK;
+    HBFP_CUDA_OK(cudaMemsetAsync(oe, 0, (size_t)Lo.exp_bytes, st));
+    const int64_t items = Lo.rows * (Lo.kst >> 4);
+    im2col_gather<<<blocks_for(items, 256), 256, 0, st>>>(xm, xe, Lx.kst, Lx.plane_stride, (int)h, (int)w, (int)ho, (int)wo, kh, kw,
+                                                         pad, (int)Lo.bp, (int)Lo.planes, Lo.rows, Lo.kst, Lo.plane_stride, Lo.rs, om, oe);
+    return launch_status();
 }
 
 int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st) {

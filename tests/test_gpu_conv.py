@@ -1,0 +1,78 @@
+"""GPU parity of the packed im2col gather through the C ABI: the convolution operand built from
+activations that were converted once per pixel is bit-identical to converting the FP32 im2col matrix,
+and the convolution GEMM on it equals the GEMM on the FP32 im2col matrix."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1804_01526_b200 import workloads as wl
+from tests.helpers import decode_packed, gfmt, ofmt, to_dev
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-6
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_1804_01526_b200 import binding
+    binding.lib()
+    return binding
+
+
+CASES = [
+    # n, h, w, c, kh, kw, pad, mantissa bits
+    (2, 32, 32, 64, 3, 3, 1, 8),       # the 64-channel 3x3 convolution of the ResNet configuration, two images
+    (1, 16, 16, 128, 3, 3, 1, 8),
+    (3, 9, 7, 24, 3, 3, 1, 8),         # channel count below the padded block width
+    (2, 8, 8, 64, 3, 3, 1, 12),        # two mantissa planes
+    (2, 10, 11, 32, 5, 3, 0, 8),       # no padding, rectangular filter: the output is smaller than the input
+    (1, 6, 6, 16, 1, 1, 0, 6),
+]
+
+
+@pytest.mark.parametrize("n,h,w,c,kh,kw,pad,m", CASES)
+def test_gathered_operand_equals_quantised_im2col_matrix(hb, n, h, w, c, kh, kw, pad, m):
+    x = wl.draw("half_normal", (n * h * w, c), seed=71).reshape(n, h, w, c)
+    x *= np.exp(wl.draw("normal", (n * h * w, 1), seed=72)).reshape(n, h, w, 1).astype(np.float32)
+    fd = dict(mant_bits=m, block=c, rounding=0, seed=0)
+    px = hb.quantize(to_dev(x.reshape(n * h * w, c)), 1, gfmt(fd))
+    pa = hb.im2col_packed(px, n, h, w, c, kh, kw, pad)
+    assert hb.device_status() == 0
+    cols = oracle.im2col(x, kh, kw, pad)
+    q_ref, s_ref = oracle.quantize(cols, 1, ofmt(fd))
+    q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
+    assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
+    # byte for byte what converting the FP32 im2col matrix gives
+    pb = hb.quantize(to_dev(cols), 1, gfmt(fd))
+    lay = hb.packed_layout(pa.rows, pa.k, pa.fmt)
+    for pl in range(lay["planes"]):
+        lo, hi = pl * lay["plane_stride"], pl * lay["plane_stride"] + pa.rows * lay["kst"]
+        assert np.array_equal(pa.mant[lo:hi].cpu().numpy(), pb.mant[lo:hi].cpu().numpy())
+    ne = lay["nkb"] * lay["rs"]
+    assert np.array_equal(pa.exps[:ne].cpu().numpy(), pb.exps[:ne].cpu().numpy())
+
+
+def test_convolution_forward_gemm_on_the_gathered_operand(hb):
+    n, h, w, c, f = 4, 32, 32, 64, 64
+    x = wl.draw("half_normal", (n * h * w, c), seed=73).reshape(n, h, w, c)
+    wt = wl.draw("he_weight", (9 * c, f), seed=74, fan_in=9 * c)
+    fd = dict(mant_bits=8, block=c, rounding=0, seed=0)
+    px = hb.quantize(to_dev(x.reshape(n * h * w, c)), 1, gfmt(fd))
+    pa = hb.im2col_packed(px, n, h, w, c, 3, 3, 1)
+    Y = hb.gemm_q(n * h * w, f, 9 * c, pa, to_dev(wt), fmtB=gfmt(fd)).cpu().numpy()
+    assert hb.device_status() == 0
+    cols = oracle.im2col(x, 3, 3, 1)
+    ref = oracle.hbfp_gemm(0, 0, cols, wt, ofmt(fd), ofmt(fd))
+    err = np.abs(Y.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+    Y2 = hb.gemm(0, 0, to_dev(cols), to_dev(wt), gfmt(fd), gfmt(fd)).cpu().numpy()
+    assert np.array_equal(Y, Y2)
+
+
+def test_gather_argument_errors(hb):
+    x = to_dev(wl.draw("normal", (64, 32), seed=1))
+    px = hb.quantize(x, 1, hb.Format(mant_bits=8, block=16))
+    with pytest.raises(hb.HbfpError) as e:               # the block must be the channel count
+        hb.im2col_packed(px, 1, 8, 8, 32, 3, 3, 1)
+    assert e.value.code == hb.ERR_INVALID_ARG
