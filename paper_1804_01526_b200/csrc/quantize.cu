@@ -672,30 +672,74 @@ __global__ void mant_generic(const float* __restrict__ x, int64_t d1, int64_t ro
 // (taps ordered (i, j, channel)) every block of an im2col row is the quantised channel vector of one input
 // pixel, so the packed operand [n ho wo][kh kw c] is a gather of the packed per-pixel operand [n h w][c]:
 // bp bytes of mantissas and one exponent per tap, zeros (exponent -63, as an all-zero block has) outside the
-// image. One thread per 16 bytes of an output row (row tails beyond the last tap are zeroed too).
-__global__ void im2col_gather(const int8_t* __restrict__ xm, const int8_t* __restrict__ xe, int64_t kst_x, int64_t ps_x,
-                              int h, int w, int ho, int wo, int kh, int kw, int pad, int bp, int planes,
-                              int64_t rows_out, int64_t kst_out, int64_t ps_out, int64_t rs_out,
-                              int8_t* __restrict__ om, int8_t* __restrict__ oe) {
-    const int64_t chunks = kst_out >> 4;
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= rows_out * chunks) return;
-    const int64_t r = i / chunks;
-    const int o = (int)(i - r * chunks) << 4;              // byte offset in the output row
-    const int tap = o / bp, within = o - tap * bp;
-    const int ox = (int)(r % wo), oy = (int)((r / wo) % ho);
-    const int64_t img = r / ((int64_t)wo * ho);
-    int64_t src = -1;
-    if (tap < kh * kw) {
-        const int iy = oy + tap / kw - pad, ix = ox + tap % kw - pad;
-        if (iy >= 0 && iy < h && ix >= 0 && ix < w) src = (img * h + iy) * w + ix;
+// image. One warp per output row, 16 bytes per lane and step (row tails beyond the last tap are zeroed too).
+constexpr int IM2COL_MAX_TAPS = 64, IM2COL_ROWS = 64;
+
+__global__ void __launch_bounds__(256)
+im2col_gather(const int8_t* __restrict__ xm, const int8_t* __restrict__ xe, int kst_x, int64_t ps_x,
+              int h, int w, int ho, int wo, int kh, int kw, int pad, int lg_bp, int planes,
+              uint32_t rows_out, int kst_out, int64_t ps_out, int64_t rs_out,
+              int8_t* __restrict__ om, int8_t* __restrict__ oe) {
+    // A CTA takes 64 consecutive output rows, a warp eight of them; the lanes sweep a row 16 bytes at a
+    // time. The filter offsets of the taps are tabulated once per CTA, the pixel coordinates once per row
+    // (32-bit arithmetic: the host checks the sizes), and the exponents of the 64 rows are collected in
+    // shared memory so that each tap's bytes leave as whole sectors.
+    __shared__ int8_t s_e[IM2COL_MAX_TAPS][IM2COL_ROWS];
+    __shared__ int8_t s_dy[IM2COL_MAX_TAPS], s_dx[IM2COL_MAX_TAPS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t r0 = blockIdx.x * IM2COL_ROWS;
+    const int taps = kh * kw, chunks = kst_out >> 4;
+    if ((int)threadIdx.x < taps) {
+        s_dy[threadIdx.x] = (int8_t)((int)threadIdx.x / kw - pad);
+        s_dx[threadIdx.x] = (int8_t)((int)threadIdx.x % kw - pad);
     }
-    for (int pl = 0; pl < planes; ++pl) {
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (src >= 0) v = *reinterpret_cast<const uint4*>(xm + pl * ps_x + src * kst_x + within);
-        *reinterpret_cast<uint4*>(om + pl * ps_out + r * kst_out + o) = v;
+    __syncthreads();
+    const uint32_t per_img = (uint32_t)(ho * wo);
+    // four rows at a time, so that four independent loads are in flight per lane (eight were slower)
+    for (int k = 0; k < IM2COL_ROWS / 8; k += 4) {
+        int oy[4], ox[4];
+        int64_t img_base[4];
+        bool live[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t r = r0 + warp * (IM2COL_ROWS / 8) + k + q;
+            live[q] = r < rows_out;
+            const uint32_t rr = live[q] ? r : 0u;
+            const uint32_t img = rr / per_img, rem = rr - img * per_img;
+            oy[q] = (int)(rem / (uint32_t)wo);
+            ox[q] = (int)(rem - (uint32_t)oy[q] * (uint32_t)wo);
+            img_base[q] = (int64_t)img * h * w;
+        }
+        for (int ck = lane; ck < chunks; ck += 32) {
+            const int o = ck << 4;                              // byte offset in the output row
+            const int tap = o >> lg_bp, within = o - (tap << lg_bp);
+            const int dy = tap < taps ? s_dy[tap] : 0, dx = tap < taps ? s_dx[tap] : 0;
+            for (int pl = 0; pl < planes; ++pl) {
+                int64_t src[4];
+                uint4 v[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int iy = oy[q] + dy, ix = ox[q] + dx;
+                    src[q] = (tap < taps && iy >= 0 && iy < h && ix >= 0 && ix < w) ? img_base[q] + iy * w + ix : -1;
+                    v[q] = make_uint4(0u, 0u, 0u, 0u);
+                    if (src[q] >= 0) v[q] = *reinterpret_cast<const uint4*>(xm + pl * ps_x + src[q] * kst_x + within);
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int lr = warp * (IM2COL_ROWS / 8) + k + q;
+                    if (live[q]) {
+                        *reinterpret_cast<uint4*>(om + pl * ps_out + (int64_t)(r0 + lr) * kst_out + o) = v[q];
+                        if (pl == 0 && within == 0 && tap < taps) s_e[tap][lr] = src[q] >= 0 ? xe[src[q]] : (int8_t)-63;
+                    }
+                }
+            }
+        }
     }
-    if (within == 0 && tap < kh * kw) oe[(int64_t)tap * rs_out + r] = src >= 0 ? xe[src] : (int8_t)-63;
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < taps * IM2COL_ROWS; idx += 256) {
+        const int tap = idx / IM2COL_ROWS, j = idx % IM2COL_ROWS;
+        if (r0 + j < rows_out) oe[(int64_t)tap * rs_out + r0 + j] = s_e[tap][j];
+    }
 }
 
 // ------------------------------------------------------------------------------ inverse helpers
@@ -1179,9 +1223,12 @@ int launch_im2col_packed(const int8_t* xm, const int8_t* xe, int64_t n, int64_t 
     if (h > (1 << 20) || w > (1 << 20) || Lo.kst > (1ll << 30)) return HBFP_ERR_UNSUPPORTED;
     if (n == 0) return HBFP_OK;
     HBFP_CUDA_OK(cudaMemsetAsync(oe, 0, (size_t)Lo.exp_bytes, st));
-    const int64_t items = Lo.rows * (Lo.kst >> 4);
-    im2col_gather<<<blocks_for(items, 256), 256, 0, st>>>(xm, xe, Lx.kst, Lx.plane_stride, (int)h, (int)w, (int)ho, (int)wo, kh, kw,
-                                                         pad, (int)Lo.bp, (int)Lo.planes, Lo.rows, Lo.kst, Lo.plane_stride, Lo.rs, om, oe);
+    const int lg_bp = Lo.bp == 32 ? 5 : Lo.bp == 64 ? 6 : 7;
+    if (kh * kw > IM2COL_MAX_TAPS || kh > 100 || kw > 100 || pad > 100) return HBFP_ERR_UNSUPPORTED;
+    if (Lo.rows >= (1ll << 31) || Lx.rows >= (1ll << 31)) return HBFP_ERR_UNSUPPORTED;
+    im2col_gather<<<blocks_for(Lo.rows, IM2COL_ROWS), 256, 0, st>>>(xm, xe, (int)Lx.kst, Lx.plane_stride, (int)h, (int)w, (int)ho, (int)wo,
+                                                                   kh, kw, pad, lg_bp, (int)Lo.planes, (uint32_t)Lo.rows, (int)Lo.kst,
+                                                                   Lo.plane_stride, Lo.rs, om, oe);
     return launch_status();
 }
 

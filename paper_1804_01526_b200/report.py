@@ -107,6 +107,33 @@ def wide_lines(hbm_gbs):
     return out
 
 
+def conv_lines():
+    """Forward GEMM operand of the two 3x3 convolutions: converting the FP32 im2col matrix against
+    converting the activations once per pixel and gathering the packed operand."""
+    out = ["", "| convolution (forward) | im2col matrix FP32 MB | convert im2col matrix µs | convert pixels µs | gather packed operand µs | GEMM µs |",
+           "|---|---|---|---|---|---|"]
+    for name, n, hw, c, f in (("c2.conv64", 128, 32, 64, 64), ("c2.conv128", 128, 16, 128, 128)):
+        fmt = hb.Format(mant_bits=8, block=c)          # one block per pixel; the configuration's 64 for the first
+        x = torch.from_numpy(wl.draw("half_normal", (n * hw * hw, c), seed=5)).cuda()
+        wt = torch.from_numpy(wl.draw("he_weight", (9 * c, f), seed=6, fan_in=9 * c)).cuda()
+        px = hb.quantize(x, 1, fmt)
+        pa = hb.im2col_packed(px, n, hw, hw, c, 3, 3, 1)
+        pw = hb.quantize(wt, 0, fmt)
+        cols = hb.dequantize(pa) * 0 + 1.0              # an FP32 matrix of the im2col shape, for timing its conversion
+        pc = hb.quantize(cols, 1, fmt)
+        M, K = n * hw * hw, 9 * c
+        t_c = _time_auto(lambda: hb.quantize(cols, 1, fmt, out=pc))
+        t_p = _time_auto(lambda: hb.quantize(x, 1, fmt, out=px))
+        t_g = _time_auto(lambda: hb.im2col_packed(px, n, hw, hw, c, 3, 3, 1, out=pa))
+        C = torch.empty((M, f), dtype=torch.float32, device="cuda")
+        ws = torch.empty(max(hb.gemm_q_workspace(M, f, K, pa, pw), 1), dtype=torch.int8, device="cuda")
+        t_m = _time_auto(lambda: hb.gemm_q(M, f, K, pa, pw, out=C, workspace=ws))
+        out.append(f"| {name} {M}x{f}x{K} | {M*K*4/1e6:.0f} | {t_c*1e3:.1f} | {t_p*1e3:.1f} | {t_g*1e3:.1f} | {t_m*1e3:.1f} |")
+        del x, wt, px, pa, pw, cols, pc, C, ws
+    torch.cuda.empty_cache()
+    return out
+
+
 def rows_for(specs, tensors_np, peak_tops, hbm_gbs):
     dev = {k: torch.from_numpy(v).cuda() for k, v in tensors_np.items()}
     out = []
@@ -171,6 +198,8 @@ def main():
         lines += [""] + mlp_step_lines()
     if not args.only or args.only == "wide":
         lines += wide_lines(args.hbm_gbs)
+    if not args.only or args.only == "conv":
+        lines += conv_lines()
     text = "\n".join(lines) + "\n"
     if args.out:
         with open(args.out, "w") as f:
