@@ -218,7 +218,7 @@ static int wide_views_ok(void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* 
 int hbfp_wide_quantize(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* fmt, int16_t* wide,
                        int8_t* wide_exps, void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
     if (d0 < 0 || d1 < 0 || ld < d1 || !fmt) return HBFP_ERR_INVALID_ARG;
-    if ((!w && d0 * d1 > 0) || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    if (d0 * d1 > 0 && (!w || !wide || !wide_exps)) return HBFP_ERR_INVALID_ARG;
     int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
     if (rc) return rc;
     return launch_wide(0, w, ld, d0, d1, fmt, wide, wide_exps, static_cast<int8_t*>(mant_c0), exps_c0,
@@ -228,7 +228,7 @@ int hbfp_wide_quantize(const float* w, int64_t d0, int64_t d1, int64_t ld, const
 int hbfp_wide_update(int16_t* wide, int8_t* wide_exps, const float* delta, int64_t d0, int64_t d1, int64_t ldd,
                      const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
     if (d0 < 0 || d1 < 0 || ldd < d1 || !fmt) return HBFP_ERR_INVALID_ARG;
-    if ((!delta && d0 * d1 > 0) || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    if (d0 * d1 > 0 && (!delta || !wide || !wide_exps)) return HBFP_ERR_INVALID_ARG;
     int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
     if (rc) return rc;
     return launch_wide(1, delta, ldd, d0, d1, fmt, wide, wide_exps, static_cast<int8_t*>(mant_c0), exps_c0,
@@ -237,7 +237,7 @@ int hbfp_wide_update(int16_t* wide, int8_t* wide_exps, const float* delta, int64
 
 int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1, const hbfp_format* fmt,
                      void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1, void* stream) {
-    if (d0 < 0 || d1 < 0 || !fmt || !wide || !wide_exps) return HBFP_ERR_INVALID_ARG;
+    if (d0 < 0 || d1 < 0 || !fmt || (d0 * d1 > 0 && (!wide || !wide_exps))) return HBFP_ERR_INVALID_ARG;
     if (!mant_c0 || !mant_c1) return HBFP_ERR_INVALID_ARG;
     int rc = wide_views_ok(mant_c0, exps_c0, mant_c1, exps_c1);
     if (rc) return rc;

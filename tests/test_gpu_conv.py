@@ -76,3 +76,17 @@ def test_gather_argument_errors(hb):
     with pytest.raises(hb.HbfpError) as e:               # the block must be the channel count
         hb.im2col_packed(px, 1, 8, 8, 32, 3, 3, 1)
     assert e.value.code == hb.ERR_INVALID_ARG
+
+
+def test_gather_of_an_empty_batch_and_of_a_single_pixel(hb):
+    import torch
+    f = hb.Format(mant_bits=8, block=16)
+    px = hb.quantize(torch.empty((0, 16), device="cuda"), 1, f)
+    pa = hb.im2col_packed(px, 0, 4, 4, 16, 3, 3, 1)
+    assert pa.rows == 0 and hb.device_status() == 0
+    x = wl.draw("normal", (1, 16), seed=3)                      # a 1 x 1 image: eight of the nine taps lie outside
+    px = hb.quantize(to_dev(x), 1, f)
+    pa = hb.im2col_packed(px, 1, 1, 1, 16, 3, 3, 1)
+    q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
+    q_ref, s_ref = oracle.quantize(oracle.im2col(x.reshape(1, 1, 1, 16), 3, 3, 1), 1, oracle.Format(mant_bits=8, block=16))
+    assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)

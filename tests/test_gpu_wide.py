@@ -131,3 +131,13 @@ def test_wide_argument_errors(hb):
     wide, _ = hb.wide_quantize(w, hb.Format(mant_bits=8, block=16, tile=16), want_views=False)
     with pytest.raises(ValueError):
         hb.wide_update(wide, torch.zeros((32, 64), device="cuda"), hb.Format(mant_bits=8, block=16, tile=16))
+
+
+def test_wide_storage_of_an_empty_matrix(hb):
+    import torch
+    f = hb.Format(mant_bits=8, block=16, tile=16)
+    wide, views = hb.wide_quantize(torch.empty((0, 32), device="cuda"), f)
+    assert wide.mant.numel() == 0 and hb.device_status() == 0
+    hb.wide_update(wide, torch.empty((0, 32), device="cuda"), f, views=views)
+    hb.wide_narrow(wide, f, views=views)
+    assert hb.device_status() == 0
