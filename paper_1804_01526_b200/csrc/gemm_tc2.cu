@@ -186,7 +186,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 }
 
 // Tile copy issued by one CTA of a pair; the completion bytes may be counted on a barrier of
-// either CTA (`bar` is a cluster-window address). Plain copy: no multicast.
+// either CTA (`bar` is a cluster-window address). A plain copy to one destination.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t hint) {
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
