@@ -28,7 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
-    "hbfp_im2col_packed",
+    "hbfp_im2col_packed", "hbfp_im2col_packed_t",
 ]
 
 
@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_wide_update.argtypes = [p, p, p, i64, i64, i64, p, p, p, p, p, p]
         L.hbfp_wide_narrow.argtypes = [p, p, i64, i64, p, p, p, p, p, p]
         L.hbfp_im2col_packed.argtypes = [p, p, i64, i64, i64, i64, i32, i32, i32, p, p, p, p]
+        L.hbfp_im2col_packed_t.argtypes = [p, i64, i64, i64, i64, i32, i32, i32, p, p, p, p]
         L.hbfp_unpack.argtypes = [p, p, i64, i64, p, p, p, p]
         L.hbfp_dequantize.argtypes = [p, p, i64, i64, p, p, i64, p]
         L.hbfp_gemm_workspace.argtypes = [i32, i32, i64, i64, i64, p, p, p]
@@ -272,6 +273,20 @@ def im2col_packed(px: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, 
     f = px.fmt.c()
     _check(lib().hbfp_im2col_packed(_dptr(px.mant), _dptr(px.exps), n, h, w, c, kh, kw, pad, ctypes.byref(f),
                                     _dptr(out.mant), _dptr(out.exps), _stream()), "hbfp_im2col_packed")
+    return out
+
+
+def im2col_packed_t(x: torch.Tensor, kh: int, kw: int, pad: int, fmt: Format, out: Optional[Packed] = None) -> Packed:
+    """hbfp_im2col_packed_t: the packed backward-weight operand ``[kh*kw*c][n*h*w]`` (blocks of
+    ``fmt.block`` consecutive output pixels) straight from FP32 activations ``x [n][h][w][c]``."""
+    if not (x.is_cuda and x.dtype == torch.float32 and x.dim() == 4 and x.is_contiguous()):
+        raise ValueError("x must be a contiguous float32 CUDA tensor [n][h][w][c]")
+    n, h, w, c = x.shape
+    if out is None:
+        out = alloc_packed(kh * kw * c, n * h * w, fmt, x.device)
+    f = fmt.c()
+    _check(lib().hbfp_im2col_packed_t(_dptr(x), n, h, w, c, kh, kw, pad, ctypes.byref(f), _dptr(out.mant),
+                                      _dptr(out.exps), _stream()), "hbfp_im2col_packed_t")
     return out
 
 

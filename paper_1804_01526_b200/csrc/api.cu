@@ -257,6 +257,15 @@ int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_t n, int6
                                 static_cast<int8_t*>(mant_out), exps_out, static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_im2col_packed_t(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw, int pad,
+                         const hbfp_format* fmt, void* mant, int8_t* exps, void* stream) {
+    if (!fmt || n < 0 || h <= 0 || w <= 0 || c <= 0 || kh <= 0 || kw <= 0 || pad < 0) return HBFP_ERR_INVALID_ARG;
+    if ((!x && n > 0) || !mant || !exps) return HBFP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mant) & 255) || (reinterpret_cast<uintptr_t>(exps) & 127)) return HBFP_ERR_ALIGNMENT;
+    return launch_im2col_cols(x, n, h, w, c, kh, kw, pad, fmt, static_cast<int8_t*>(mant), exps,
+                              static_cast<cudaStream_t>(stream));
+}
+
 int hbfp_unpack(const void* mant, const int8_t* exps, int64_t rows, int64_t k, const hbfp_format* fmt,
                 int16_t* q, int8_t* s, void* stream) {
     Packed p;

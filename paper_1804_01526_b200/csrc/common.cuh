@@ -77,6 +77,9 @@ int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, 
 // Packed convolution operand gathered from the packed per-pixel operand.
 int launch_im2col_packed(const int8_t* xm, const int8_t* xe, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
                          int pad, const hbfp_format* f, int8_t* om, int8_t* oe, cudaStream_t st);
+// Packed transposed convolution operand (blocks along the output pixels) straight from the FP32 activations.
+int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw, int pad,
+                       const hbfp_format* f, int8_t* mant, int8_t* exps, cudaStream_t st);
 int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st);
 int launch_dequantize(const Packed& p, float* out, int64_t ld, cudaStream_t st);
 

@@ -742,6 +742,73 @@ im2col_gather(const int8_t* __restrict__ xm, const int8_t* __restrict__ xe, int 
     }
 }
 
+// Backward-weight operand of a convolution without the FP32 im2col matrix: dW = cols^T dY contracts over the
+// output pixels, so cols^T [kh kw c][n h w] is quantised with blocks of b consecutive pixels along each
+// (tap, channel) row. A block is a window of the image shifted by the tap, so nothing can be shared between
+// taps except the loads: a CTA takes one block of b pixels (whole image rows: b % w == 0, h w % b == 0,
+// output as large as the input), stages the b / w + kh - 1 image rows it touches in shared memory once
+// (zeros outside the image) and lets each thread quantise (tap, channel) rows: two passes over its b
+// values in shared memory, b contiguous mantissa bytes out.
+template <int PLANES>
+__global__ void __launch_bounds__(256)
+im2col_cols(const float* __restrict__ x, int h, int w, int c, int kh, int kw, int pad, int b, int bp, QParams p,
+            int64_t kst, int64_t plane_stride, int64_t rs, int8_t* __restrict__ mant, int8_t* __restrict__ exps) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* img_rows = reinterpret_cast<float*>(smem_raw);        // [b / w + kh - 1][w][c]
+    const int tid = threadIdx.x;
+    const int64_t pb = blockIdx.x;                               // pixel block
+    const int64_t p0 = pb * b;
+    const int per_img = h * w;
+    const int64_t img = p0 / per_img;
+    const int oy0 = (int)((p0 - img * per_img) / w);
+    const int rows_here = b / w, srows = rows_here + kh - 1;
+    // stage the source rows oy0 - pad .. oy0 + rows_here - 1 + (kh - 1 - pad)
+    const int row_elems = w * c;
+    for (int e = tid * 4; e < srows * row_elems; e += 256 * 4) {
+        const int sr = e / row_elems, off = e - sr * row_elems;
+        const int iy = oy0 - pad + sr;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (iy >= 0 && iy < h) v = __ldg(reinterpret_cast<const float4*>(x + ((img * h + iy) * (int64_t)w) * c + off));
+        *reinterpret_cast<float4*>(img_rows + e) = v;
+    }
+    __syncthreads();
+    const int taps = kh * kw;
+    for (int pair = tid; pair < taps * c; pair += 256) {
+        const int tap = pair / c, ch = pair - tap * c;
+        const int dy = tap / kw, dx = tap - dy * kw - pad;       // dy indexes the staged rows directly
+        uint32_t am = 0;
+        for (int px = 0; px < b; ++px) {
+            const int ry = px / w, ox = px - ry * w, ix = ox + dx;
+            const float v = (ix >= 0 && ix < w) ? img_rows[((ry + dy) * w + ix) * c + ch] : 0.f;
+            am = max(am, abs_bits(v));
+        }
+        const int s = block_exponent(am, p.m, p.exp_mode);
+        exps[pb * rs + pair] = (int8_t)s;
+        int8_t* dst = mant + (int64_t)pair * kst + pb * bp;
+        for (int px0 = 0; px0 < bp; px0 += 4) {
+            uint32_t hi = 0, lo = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int px = px0 + j;
+                int q = 0;
+                if (px < b) {
+                    const int ry = px / w, ox = px - ry * w, ix = ox + dx;
+                    const int iy = oy0 - pad + ry + dy;
+                    if (ix >= 0 && ix < w && iy >= 0 && iy < h) {
+                        const float v = img_rows[((ry + dy) * w + ix) * c + ch];
+                        // stochastic rounding draws by the element's index in the activation tensor
+                        q = quantize_one(v, s, p, (uint64_t)(((img * h + iy) * (int64_t)w + ix) * c + ch));
+                    }
+                }
+                if (PLANES == 1) hi |= (uint32_t)(q & 0xff) << (8 * j);
+                else { hi |= (uint32_t)((q >> 4) & 0xff) << (8 * j); lo |= (uint32_t)(q & 15) << (8 * j); }
+            }
+            *reinterpret_cast<uint32_t*>(dst + px0) = hi;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + plane_stride + px0) = lo;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------ inverse helpers
 
 __global__ void unpack_kernel(const int8_t* __restrict__ mant, const int8_t* __restrict__ exps, int64_t rows,
@@ -1229,6 +1296,33 @@ int launch_im2col_packed(const int8_t* xm, const int8_t* xe, int64_t n, int64_t 
     im2col_gather<<<blocks_for(Lo.rows, IM2COL_ROWS), 256, 0, st>>>(xm, xe, (int)Lx.kst, Lx.plane_stride, (int)h, (int)w, (int)ho, (int)wo,
                                                                    kh, kw, pad, lg_bp, (int)Lo.planes, (uint32_t)Lo.rows, (int)Lo.kst,
                                                                    Lo.plane_stride, Lo.rs, om, oe);
+    return launch_status();
+}
+
+int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw, int pad,
+                       const hbfp_format* f, int8_t* mant, int8_t* exps, cudaStream_t st) {
+    if (f->tile != 0 || f->block <= 0) return HBFP_ERR_INVALID_ARG;
+    const int64_t b = f->block;
+    // same-size output, blocks of whole image rows that do not straddle images
+    if (2 * pad != kh - 1 || 2 * pad != kw - 1) return HBFP_ERR_UNSUPPORTED;
+    if (b > 128 || b % w != 0 || (h * w) % b != 0 || c % 4 != 0 || (reinterpret_cast<uintptr_t>(x) & 15)) return HBFP_ERR_UNSUPPORTED;
+    Layout L;
+    int rc = make_layout((int64_t)kh * kw * c, n * h * w, f, &L);
+    if (rc) return rc;
+    if (n == 0) return HBFP_OK;
+    if (h > 32768 || w > 32768 || c > 4096 || L.nkb >= (1ll << 31)) return HBFP_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)(b / w + kh - 1) * w * c * sizeof(float);
+    if (smem > 200 * 1024) return HBFP_ERR_UNSUPPORTED;
+    const QParams p = make_params(f);
+    if (L.rs != L.rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+    if (L.kst != L.nkb * L.bp) HBFP_CUDA_OK(cudaMemsetAsync(mant, 0, (size_t)L.mant_bytes, st));     // row tails
+    if (L.planes == 1) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(im2col_cols<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        im2col_cols<1><<<(unsigned)L.nkb, 256, smem, st>>>(x, (int)h, (int)w, (int)c, kh, kw, pad, (int)b, (int)L.bp, p, L.kst, L.plane_stride, L.rs, mant, exps);
+    } else {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(im2col_cols<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        im2col_cols<2><<<(unsigned)L.nkb, 256, smem, st>>>(x, (int)h, (int)w, (int)c, kh, kw, pad, (int)b, (int)L.bp, p, L.kst, L.plane_stride, L.rs, mant, exps);
+    }
     return launch_status();
 }
 

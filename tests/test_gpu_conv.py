@@ -90,3 +90,42 @@ def test_gather_of_an_empty_batch_and_of_a_single_pixel(hb):
     q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
     q_ref, s_ref = oracle.quantize(oracle.im2col(x.reshape(1, 1, 1, 16), 3, 3, 1), 1, oracle.Format(mant_bits=8, block=16))
     assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
+
+
+@pytest.mark.parametrize("n,hw,c,b,m,rounding", [(2, 32, 64, 64, 8, 0), (3, 16, 128, 64, 8, 0), (2, 8, 24, 32, 8, 0),
+                                                 (1, 16, 32, 128, 12, 0), (2, 16, 16, 16, 6, 0)])
+def test_backward_weight_operand_equals_column_quantised_im2col_matrix(hb, n, hw, c, b, m, rounding):
+    x = wl.draw("half_normal", (n * hw * hw, c), seed=81).reshape(n, hw, hw, c)
+    x *= np.exp(wl.draw("normal", (n * hw * hw, 1), seed=82)).reshape(n, hw, hw, 1).astype(np.float32)
+    fd = dict(mant_bits=m, block=b, rounding=rounding, seed=0)
+    pa = hb.im2col_packed_t(to_dev(x), 3, 3, 1, gfmt(fd))
+    assert hb.device_status() == 0
+    cols = oracle.im2col(x, 3, 3, 1)
+    q_ref, s_ref = oracle.quantize(cols, 0, ofmt(fd))
+    q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
+    assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
+
+
+def test_convolution_backward_weight_gemm(hb):
+    n, hw, c, f = 4, 32, 64, 64
+    x = wl.draw("half_normal", (n * hw * hw, c), seed=83).reshape(n, hw, hw, c)
+    dy = wl.draw("grad", (n * hw * hw, f), seed=84)
+    fd = dict(mant_bits=8, block=64, rounding=0, seed=0)
+    pa = hb.im2col_packed_t(to_dev(x), 3, 3, 1, gfmt(fd))
+    dW = hb.gemm_q(9 * c, f, n * hw * hw, pa, to_dev(dy), fmtB=gfmt(fd)).cpu().numpy()
+    assert hb.device_status() == 0
+    cols = oracle.im2col(x, 3, 3, 1)
+    ref = oracle.hbfp_gemm(1, 0, cols, dy, ofmt(fd), ofmt(fd))
+    err = np.abs(dW.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+
+
+def test_backward_weight_operand_refuses_what_it_does_not_cover(hb):
+    import torch
+    x = torch.zeros((1, 8, 8, 16), device="cuda")
+    with pytest.raises(hb.HbfpError) as e:                 # a block that is not whole image rows
+        hb.im2col_packed_t(x, 3, 3, 1, hb.Format(mant_bits=8, block=12))
+    assert e.value.code == hb.ERR_UNSUPPORTED
+    with pytest.raises(hb.HbfpError) as e:                 # an output smaller than the input
+        hb.im2col_packed_t(x, 3, 3, 0, hb.Format(mant_bits=8, block=16))
+    assert e.value.code == hb.ERR_UNSUPPORTED
