@@ -746,23 +746,27 @@ im2col_gather(const int8_t* __restrict__ xm, const int8_t* __restrict__ xe, int 
 // output pixels, so cols^T [kh kw c][n h w] is quantised with blocks of b consecutive pixels along each
 // (tap, channel) row. A block is a window of the image shifted by the tap, so nothing can be shared between
 // taps except the loads: a CTA takes one block of b pixels (whole image rows: b % w == 0, h w % b == 0,
-// output as large as the input), stages the b / w + kh - 1 image rows it touches in shared memory once
-// (zeros outside the image) and lets each thread quantise (tap, channel) rows: two passes over its b
-// values in shared memory, b contiguous mantissa bytes out.
-template <int PLANES>
+// output as large as the input) and stages the b / w + kh - 1 image rows it touches in shared memory once
+// (zeros outside the image). Then, tap by tap and 64 channels at a time, thread (channel, quarter) keeps its
+// quarter of the block's pixels in registers between the maximum (exchanged through shared memory) and the
+// rounding, and writes its b / 4 mantissa bytes with 16-byte stores.
+template <int PLANES, int NPX, bool SR>      // NPX = b / 4 pixels per thread: 4, 8, 16 or 32
 __global__ void __launch_bounds__(256)
-im2col_cols(const float* __restrict__ x, int h, int w, int c, int kh, int kw, int pad, int b, int bp, QParams p,
+im2col_cols(const float* __restrict__ x, int h, int w, int lg_w, int c, int kh, int kw, int pad, QParams p,
             int64_t kst, int64_t plane_stride, int64_t rs, int8_t* __restrict__ mant, int8_t* __restrict__ exps) {
+    constexpr int B = 4 * NPX;
+    constexpr int BP = B <= 32 ? 32 : B <= 64 ? 64 : 128;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* img_rows = reinterpret_cast<float*>(smem_raw);        // [b / w + kh - 1][w][c]
-    const int tid = threadIdx.x;
+    float* img_rows = reinterpret_cast<float*>(smem_raw);        // [B / w + kh - 1][w][c]
+    __shared__ uint32_t pmax[4][64];
+    const int tid = threadIdx.x, chl = tid & 63, q = tid >> 6;
     const int64_t pb = blockIdx.x;                               // pixel block
-    const int64_t p0 = pb * b;
+    const int64_t p0 = pb * B;
     const int per_img = h * w;
     const int64_t img = p0 / per_img;
-    const int oy0 = (int)((p0 - img * per_img) / w);
-    const int rows_here = b / w, srows = rows_here + kh - 1;
-    // stage the source rows oy0 - pad .. oy0 + rows_here - 1 + (kh - 1 - pad)
+    const int oy0 = (int)((p0 - img * per_img) >> lg_w);
+    const int srows = (B >> lg_w) + kh - 1;
+    // stage the source rows oy0 - pad .. oy0 + B / w - 1 + (kh - 1 - pad)
     const int row_elems = w * c;
     for (int e = tid * 4; e < srows * row_elems; e += 256 * 4) {
         const int sr = e / row_elems, off = e - sr * row_elems;
@@ -772,39 +776,83 @@ im2col_cols(const float* __restrict__ x, int h, int w, int c, int kh, int kw, in
         *reinterpret_cast<float4*>(img_rows + e) = v;
     }
     __syncthreads();
+    const uint32_t qm = qmax_pair(p.qmax), nqm = neg_qmax_pair(p.qmax);
     const int taps = kh * kw;
-    for (int pair = tid; pair < taps * c; pair += 256) {
-        const int tap = pair / c, ch = pair - tap * c;
-        const int dy = tap / kw, dx = tap - dy * kw - pad;       // dy indexes the staged rows directly
-        uint32_t am = 0;
-        for (int px = 0; px < b; ++px) {
-            const int ry = px / w, ox = px - ry * w, ix = ox + dx;
-            const float v = (ix >= 0 && ix < w) ? img_rows[((ry + dy) * w + ix) * c + ch] : 0.f;
-            am = max(am, abs_bits(v));
-        }
-        const int s = block_exponent(am, p.m, p.exp_mode);
-        exps[pb * rs + pair] = (int8_t)s;
-        int8_t* dst = mant + (int64_t)pair * kst + pb * bp;
-        for (int px0 = 0; px0 < bp; px0 += 4) {
-            uint32_t hi = 0, lo = 0;
+    // this thread's pixels: column in the image row and offset in the staged rows, worked out once
+    int ox_of[NPX], off_of[NPX];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int px = px0 + j;
-                int q = 0;
-                if (px < b) {
-                    const int ry = px / w, ox = px - ry * w, ix = ox + dx;
-                    const int iy = oy0 - pad + ry + dy;
-                    if (ix >= 0 && ix < w && iy >= 0 && iy < h) {
-                        const float v = img_rows[((ry + dy) * w + ix) * c + ch];
-                        // stochastic rounding draws by the element's index in the activation tensor
-                        q = quantize_one(v, s, p, (uint64_t)(((img * h + iy) * (int64_t)w + ix) * c + ch));
+    for (int j = 0; j < NPX; ++j) {
+        const int px = q * NPX + j;
+        ox_of[j] = px & (w - 1);
+        off_of[j] = px * c;                                      // ((px >> lg_w) * w + ox) * c
+    }
+    for (int c0 = 0; c0 < c; c0 += 64) {
+        const int ch = c0 + chl;
+        const bool live = ch < c;
+        for (int tap = 0; tap < taps; ++tap) {
+            const int dy = tap / kw, dx = tap - dy * kw - pad;   // dy indexes the staged rows directly
+            const float* tap_base = img_rows + (dy * w + dx) * c + (live ? ch : 0);
+            float v[NPX];
+            uint32_t am = 0;
+#pragma unroll
+            for (int j = 0; j < NPX; ++j)
+                v[j] = (live && (unsigned)(ox_of[j] + dx) < (unsigned)w) ? tap_base[off_of[j]] : 0.f;
+#pragma unroll
+            for (int j = 0; j < NPX; j += 2) am = max3_abs_bits(am, v[j], v[j + 1]);
+            pmax[q][chl] = am;
+            __syncthreads();
+            am = max(max(pmax[0][chl], pmax[1][chl]), max(pmax[2][chl], pmax[3][chl]));
+            __syncthreads();                                     // pmax is rewritten by the next tap
+            if (!live) continue;
+            const int s = block_exponent(am, p.m, p.exp_mode);
+            const int64_t row = (int64_t)tap * c + ch;
+            if (q == 0) exps[pb * rs + row] = (int8_t)s;
+            const float sc = pow2f(SR ? 16 - s : -s);
+            uint32_t hi[NPX / 4], lo[NPX / 4];
+#pragma unroll
+            for (int wi = 0; wi < NPX / 4; ++wi) {
+                uint32_t r[4] = {0u, 0u, 0u, 0u};
+                if (SR) {
+                    // stochastic rounding draws by the element's index in the activation tensor
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int px = q * NPX + 4 * wi + j, ry = px >> lg_w, ix = (px & (w - 1)) + dx;
+                        const int iy = oy0 - pad + ry + dy;
+                        if (ix >= 0 && ix < w && iy >= 0 && iy < h)
+                            r[j] = draw_of_element(p, (uint64_t)(((img * h + iy) * (int64_t)w + ix) * c + ch));
                     }
                 }
-                if (PLANES == 1) hi |= (uint32_t)(q & 0xff) << (8 * j);
-                else { hi |= (uint32_t)((q >> 4) & 0xff) << (8 * j); lo |= (uint32_t)(q & 15) << (8 * j); }
+                uint32_t h01, h23;
+                if (SR) {
+                    h01 = round_sr_pair2(v[4 * wi], v[4 * wi + 1], sc, r[0], r[1], qm, nqm);
+                    h23 = round_sr_pair2(v[4 * wi + 2], v[4 * wi + 3], sc, r[2], r[3], qm, nqm);
+                } else {
+                    h01 = round_rne_pair(v[4 * wi], v[4 * wi + 1], sc, qm, nqm);
+                    h23 = round_rne_pair(v[4 * wi + 2], v[4 * wi + 3], sc, qm, nqm);
+                }
+                pack4<PLANES>(h01, h23, hi[wi], lo[wi]);
             }
-            *reinterpret_cast<uint32_t*>(dst + px0) = hi;
-            if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + plane_stride + px0) = lo;
+            int8_t* dst = mant + row * kst + pb * BP + q * NPX;
+            if (NPX >= 16) {
+#pragma unroll
+                for (int i = 0; i < NPX / 16; ++i) {
+                    *reinterpret_cast<uint4*>(dst + 16 * i) = make_uint4(hi[4 * i], hi[4 * i + 1], hi[4 * i + 2], hi[4 * i + 3]);
+                    if (PLANES == 2) *reinterpret_cast<uint4*>(dst + plane_stride + 16 * i) = make_uint4(lo[4 * i], lo[4 * i + 1], lo[4 * i + 2], lo[4 * i + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < NPX / 4; ++i) {
+                    *reinterpret_cast<uint32_t*>(dst + 4 * i) = hi[i];
+                    if (PLANES == 2) *reinterpret_cast<uint32_t*>(dst + plane_stride + 4 * i) = lo[i];
+                }
+            }
+            if (B < BP && q == 0) {                              // block padding (16-pixel blocks in 32 bytes)
+#pragma unroll
+                for (int px0 = B; px0 < BP; px0 += 4) {
+                    *reinterpret_cast<uint32_t*>(mant + row * kst + pb * BP + px0) = 0u;
+                    if (PLANES == 2) *reinterpret_cast<uint32_t*>(mant + plane_stride + row * kst + pb * BP + px0) = 0u;
+                }
+            }
         }
     }
 }
@@ -1305,24 +1353,38 @@ int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t 
     const int64_t b = f->block;
     // same-size output, blocks of whole image rows that do not straddle images
     if (2 * pad != kh - 1 || 2 * pad != kw - 1) return HBFP_ERR_UNSUPPORTED;
-    if (b > 128 || b % w != 0 || (h * w) % b != 0 || c % 4 != 0 || (reinterpret_cast<uintptr_t>(x) & 15)) return HBFP_ERR_UNSUPPORTED;
+    if (!(b == 16 || b == 32 || b == 64 || b == 128) || b % w != 0 || w < 4 || (w & (w - 1)) != 0 || (h * w) % b != 0 ||
+        c % 4 != 0 || (reinterpret_cast<uintptr_t>(x) & 15))
+        return HBFP_ERR_UNSUPPORTED;
     Layout L;
     int rc = make_layout((int64_t)kh * kw * c, n * h * w, f, &L);
     if (rc) return rc;
     if (n == 0) return HBFP_OK;
-    if (h > 32768 || w > 32768 || c > 4096 || L.nkb >= (1ll << 31)) return HBFP_ERR_UNSUPPORTED;
+    if (h > 32768 || c > 4096 || L.nkb >= (1ll << 31)) return HBFP_ERR_UNSUPPORTED;
     const size_t smem = (size_t)(b / w + kh - 1) * w * c * sizeof(float);
     if (smem > 200 * 1024) return HBFP_ERR_UNSUPPORTED;
     const QParams p = make_params(f);
     if (L.rs != L.rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
     if (L.kst != L.nkb * L.bp) HBFP_CUDA_OK(cudaMemsetAsync(mant, 0, (size_t)L.mant_bytes, st));     // row tails
+    int lg_w = 0;
+    while ((1 << lg_w) < w) ++lg_w;
+#define HBFP_COLS_LAUNCH2(PL, NPX, SRV)                                                                                       \
+    do {                                                                                                                       \
+        HBFP_CUDA_OK(cudaFuncSetAttribute(im2col_cols<PL, NPX, SRV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   \
+        im2col_cols<PL, NPX, SRV><<<(unsigned)L.nkb, 256, smem, st>>>(x, (int)h, (int)w, lg_w, (int)c, kh, kw, pad, p, L.kst,     \
+                                                                     L.plane_stride, L.rs, mant, exps);                        \
+    } while (0)
+#define HBFP_COLS_LAUNCH(PL, NPX)                                                 \
+    do {                                                                          \
+        if (p.rounding == 1) HBFP_COLS_LAUNCH2(PL, NPX, true); else HBFP_COLS_LAUNCH2(PL, NPX, false); \
+    } while (0)
     if (L.planes == 1) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(im2col_cols<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        im2col_cols<1><<<(unsigned)L.nkb, 256, smem, st>>>(x, (int)h, (int)w, (int)c, kh, kw, pad, (int)b, (int)L.bp, p, L.kst, L.plane_stride, L.rs, mant, exps);
+        if (b == 16) HBFP_COLS_LAUNCH(1, 4); else if (b == 32) HBFP_COLS_LAUNCH(1, 8); else if (b == 64) HBFP_COLS_LAUNCH(1, 16); else HBFP_COLS_LAUNCH(1, 32);
     } else {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(im2col_cols<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        im2col_cols<2><<<(unsigned)L.nkb, 256, smem, st>>>(x, (int)h, (int)w, (int)c, kh, kw, pad, (int)b, (int)L.bp, p, L.kst, L.plane_stride, L.rs, mant, exps);
+        if (b == 16) HBFP_COLS_LAUNCH(2, 4); else if (b == 32) HBFP_COLS_LAUNCH(2, 8); else if (b == 64) HBFP_COLS_LAUNCH(2, 16); else HBFP_COLS_LAUNCH(2, 32);
     }
+#undef HBFP_COLS_LAUNCH2
+#undef HBFP_COLS_LAUNCH
     return launch_status();
 }
 
