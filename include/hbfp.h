@@ -182,11 +182,10 @@ HBFP_API int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_
  * the n*h*w output pixels, so the A operand is cols^T with blocks of fmt->block consecutive pixels
  * along each (tap, channel) row. This call converts it straight from the FP32 activations x
  * [n][h][w][c] (16-byte aligned, c % 4 == 0): rows = kh*kw*c, k = n*h*w, bit-identical to
- * hbfp_quantize(im2col matrix, contract_axis 0) under nearest-even rounding (stochastic rounding
- * draws by the element's index in x). Supported: output as large as the input (2 pad == kh - 1 ==
- * kw - 1), blocks of whole image rows (block in {16, 32, 64, 128}, block % w == 0, h*w % block == 0), w a power
- * of two >= 4; anything else
- * returns HBFP_ERR_UNSUPPORTED (convert the im2col matrix instead). mant / exps: buffers of the
+ * hbfp_quantize(im2col matrix, contract_axis 0). Supported: nearest-even rounding, an output as
+ * large as the input (2 pad == kh - 1 == kw - 1), blocks of whole image rows (block in {16, 32, 64,
+ * 128}, block % w == 0, h*w % block == 0), w a power of two >= 4; anything else returns
+ * HBFP_ERR_UNSUPPORTED (convert the im2col matrix instead). mant / exps: buffers of the
  * sizes hbfp_packed_sizes(kh*kw*c, n*h*w) returns, fully overwritten. */
 HBFP_API int hbfp_im2col_packed_t(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
                                   int pad, const hbfp_format* fmt, void* mant, int8_t* exps, void* stream);

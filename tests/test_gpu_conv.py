@@ -129,3 +129,11 @@ def test_backward_weight_operand_refuses_what_it_does_not_cover(hb):
     with pytest.raises(hb.HbfpError) as e:                 # an output smaller than the input
         hb.im2col_packed_t(x, 3, 3, 0, hb.Format(mant_bits=8, block=16))
     assert e.value.code == hb.ERR_UNSUPPORTED
+
+
+def test_backward_weight_operand_is_nearest_even_only(hb):
+    import torch
+    x = torch.zeros((1, 8, 8, 16), device="cuda")
+    with pytest.raises(hb.HbfpError) as e:
+        hb.im2col_packed_t(x, 3, 3, 1, hb.Format(mant_bits=8, block=16, rounding=1))
+    assert e.value.code == hb.ERR_UNSUPPORTED
