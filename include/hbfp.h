@@ -138,8 +138,11 @@ HBFP_API int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t
  * tile x tile square, [ceil(d0/t)][ceil(d1/t)] (device). fmt->tile == fmt->block = t in 1..128;
  * fmt->rounding, seed, stream_id and exp_mode govern the conversion to 16 bits (stochastic rounding
  * draws by the element's row-major index in w); fmt->mant_bits = m in 3..12 is the width of the narrow
- * copy: its mantissas are the top m bits of the wide ones (floor(q16 / 2^(16-m)), which can reach
- * -2^(m-1)) under the exponent s16 + 16 - m. The narrow copy is written as the two packed views of
+ * copy: its mantissas are the top m bits of the stored words, a stored word being the mantissa plus
+ * half a narrow unit, i.e. clamp(floor((q16 + 2^(15-m)) / 2^(16-m)), +-(2^(m-1) - 1)): the wide value
+ * rounded to nearest, ties upward (plain truncation would leave every narrow weight half a narrow ULP
+ * low, a bias that adds up over a dot product), under the exponent s16 + 16 - m. The narrow copy is
+ * written as the two packed views of
  * hbfp_quantize_tiles (`*_c0`: rows = d1, k = d0; `*_c1`: rows = d0, k = d1; buffers of the sizes
  * hbfp_packed_sizes returns, fully overwritten); both mant_c0 and mant_c1 may be NULL to skip it, one
  * of them alone may not.

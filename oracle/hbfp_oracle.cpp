@@ -22,8 +22,8 @@
 // a float64 numpy restatement, idempotence, exact pass-through, power-of-two equivariance,
 // sign symmetry, half-ULP / one-ULP error bounds, exhaustive stochastic-rounding mean,
 // published Philox4x32-10 known answers, Eq. 2 against a float64 matmul of de-quantised
-// operands, exact-rational sums on tiny shapes and closed forms; wide storage: the floor
-// bracket in exact rationals, agreement with direct quantisation on narrow-representable
+// operands, exact-rational sums on tiny shapes and closed forms; wide storage: the half-ULP
+// bracket in exact rationals, the absence of a systematic offset, agreement with direct quantisation on narrow-representable
 // weights, idempotence of the zero update, a binary32 numpy restatement of the update and
 // exact integer steps. No function here is "parity unpinned".
 
@@ -313,10 +313,15 @@ int oracle_hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K,
 // ---------------------------------------------------------------------------------------
 // Wide weight storage (Sec. 4.2): the long-lived copy of a weight matrix keeps 16-bit
 // mantissas (one exponent per t x t tile); forward and backward passes read only the m most
-// significant bits of each mantissa. In canonical arrays:
-//   narrow mantissa = floor(q16 / 2^(16-m))     (the top m bits of the two's-complement word)
+// significant bits of each stored word. Plain truncation of the two's-complement mantissa would
+// make every narrow weight half a narrow ULP too small on average, a bias that adds up coherently
+// over a dot product with same-signed activations; the stored word is therefore the mantissa plus
+// half a narrow ULP, so that its top m bits are the mantissa rounded to nearest (ties upward),
+// which is also what the paper's simulation feeds the passes (the weights rounded to the narrow
+// format, Sec. 5.1). In canonical arrays:
+//   narrow mantissa = clamp( floor((q16 + 2^(15-m)) / 2^(16-m)), +-(2^(m-1) - 1) )
 //   narrow exponent = s16 + (16 - m)            (the weight of the narrow LSB)
-// so the narrow value never exceeds the wide one and lies less than one narrow ULP below it.
+// so the narrow value lies within half a narrow ULP of the wide one (one ULP where it saturates).
 // n_q mantissas, n_s exponents. Returns 0; -2 for m outside [2, 16].
 // ---------------------------------------------------------------------------------------
 int oracle_wide_narrow(const int16_t* q16, const int8_t* s16, int64_t n_q, int64_t n_s, int m,
@@ -324,10 +329,11 @@ int oracle_wide_narrow(const int16_t* q16, const int8_t* s16, int64_t n_q, int64
     if (!q16 || !s16 || !qm || !sm || n_q < 0 || n_s < 0) return -1;
     if (m < 2 || m > 16) return -2;
     const int64_t d = (int64_t)1 << (16 - m);
+    const int64_t half = d / 2;                                  // 0 when m = 16
     for (int64_t i = 0; i < n_q; ++i) {
-        int64_t v = q16[i];
+        int64_t v = (int64_t)q16[i] + half;
         int64_t fl = v >= 0 ? v / d : -((-v + d - 1) / d);      // floor division
-        qm[i] = (int16_t)fl;
+        qm[i] = (int16_t)clamp_q(fl, m);
     }
     for (int64_t i = 0; i < n_s; ++i) sm[i] = (int8_t)(s16[i] + (16 - m));
     return 0;

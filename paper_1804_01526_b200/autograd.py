@@ -92,3 +92,76 @@ class HbfpLinear(torch.nn.Module):
 
     def forward(self, x: torch.Tensor) -> torch.Tensor:
         return _HbfpLinearFn.apply(x, self.weight, self.bias, self)
+
+
+class _HbfpConv3x3Fn(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, x, weight, layer):
+        n, h, w, c = x.shape
+        ctx.layer = layer
+        ctx.save_for_backward(x)
+        x = x.contiguous()
+        px = hb.quantize(x.view(n * h * w, c), 1, layer.fmt_pixels(0))
+        pa = hb.im2col_packed(px, n, h, w, c, 3, 3, 1)
+        y = hb.gemm_q(n * h * w, layer.fout, 9 * c, pa, layer.views[0])
+        return y.view(n, h, w, layer.fout)
+
+    @staticmethod
+    def backward(ctx, dy):
+        layer = ctx.layer
+        (x,) = ctx.saved_tensors
+        n, h, w, c = x.shape
+        f = layer.fout
+        dy2 = dy.contiguous().view(n * h * w, f)
+        dx = dw = None
+        if ctx.needs_input_grad[0]:
+            # gradient of the im2col matrix, then its scatter back onto the pixels (an FP32 operation)
+            dcols = hb.gemm_q(n * h * w, 9 * c, f, dy2, layer.views[1], fmtA=layer.fmt_pixels(2)).view(n, h, w, 3, 3, c)
+            dxp = torch.zeros((n, h + 2, w + 2, c), device=x.device)
+            for i in range(3):
+                for j in range(3):
+                    dxp[:, i:i + h, j:j + w, :] += dcols[:, :, :, i, j, :]
+            dx = dxp[:, 1:h + 1, 1:w + 1, :].contiguous()
+        if ctx.needs_input_grad[1]:
+            pa_t = hb.im2col_packed_t(x.contiguous(), 3, 3, 1, layer.fmt_batch(0))
+            dw = hb.gemm_q(9 * c, f, n * h * w, pa_t, dy2, fmtB=layer.fmt_batch(2))
+        return dx, dw, None
+
+
+class HbfpConv3x3(torch.nn.Module):
+    """3 x 3 convolution, stride 1, one pixel of zero padding, channels-last activations ``[n][h][w][c]``,
+    as three BFP GEMMs (Sec. 5.1) without an FP32 im2col matrix: the forward operand is gathered from
+    activations converted once per pixel, the backward-weight operand is converted straight from the
+    activations, backward-data is a GEMM followed by the FP32 scatter onto the pixels. The weights
+    ``[9 c][filters]`` (rows ordered (filter row, filter column, channel)) live in wide storage with
+    ``c x c`` tiles, so the K-blocks of weights and activations coincide. Nearest-even rounding."""
+
+    def __init__(self, c: int, fout: int, mant_bits: int = 8, pixel_block: int = 64, device="cuda"):
+        super().__init__()
+        self.c, self.fout, self.mant_bits, self.pixel_block = c, fout, mant_bits, pixel_block
+        self.weight = torch.nn.Parameter(torch.randn(9 * c, fout, device=device) * (2.0 / (9 * c)) ** 0.5)
+        self.wide, self.views = hb.wide_quantize(self.weight.data, self.fmt_weight())
+        self._refresh_fp32_copy()
+
+    def fmt_weight(self) -> hb.Format:
+        return hb.Format(mant_bits=self.mant_bits, block=self.c, tile=self.c)
+
+    def fmt_pixels(self, which: int) -> hb.Format:
+        """X (blocks of c channels per pixel) or dY (blocks of c filters per pixel)."""
+        return hb.Format(mant_bits=self.mant_bits, block=self.c, stream_id=which)
+
+    def fmt_batch(self, which: int) -> hb.Format:
+        """Backward-weight: blocks of ``pixel_block`` consecutive output pixels."""
+        return hb.Format(mant_bits=self.mant_bits, block=self.pixel_block, stream_id=which)
+
+    def _refresh_fp32_copy(self) -> None:
+        t = self.c
+        scale = torch.exp2(self.wide.exps.float()).repeat_interleave(t, 0).repeat_interleave(t, 1)
+        self.weight.data = self.wide.mant.float() * scale[: 9 * self.c, : self.fout]
+
+    def apply_update(self, delta: torch.Tensor) -> None:
+        hb.wide_update(self.wide, delta.contiguous(), self.fmt_weight(), views=self.views)
+        self._refresh_fp32_copy()
+
+    def forward(self, x: torch.Tensor) -> torch.Tensor:
+        return _HbfpConv3x3Fn.apply(x, self.weight, self)

@@ -369,10 +369,12 @@ struct TileViews {
 };
 
 // qt rows have a pitch of tp + 2 halfwords, so that the column reads of view c0 spread over the banks.
-// sh: the views take the mantissas shifted down by sh bits (arithmetic: the top bits of wide storage).
+// sh: the views take the top bits of wide storage: the mantissa plus half a narrow unit, shifted down by sh
+// bits (arithmetic) and clamped to the symmetric range, i.e. rounded to nearest; sh = 0 copies.
 template <int PLANES>
 __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int hi, int wj, int64_t i0, int64_t j0,
-                                                 int64_t u, int64_t v, int s, int sh, const TileViews& tv, int tid) {
+                                                 int64_t u, int64_t v, int s, int sh, int qmax, const TileViews& tv, int tid) {
+    const int half = sh > 0 ? 1 << (sh - 1) : 0;
     const int qp = tp + 2;
     const int lg = 31 - __clz(tp >> 2), gmask = (tp >> 2) - 1;       // tp is 32, 64 or 128
     int8_t* const mant_c0 = tv.mant_c0; int8_t* const mant_c1 = tv.mant_c1;
@@ -385,7 +387,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[ii * qp + g + j] >> sh;
+            const int q = clampq((qt[ii * qp + g + j] + half) >> sh, qmax);
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -400,7 +402,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = qt[(g + j) * qp + jj] >> sh;
+            const int q = clampq((qt[(g + j) * qp + jj] + half) >> sh, qmax);
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -443,8 +445,8 @@ __device__ __forceinline__ int round_sr_wide(float x, int s, uint32_t r) {
 //   MODE 2  read wide storage only
 // In every mode, when view pointers are given, the tile goes to the two packed views
 //   c1: rows = d0, contraction along d1 (the stored orientation);  c0: rows = d1, contraction along d0
-// with, for the wide modes, the top p.m bits of the 16-bit mantissas (an arithmetic shift) under the
-// exponent s + 16 - p.m.
+// with, for the wide modes, the top p.m bits of the stored 16-bit words (the mantissa plus half a narrow
+// unit: rounded to nearest, clamped to the symmetric range) under the exponent s + 16 - p.m.
 // FAST: t, d1 multiples of 8, pitches and bases 16-byte aligned: a thread handles eight consecutive
 // weights of a row at a time (two 128-bit loads, one Philox call, 128-bit store of the int16 mantissas).
 template <int MODE, int PLANES, bool FAST>
@@ -578,7 +580,7 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
     if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
     __syncthreads();
     const int sh = MODE == 3 ? 0 : 16 - p.m;                  // wide modes: the views hold the top p.m bits
-    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, tv, tid);
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, p.qmax, tv, tid);
 }
 
 // ------------------------------------------------------------------------------ generic two-pass path

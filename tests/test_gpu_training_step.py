@@ -105,3 +105,47 @@ def test_small_classifier_trains_like_fp32(env):
     first, last_h, last_f = np.mean(hist_h[:5]), np.mean(hist_h[-10:]), np.mean(hist_f[-10:])
     assert last_h < 0.5 * first, (first, last_h)                     # it learns
     assert abs(last_h - last_f) <= 0.15 * max(last_f, 0.05), (last_h, last_f)   # and follows the FP32 curve
+
+
+def test_convolution_layer_products_match_the_oracle_and_fp32(env):
+    torch, hbfp_nn, hb = env
+    torch.manual_seed(2)
+    n, hw, c, f = 2, 16, 64, 64
+    layer = hbfp_nn.HbfpConv3x3(c, f, mant_bits=8, pixel_block=64)
+    x = torch.randn(n, hw, hw, c, device="cuda").relu().requires_grad_(True)
+    y = layer(x)
+    dy = torch.randn(n, hw, hw, f, device="cuda") * 1e-2
+    y.backward(dy)
+    assert hb.device_status() == 0
+    t = c
+    q16, g16 = layer.wide.mant.cpu().numpy(), layer.wide.exps.cpu().numpy()
+    s16 = np.repeat(g16, t, axis=0)[: 9 * c, :]
+    qm, sm = oracle.wide_narrow(q16, s16, 8)
+    grid = sm[::t, :]
+    X, dY = x.detach().cpu().numpy(), dy.cpu().numpy().reshape(n * hw * hw, f)
+    cols = oracle.im2col(X, 3, 3, 1)
+    fa = dict(mant_bits=8, block=c, rounding=0, seed=0)
+    # forward
+    qx, sx = oracle.quantize(cols, 1, ofmt(fa))
+    ref = oracle.gemm(qx, sx, np.ascontiguousarray(qm.T), np.ascontiguousarray(np.repeat(grid.T, t, axis=0)[:f, :]), t)
+    Y = y.detach().cpu().numpy().reshape(n * hw * hw, f)
+    assert (np.abs(Y.astype(np.float64) - ref["c_ref"]) <= TOL * ref["a_mag"] + 1e-12).all()
+    # backward-weight
+    fb = dict(mant_bits=8, block=64, rounding=0, seed=0)
+    ref = oracle.hbfp_gemm(1, 0, cols, dY, ofmt(fb), ofmt(fb))
+    assert (np.abs(layer.weight.grad.cpu().numpy().astype(np.float64) - ref["c_ref"]) <= TOL * ref["a_mag"]).all()
+    # backward-data: the GEMM against the oracle, the scatter against torch's own convolution gradient
+    qd, sd = oracle.quantize(dY, 1, ofmt(fa))
+    ref = oracle.gemm(qd, sd, qm, sm, t)                         # gradient of the im2col matrix [pixels][9 c]
+    dcols = ref["c_ref"].reshape(n, hw, hw, 3, 3, c)
+    dxp = np.zeros((n, hw + 2, hw + 2, c))
+    for i in range(3):
+        for j in range(3):
+            dxp[:, i:i + hw, j:j + hw, :] += dcols[:, :, :, i, j, :]
+    dx_ref = dxp[:, 1:hw + 1, 1:hw + 1, :]
+    assert np.allclose(x.grad.cpu().numpy(), dx_ref, rtol=1e-4, atol=1e-6)
+    # and the whole layer stays close to the FP32 convolution it stands for
+    w4 = layer.weight.detach().view(3, 3, c, f).permute(3, 2, 0, 1).contiguous()          # [f][c][3][3]
+    y32 = torch.nn.functional.conv2d(x.detach().permute(0, 3, 1, 2), w4, padding=1).permute(0, 2, 3, 1)
+    rel = (y.detach() - y32).norm() / y32.norm()
+    assert float(rel) < 2e-2

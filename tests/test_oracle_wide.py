@@ -63,21 +63,44 @@ def test_one_exponent_per_tile_of_the_stored_matrix():
 
 
 @pytest.mark.parametrize("m", [4, 8, 12, 16])
-def test_narrow_copy_is_the_floor_of_the_wide_value_on_the_narrow_grid(m):
+def test_narrow_copy_is_the_wide_value_rounded_to_the_narrow_grid(m):
     rng = np.random.default_rng(m)
     q16 = rng.integers(-32767, 32768, size=(40, 50)).astype(np.int16)
-    q16[0, :6] = [-1, 0, 1, -32767, 32767, -(1 << (16 - m))]
+    half = (1 << (16 - m)) >> 1
+    q16[0, :8] = [-1, 0, 1, -32767, 32767, -(1 << (16 - m)), half, -half]
     s16 = rng.integers(-63, 100, size=(40, 3)).astype(np.int8)
     qm, sm = oracle.wide_narrow(q16, s16, m)
     assert np.array_equal(sm.astype(int), s16.astype(int) + (16 - m))
+    qmax = (1 << (m - 1)) - 1
     for i in range(0, 40, 7):
         for j in range(50):
             wide = Fraction(int(q16[i, j])) * Fraction(2) ** int(s16[i, 0])
             step = Fraction(2) ** int(sm[i, 0])
             narrow = Fraction(int(qm[i, j])) * step
-            assert narrow <= wide < narrow + step                    # a floor: never above, less than one ULP below
-    assert int(qm[0, 0]) == -1                                       # -1 floors to -1, it does not truncate to 0
-    assert -(1 << (m - 1)) <= int(qm.min()) and int(qm.max()) <= (1 << (m - 1)) - 1
+            if abs(int(qm[i, j])) < qmax:
+                assert -step / 2 <= wide - narrow < step / 2         # nearest point of the grid, ties upward
+            else:
+                assert abs(wide - narrow) < step                     # saturated at the top of the range
+    if m < 15:
+        assert int(qm[0, 0]) == 0 and int(qm[0, 2]) == 0             # +-1 of the wide grid round to 0 ...
+    if m < 16:
+        assert int(qm[0, 6]) == 1 and int(qm[0, 7]) == 0             # ... and exact halves go upward
+    else:
+        assert np.array_equal(qm, q16)                               # sixteen bits: the copy is the mantissa itself
+    assert -qmax <= int(qm.min()) and int(qm.max()) <= qmax          # the symmetric range of every mantissa
+
+
+@pytest.mark.parametrize("m", [8, 12])
+def test_narrow_copy_has_no_systematic_offset(m):
+    # truncating the mantissa would leave every weight half a narrow ULP low; rounded, the mean error over
+    # many weights is a small fraction of an ULP
+    rng = np.random.default_rng(20 + m)
+    q16 = rng.integers(-30000, 30001, size=(200, 500)).astype(np.int16)
+    s16 = np.zeros((200, 1), dtype=np.int8)
+    qm, _ = oracle.wide_narrow(q16, s16, m)
+    ulp = 1 << (16 - m)
+    err = qm.astype(np.float64) * ulp - q16
+    assert abs(err.mean()) < 0.04 * ulp and np.abs(err).max() <= ulp / 2      # (ties upward: +1/2 of a wide unit)
 
 
 @pytest.mark.parametrize("m", [8, 12])
