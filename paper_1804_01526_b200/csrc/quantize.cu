@@ -369,12 +369,11 @@ struct TileViews {
 };
 
 // qt rows have a pitch of tp + 2 halfwords, so that the column reads of view c0 spread over the banks.
-// sh: the views take the top bits of wide storage: the mantissa plus half a narrow unit, shifted down by sh
-// bits (arithmetic) and clamped to the symmetric range, i.e. rounded to nearest; sh = 0 copies.
+// sh: the views take the top bits of the words in qt (an arithmetic shift by sh bits); for wide storage qt
+// holds the stored words, i.e. the mantissas plus half a narrow unit (see tile_kernel); sh = 0 copies.
 template <int PLANES>
 __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int hi, int wj, int64_t i0, int64_t j0,
-                                                 int64_t u, int64_t v, int s, int sh, int qmax, const TileViews& tv, int tid) {
-    const int half = sh > 0 ? 1 << (sh - 1) : 0;
+                                                 int64_t u, int64_t v, int s, int sh, const TileViews& tv, int tid) {
     const int qp = tp + 2;
     const int lg = 31 - __clz(tp >> 2), gmask = (tp >> 2) - 1;       // tp is 32, 64 or 128
     int8_t* const mant_c0 = tv.mant_c0; int8_t* const mant_c1 = tv.mant_c1;
@@ -387,7 +386,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = clampq((qt[ii * qp + g + j] + half) >> sh, qmax);
+            const int q = qt[ii * qp + g + j] >> sh;
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -402,7 +401,7 @@ __device__ __forceinline__ void write_tile_views(const int16_t* qt, int tp, int 
         uint32_t h = 0, l = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const int q = clampq((qt[(g + j) * qp + jj] + half) >> sh, qmax);
+            const int q = qt[(g + j) * qp + jj] >> sh;
             if (PLANES == 1) h |= (uint32_t)(q & 0xff) << (8 * j);
             else { h |= (uint32_t)((q >> 4) & 0xff) << (8 * j); l |= (uint32_t)(q & 15) << (8 * j); }
         }
@@ -467,6 +466,16 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
     const int hi = (int)min((int64_t)t, d0 - i0), wj = (int)min((int64_t)t, d1 - j0);
     const int G = wj >> 3;                              // FAST: groups of eight per tile row
     const int wbits = MODE == 3 ? p.m : 16, wqmax = MODE == 3 ? p.qmax : 32767;
+    // Wide modes: qt holds the stored word the views are cut from: the mantissa plus half a narrow unit,
+    // held inside the range whose top bits stay within +-qmax (so the shift alone rounds to nearest and
+    // saturates symmetrically). MODE 3 copies (sh = 0).
+    const int sh = MODE == 3 ? 0 : 16 - p.m;
+    const int half = sh > 0 ? 1 << (sh - 1) : 0;
+    const int w_hi = ((p.qmax + 1) << sh) - half - 1, w_lo = -(p.qmax << sh) - half;
+    const uint32_t w_hi2 = ((uint32_t)w_hi & 0xFFFFu) * 0x10001u, w_lo2 = ((uint32_t)w_lo & 0xFFFFu) * 0x10001u;
+    const uint32_t half2 = (uint32_t)half * 0x10001u;
+    auto stored_pair = [&](uint32_t h) { return MODE == 3 ? h : __vadd2(__vmaxs2(__vmins2(h, w_hi2), w_lo2), half2); };
+    auto stored_one = [&](int q) { return MODE == 3 ? q : max(w_lo, min(w_hi, q)) + half; };
     for (int e = tid; e < tp * qp / 2; e += 256) reinterpret_cast<uint32_t*>(qt)[e] = 0;
     int s;
     if (MODE == 2) {
@@ -477,11 +486,11 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
                 const int ii = item / G, gj = item - ii * G;
                 const uint4 q8 = *reinterpret_cast<const uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj);
                 uint32_t* dst = reinterpret_cast<uint32_t*>(qt + ii * qp + 8 * gj);
-                dst[0] = q8.x; dst[1] = q8.y; dst[2] = q8.z; dst[3] = q8.w;
+                dst[0] = stored_pair(q8.x); dst[1] = stored_pair(q8.y); dst[2] = stored_pair(q8.z); dst[3] = stored_pair(q8.w);
             }
         } else {
             for (int ii = wrow; ii < hi; ii += 8)
-                for (int jj = lane; jj < wj; jj += 32) qt[ii * qp + jj] = wide[(i0 + ii) * d1 + j0 + jj];
+                for (int jj = lane; jj < wj; jj += 32) qt[ii * qp + jj] = (int16_t)stored_one(wide[(i0 + ii) * d1 + j0 + jj]);
         }
     } else {
         const float old_scale = MODE == 1 ? pow2f(grid[u * grid_ld + v]) : 0.f;
@@ -560,7 +569,7 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
                     }
                 }
                 uint32_t* dst = reinterpret_cast<uint32_t*>(qt + ii * qp + 8 * gj);
-                dst[0] = h[0]; dst[1] = h[1]; dst[2] = h[2]; dst[3] = h[3];
+                dst[0] = stored_pair(h[0]); dst[1] = stored_pair(h[1]); dst[2] = stored_pair(h[2]); dst[3] = stored_pair(h[3]);
                 if (MODE != 3) *reinterpret_cast<uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj) = make_uint4(h[0], h[1], h[2], h[3]);
             }
         } else {
@@ -572,15 +581,14 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
                     if (MODE == 3) q = quantize_one(val, s, p, L);
                     else if (p.rounding == 0) q = round_rne(val, s, 32767);
                     else q = round_sr_wide(val, s, draw_of_element(p, L));
-                    qt[ii * qp + jj] = (int16_t)q;
+                    qt[ii * qp + jj] = (int16_t)stored_one(q);
                     if (MODE != 3) wide[(i0 + ii) * d1 + j0 + jj] = (int16_t)q;
                 }
         }
     }
     if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
     __syncthreads();
-    const int sh = MODE == 3 ? 0 : 16 - p.m;                  // wide modes: the views hold the top p.m bits
-    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, p.qmax, tv, tid);
+    write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, tv, tid);
 }
 
 // ------------------------------------------------------------------------------ generic two-pass path
