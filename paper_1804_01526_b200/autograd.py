@@ -1,4 +1,4 @@
-"""A dense layer whose three GEMMs run in block floating point (Sec. 4.1, Sec. 5.1).
+"""A dense layer and a 3 x 3 convolution whose three GEMMs run in block floating point (Sec. 4.1, Sec. 5.1).
 
 The paper simulates HBFP by redefining PyTorch's linear module with ``autograd.Function``: the
 forward product ``Y = X W``, the backward-data product ``dX = dY W^T`` and the backward-weight
@@ -16,6 +16,9 @@ no arithmetic of its own:
 
 Stochastic rounding draws are keyed by (seed + step, stream id, element index): a layer takes three
 consecutive stream ids (X, W, dY) from ``stream_id``.
+
+``HbfpConv3x3`` does the same for a convolution on channels-last activations, on the two operands the
+library builds without an FP32 im2col matrix (``hbfp_im2col_packed``, ``hbfp_im2col_packed_t``).
 """
 from __future__ import annotations
 
