@@ -69,7 +69,8 @@ typedef enum hbfp_status {
     HBFP_ERR_WORKSPACE = 4,   /* workspace pointer null or smaller than the query returned   */
     HBFP_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor map, ...)  */
     HBFP_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (see hbfp_device_status) */
-    HBFP_ERR_STATIC_LIMIT = 7 /* hbfp_gemm_static: the problem needs more than the built-in scratch */
+    HBFP_ERR_STATIC_LIMIT = 7, /* hbfp_gemm_static: the problem needs more than the built-in scratch */
+    HBFP_ERR_EXPONENT_RANGE = 8 /* hbfp_device_status: a tensor-core GEMM met block exponents outside its exact range */
 } hbfp_status;
 
 #define HBFP_ROUND_NEAREST_EVEN 0
@@ -241,8 +242,14 @@ HBFP_API int hbfp_gemm_q_workspace(int64_t M, int64_t N, int64_t K, const hbfp_o
  * (1,0). Without split-K the blocks are accumulated in ascending order with one FP32 rounding
  * each; with split-K (chosen for small C and long K) each split does so and the splits are
  * summed in ascending order. Exactness of the scaled FP32 accumulation needs sA + sB in
- * [-126, 127] (else the true product is outside binary32) and, on the tensor-core path,
- * sA <= 103 (|A| < 2^110 at 8-bit mantissas). */
+ * [-126, 127] (else the true product is outside binary32). The tensor-core kernels split the scale
+ * 2^(sA + sB) into two factors and need more: the paired-SM kernel chooses the split per K-block and
+ * 128-row tile and fails only when that tile's row exponents span more than 104 within one block
+ * (or the products leave binary32); the single-SM kernel's biased path needs sA <= 103 (|A| < 2^110
+ * at 8-bit mantissas). A kernel that meets exponents outside its range does not depart silently: it
+ * records a code in the device status word (hbfp_device_status then returns
+ * HBFP_ERR_EXPONENT_RANGE) and the values of C it wrote for that call are unspecified;
+ * HBFP_GEMM_FORCE_SIMT computes the same product without the restriction. */
 HBFP_API int hbfp_gemm(int transA, int transB, int64_t M, int64_t N, int64_t K, const float* A,
                        int64_t lda, const float* B, int64_t ldb, float* C, int64_t ldc,
                        const hbfp_format* fmtA, const hbfp_format* fmtB, void* workspace,
@@ -288,8 +295,10 @@ HBFP_API int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbf
                                       void* stream);
 
 /* Synchronises `stream`, then returns and clears the device-side status word of the current
- * device in *status (host int): 0, or a code recorded by a kernel whose bounded wait on a
- * barrier expired (the kernel then abandons its work and exits; HBFP_ERR_TIMEOUT is returned). */
+ * device in *status (host int): 0, or a code recorded by a kernel. Codes below 900: a bounded wait
+ * on a barrier expired (the kernel then abandons its work and exits; HBFP_ERR_TIMEOUT is returned).
+ * Codes 900-999: a tensor-core GEMM met block exponents outside the range in which its scaled
+ * accumulation is exact (see hbfp_gemm; HBFP_ERR_EXPONENT_RANGE is returned). */
 HBFP_API int hbfp_device_status(void* stream, int32_t* status);
 
 #ifdef __cplusplus

@@ -18,7 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("HBFP_LIBRARY") or os.path.join(_HERE, "libhbfp.so")
 
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT,
- ERR_STATIC_LIMIT) = range(8)
+ ERR_STATIC_LIMIT, ERR_EXPONENT_RANGE) = range(9)
 STATIC_WORKSPACE_BYTES = 16 << 20
 GEMM_AUTO, GEMM_FORCE_SIMT, GEMM_FORCE_TENSOR, GEMM_FORCE_TENSOR_1SM, GEMM_FORCE_TENSOR_2SM = 0, 1, 2, 3, 4
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
@@ -405,6 +405,12 @@ def gemm_block_partials(a: Packed, b: Packed, impl: int = GEMM_FORCE_SIMT) -> to
 
 def device_status() -> int:
     """hbfp_device_status: synchronises the current stream, returns and clears the status word."""
+    return device_status_rc()[1]
+
+
+def device_status_rc():
+    """hbfp_device_status as (return code, recorded code): (OK, 0), (ERR_TIMEOUT, code below 900) or
+    (ERR_EXPONENT_RANGE, code 900-999)."""
     v = ctypes.c_int32()
-    lib().hbfp_device_status(_stream(), ctypes.byref(v))
-    return v.value
+    rc = lib().hbfp_device_status(_stream(), ctypes.byref(v))
+    return rc, v.value

@@ -19,7 +19,8 @@ int read_clear_device_status(cudaStream_t st, int32_t* out) {
     HBFP_CUDA_OK(cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)));
     HBFP_CUDA_OK(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)));
     *out = v;
-    return v == 0 ? HBFP_OK : HBFP_ERR_TIMEOUT;
+    if (v == 0) return HBFP_OK;
+    return v >= 900 && v < 1000 ? HBFP_ERR_EXPONENT_RANGE : HBFP_ERR_TIMEOUT;
 }
 
 namespace {
@@ -158,6 +159,7 @@ const char* hbfp_status_string(int status) {
         case HBFP_ERR_WORKSPACE: return "workspace missing or too small";
         case HBFP_ERR_CUDA: return "CUDA call failed";
         case HBFP_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case HBFP_ERR_EXPONENT_RANGE: return "operand exponents outside the tensor-core path's exact range";
         case HBFP_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of hbfp_gemm_static";
         default: return "unknown status";
     }

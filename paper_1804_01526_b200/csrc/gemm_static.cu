@@ -9,6 +9,8 @@
 // the process exits. Nothing is allocated or freed by the call.
 #include "common.cuh"
 
+#include <atomic>
+
 namespace {
 
 // The built-in workspace. Every GPU that loads the library carries these bytes until exit.
@@ -16,18 +18,20 @@ static __device__ __align__(256) unsigned char g_static_workspace[HBFP_STATIC_WO
 
 // Device address of the array, per device. In host code the array's name only stands for the
 // symbol; the address a kernel can use has to be asked for, with that device current.
+// Host threads may make their first calls at the same time: the cache is atomic (they would all
+// store the same address).
 constexpr int kMaxDevices = 64;
-void* g_workspace_ptr[kMaxDevices] = {};
+std::atomic<void*> g_workspace_ptr[kMaxDevices];
 
 int static_workspace(void** out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return HBFP_ERR_CUDA;
-    if (!g_workspace_ptr[dev]) {
-        void* p = nullptr;
+    void* p = g_workspace_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return HBFP_ERR_CUDA;
-        g_workspace_ptr[dev] = p;
+        g_workspace_ptr[dev].store(p, std::memory_order_release);
     }
-    *out = g_workspace_ptr[dev];
+    *out = p;
     return HBFP_OK;
 }
 

@@ -39,13 +39,6 @@
 namespace hbfp {
 namespace {
 
-// Build-time probe for performance bisection (never set in the shipped library; results are
-// wrong when it is): 1 = rescale warps skip the tensor-memory reads and the math, 2 = no MMA is
-// issued, 4 = no mantissa tile is copied.
-#ifndef HBFP_TC_PROBE
-#define HBFP_TC_PROBE 0
-#endif
-
 constexpr int RESCALE_WARPS = 8;                   // two per sub-partition
 constexpr int COL_GROUPS = RESCALE_WARPS / 4;      // warps sharing a lane quarter split the columns
 // The control warps take the lowest warp ids: the issue logic favours them over the rescale
@@ -98,17 +91,7 @@ struct Problem {
     int64_t ldp;
     int32_t* P;             // optional dump of block sums [M][N][nkb]
     int32_t* status;
-    long long* trace;       // probe builds only: per-role timestamps of CTA 0
 };
-
-#if HBFP_TC_PROBE & 8
-#define HBFP_TRACE(role, idx)                                                        \
-    do {                                                                              \
-        if (p.trace && blockIdx.x == 0 && (idx) < 512) p.trace[(role) * 512 + (idx)] = clock64(); \
-    } while (0)
-#else
-#define HBFP_TRACE(role, idx) do { } while (0)
-#endif
 
 struct Work {
     int m0, nt, split;
@@ -211,7 +194,6 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
         for (int si = 0; ok && si < nst; ++si, ++it) {
             if (pre_full) pre_full = false;
             else if (!mbar_wait(a.full_bar + 8 * s, ph, a.abort_flag, p.status, 201)) { ok = false; break; }
-            HBFP_TRACE(2, it);
             tc_fence_after();
             const uint32_t ms = a.mant_base + s * C::MANT_STAGE;
             const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
@@ -227,7 +209,6 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
                         // the group was read (and, on the biased path, re-armed) by all rescale warps
                         if (pre_tempty) pre_tempty = false;
                         else if (!mbar_wait(a.tempty_bar + 8 * g, gph, a.abort_flag, p.status, 202)) { ok = false; break; }
-                        HBFP_TRACE(3, blk);
                         tc_fence_after();
                     }
                     const uint32_t d = a.tmem_base + g * PARTS * N_TILE;
@@ -250,8 +231,8 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
                         // biased path: always accumulate on top of the bias; else the first step of a block overwrites
                         const uint32_t acc = MAGIC ? 1u : (uint32_t)!(first && q == 0);
                         if (PLANES == 1) {
-                            if (!(HBFP_TC_PROBE & 2)) tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
-                        } else if (!(HBFP_TC_PROBE & 2)) {
+                            tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, acc);
+                        } else {
                             if (acc == 0u) {
                                 tc_mma_i8(d + N_TILE, a_lo + ko, b_hi + ko, idesc2, 0u);
                                 tc_mma_i8(d, a_hi + ko, b_hi + ko, idesc, 0u);
@@ -274,7 +255,6 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
             }
             left -= nb;
             tc_commit(a.empty_bar + 8 * s);        // the stage is free once these MMAs have read it
-            HBFP_TRACE(4, it);
             ring_next<STAGES>(s, ph);
         }
     }
@@ -356,16 +336,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     int kbyte = w.kb0 * p.bp;
                     for (int si = 0; si < nst; ++si, kbyte += STAGE_K, ++it) {
                         if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 101)) { ok = false; break; }
-                        HBFP_TRACE(0, it);
                         const uint32_t fb = full_bar + 8 * s;
-                        mbar_expect_tx(fb, (HBFP_TC_PROBE & 4) ? (uint32_t)C::EXP_STAGE : C::TX_BYTES);
+                        mbar_expect_tx(fb, C::TX_BYTES);
                         const uint32_t ms = mant_base + s * C::MANT_STAGE;
                         // A panels are re-used by every column tile of a group of 16 tile rows: ask L2 to keep
                         // them while the B panels stream past (marking B evict-first doubled the DRAM reads:
                         // the 16 CTAs that share a B panel do not read it at the same instant).
-                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d_hint(ms, &mapA0, kbyte, w.m0, fb, L2_EVICT_LAST);
-                        if (!(HBFP_TC_PROBE & 4)) tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
-                        if (PLANES == 2 && !(HBFP_TC_PROBE & 4)) {
+                        tma_load_2d_hint(ms, &mapA0, kbyte, w.m0, fb, L2_EVICT_LAST);
+                        tma_load_2d(ms + PLANES * C::A_BYTES, &mapB0, kbyte, n0, fb);
+                        if (PLANES == 2) {
                             tma_load_2d_hint(ms + C::A_BYTES, &mapA1, kbyte, w.m0, fb, L2_EVICT_LAST);
                             tma_load_2d(ms + 2 * C::A_BYTES + C::B_BYTES, &mapB1, kbyte, n0, fb);
                         }
@@ -400,7 +379,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             // b - 2 GROUPS, the last reader of the slot, and the barrier is back in the phase that the
             // arrival for b belongs to.
             uint32_t s = 0, ph = 0, g = 0, gph = 0, slot = 0, it = 0, blk = 0;
-            bool ok = true;
+            bool ok = true, out_of_range = false;
             for (int wi = blockIdx.x; ok && wi < total_work; wi += gridDim.x) {
                 const Work w = get_work(p, wi);
                 const int nst = stages_of(sh, w.nblk);
@@ -418,6 +397,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         else if (CPL == 4) cw[0] = *reinterpret_cast<const uint32_t*>(eB + jb * N_TILE + 4 * lane);
                         else cw[0] = *reinterpret_cast<const uint16_t*>(eB + jb * N_TILE + 2 * lane);
                         const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
+                        // the biased path forms 1.5 * 2^23 * 2^sA: finite up to sA = 103; beyond it the result
+                        // would be wrong, which is reported instead
+                        if (MAGIC) out_of_range |= __vmaxs4(ra, 0x67676767u) != 0x67676767u;
                         uint32_t cs[CPL];
 #pragma unroll
                         for (int i = 0; i < CPL; ++i) cs[i] = exp_to_field(cw[i >> 2], i & 3, MAGIC ? 127 : 0);
@@ -448,6 +430,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                     ring_next<STAGES>(s, ph);
                 }
             }
+            if (out_of_range) atomicCAS(p.status, 0, STATUS_EXPONENT_RANGE);
         }
     } else {
         // ------------------------------------------------------------------ rescale warps
@@ -492,13 +475,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             for (int kb = w.kb0; kb < w.kb0 + w.nblk; ++kb, ++blk) {
                 // one wait per block: the block sums are complete and the scale table is written
                 if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
-                if (lane == 0) HBFP_TRACE(17 + rwarp, blk);
                 tc_fence_after();
                 const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
                 const uint32_t* tab = tables + slot * C::TABLE_SLOT_WORDS + col0;
                 const uint32_t sa_u = tables[slot * C::TABLE_SLOT_WORDS + N_TILE + row];
-                if (HBFP_TC_PROBE & 1) {
-                } else if (MAGIC) {
+                if (MAGIC) {
                     // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
                     // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
                     const float sa_f = __uint_as_float(sa_u);
@@ -575,7 +556,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(tempty_bar + 8 * g);
-                    HBFP_TRACE(9 + rwarp, blk);
                 }
                 ring_next<GROUPS>(g, gph);
                 if (++slot == (uint32_t)TSLOTS) slot = 0;
@@ -655,10 +635,13 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
     if (rc) return rc;
     rc = make_map(&mEB, b.exps, b.L.rs, b.L.nkb, b.L.rs, N_TILE, 4, false);
     if (rc) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the device: set once per device, not once per process
+    static bool attr_set[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return HBFP_ERR_CUDA;
+    if (!attr_set[dev]) {
         HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
-        attr_set = true;
+        attr_set[dev] = true;
     }
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     const int grid = (int)(work < sm_count() ? work : sm_count());
@@ -667,11 +650,6 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
 }
 
 }  // namespace
-
-#if HBFP_TC_PROBE & 8
-long long* g_probe_trace = nullptr;
-extern "C" __attribute__((visibility("default"))) void hbfp_probe_set_trace(long long* ptr) { g_probe_trace = ptr; }
-#endif
 
 TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, const Layout& lb, int mant_bits_a,
                             int mant_bits_b) {
@@ -692,9 +670,6 @@ TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, c
         n_tile = 256;
         while (n_tile > 64 && (tiles_m * ((N + n_tile - 1) / n_tile) < SMS || N <= n_tile / 2)) n_tile /= 2;
     }
-#if HBFP_TC_PROBE
-    if (const char* e = getenv("HBFP_TC_NTILE")) n_tile = atoi(e);
-#endif
     const int64_t tiles = tiles_m * ((N + n_tile - 1) / n_tile);
     // split-K for small outputs with a long contraction: at least two stages per split, split
     // boundaries on stage boundaries.
@@ -736,9 +711,6 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     p.ldp = round_up(N, 4);
     p.P = P;
     p.status = device_status_word();
-#if HBFP_TC_PROBE & 8
-    p.trace = g_probe_trace;
-#endif
     if (!p.status) return HBFP_ERR_CUDA;
     if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
     int rc;

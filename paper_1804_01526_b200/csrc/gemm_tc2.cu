@@ -32,22 +32,21 @@ namespace {
 constexpr int N_TILE = 256;            // columns of the pair tile = accumulator columns per CTA
 constexpr int PAIR_M = 2 * TILE_M;     // rows of the pair tile
 constexpr int B_HALF = N_TILE / 2;     // B rows staged in each CTA
-// Rescale warps: 12 (three per sub-partition, 88 + 88 + 80 columns) or 8 (two, 128 columns each). The
-// rescale is bound by latencies, not by a pipe (FP32 pipe about half busy), so the third warp pays.
-#ifndef HBFP_TC2_RWARPS
-#define HBFP_TC2_RWARPS 12
-#endif
-constexpr int RESCALE_WARPS = HBFP_TC2_RWARPS;
+// Rescale warps: three per sub-partition (88 + 88 + 80 columns). The rescale is bound by latencies, not
+// by a pipe, so the third warp pays.
+constexpr int RESCALE_WARPS = 12;
 constexpr int CONTROL_WARPS = 4;
 constexpr int PRODUCER_WARP = 0, MMA_WARP = 1, TABLE_WARP = 2;
 constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
-// setmaxnreg totals must not exceed the launch allocation (384 threads x 168 or 512 x 128 registers)
-constexpr int REGS_RESCALE = RESCALE_WARPS == 8 ? 216 : 144;
-constexpr int REGS_CONTROL = RESCALE_WARPS == 8 ? 72 : 64;
-constexpr int REGS_LAUNCH = RESCALE_WARPS == 8 ? 168 : 128;
-static_assert(RESCALE_WARPS == 8 || RESCALE_WARPS == 12, "rescale warp count");
-static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= THREADS * REGS_LAUNCH - (RESCALE_WARPS == 8 ? 0 : 512), "register split");
+// setmaxnreg totals must not exceed the launch allocation (512 threads x 128 registers)
+constexpr int REGS_RESCALE = 144, REGS_CONTROL = 64, REGS_LAUNCH = 128;
+static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= THREADS * REGS_LAUNCH - 512, "register split");
 
+// Offset step (see rescale_loop): 32 products 255 * 255 per accumulator word. The scale of a block
+// is split 2^(sA + c) * 2^(sB + 149 - c); c = SHIFT suits sA in [-63, 41] and sB in [-63, 64], and the
+// table warp moves it per block when the exponents ask for it.
+constexpr int OFFSET = 32 * 255 * 255;
+constexpr int SHIFT = 86;
 constexpr int GROUPS = TMEM_COLS / N_TILE;                  // 2 accumulator groups
 constexpr int A_BYTES = TILE_M * STAGE_K, B_BYTES = B_HALF * STAGE_K;
 constexpr int MANT_STAGE = A_BYTES + B_BYTES;               // 32 KB per CTA and stage
@@ -57,22 +56,15 @@ constexpr int TSLOTS = 4;
 constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
 constexpr int TABLE_BYTES = 4 * TSLOTS * TABLE_SLOT_WORDS;
 constexpr int STAGES = 6;
-constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024;
+constexpr int ONES_BYTES = TILE_M * STAGE_K;   // 128 rows of 0xFF bytes: both operands of the offset step
+constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + ONES_BYTES + 1024;
 static_assert(SMEM <= 232448, "shared memory");
-
-// Build-time probe for performance bisection (never set in the shipped library; results are wrong
-// when it is): 1 = rescale warps skip the tensor-memory traffic and the math, 2 = no MMA is issued,
-// 4 = no mantissa tile is copied, 8 = cluster 0 records per-role timestamps.
-#ifndef HBFP_TC2_PROBE
-#define HBFP_TC2_PROBE 0
-#endif
 
 struct Problem {
     int64_t M, N;
     int64_t nkb;
     int bp;
     int tiles_m, tiles_n;   // pair tiles
-    long long* trace;       // probe builds only
     int splits;
     int64_t kb_per_split;
     float* C;
@@ -81,15 +73,6 @@ struct Problem {
     int64_t ldp;
     int32_t* status;
 };
-
-#if HBFP_TC2_PROBE & 8
-#define TC2_TRACE(role, idx)                                                                     \
-    do {                                                                                          \
-        if (p.trace && cluster == 0 && (idx) < 512) p.trace[((int)rank * 32 + (role)) * 512 + (idx)] = clock64(); \
-    } while (0)
-#else
-#define TC2_TRACE(role, idx) do { } while (0)
-#endif
 
 struct Work {
     int m0, n0, split;
@@ -151,6 +134,13 @@ __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
 }
 
+// Non-blocking look at a barrier phase.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+
 // Wait on a barrier that threads of the other CTA arrive on. What the arrivals order are tensor-memory
 // accesses, fenced with tcgen05.fence on both sides, so the default (CTA-scope) acquire is enough.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
@@ -164,6 +154,10 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   int32_t* status, int code) {
+    // The MMA thread has nothing else to do, and a thread that try_wait has put to sleep wakes up late
+    // (the kernel then settles in a mode 20 % slower): poll first, sleep only when that runs out.
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -176,13 +170,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity,
             return false;
         }
     }
-}
-
-// Non-blocking look at a barrier phase.
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
 }
 
 // Tile copy issued by one CTA of a pair; the completion bytes may be counted on a barrier of
@@ -210,11 +197,26 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint16_t cta_mask) 
 __device__ __forceinline__ constexpr uint32_t idesc_i8_pair() {
     return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
 }
+// The same shape with both operands taken as unsigned bytes (the offset step).
+__device__ __forceinline__ constexpr uint32_t idesc_u8_pair() {
+    return (2u << 4) | ((uint32_t)(N_TILE >> 3) << 17) | ((uint32_t)(PAIR_M >> 4) << 24);
+}
 
-// 2^e as binary32 bits, e = signed byte i of a packed word of four exponents.
-__device__ __forceinline__ uint32_t exp_to_scale(uint32_t packed, int i) {
+// 2^(e + sh) as binary32 bits, e = signed byte i of a packed word of four exponents.
+__device__ __forceinline__ uint32_t exp_to_scale(uint32_t packed, int i, int sh) {
     const int e = (int)(int8_t)(packed >> (8 * i));
-    return (uint32_t)(e + 127) << 23;
+    return (uint32_t)(e + 127 + sh) << 23;
+}
+// Smallest / largest of the four signed bytes of a word.
+__device__ __forceinline__ int byte_min(uint32_t w) {
+    w = __vmins4(w, w >> 16);
+    w = __vmins4(w, w >> 8);
+    return (int)(int8_t)w;
+}
+__device__ __forceinline__ int byte_max(uint32_t w) {
+    w = __vmaxs4(w, w >> 16);
+    w = __vmaxs4(w, w >> 8);
+    return (int)(int8_t)w;
 }
 
 // Advances a ring position (stage, accumulator group or table slot) and its phase bit.
@@ -235,83 +237,86 @@ struct RescaleArgs {
 
 // The loop of one rescale warp: rows = its lane quarter of this CTA's half tile, columns
 // [col0, col0 + NCOLS) of every accumulator group, read in chunks of CHW columns.
+//
+// Every block's first MMA step multiplies two constant operands (all bytes 255, taken as unsigned)
+// and overwrites the group with OFFSET = 32 * 255 * 255; the block's own steps accumulate on top, so
+// a word read back is X = OFFSET + P with 0 < X < 2^23 (|P| <= 127 * 127 * 128 < OFFSET): as a
+// binary32 pattern that is the subnormal X * 2^-149, exactly linear in P. Two packed FMAs finish Eq. 2:
+//   t   = fma(x, 2^(sA + c), -OFFSET * 2^(sA + c - 149)) = P * 2^(sA + c - 149)   (exact)
+//   acc = fma(t, 2^(sB + 149 - c), acc)                                        (one rounding)
+// with the block's split c chosen by the table warp.
+// Nothing has to be written back to tensor memory, and the group is handed back as soon as its last
+// chunk is in registers.
 template <int NCOLS, int CHW>
-__device__ __forceinline__ void rescale_loop(const Problem& p, const RescaleArgs& a, int col0, int rwarp) {
-    constexpr int NCHK = (HBFP_TC2_PROBE & 1) ? 0 : NCOLS / CHW;
+__device__ __forceinline__ void rescale_loop(const Problem& p, const RescaleArgs& a, int col0) {
+    constexpr int NCHK = NCOLS / CHW;
     static_assert(NCOLS % CHW == 0 && NCOLS % 8 == 0, "column split");
     const int lane = threadIdx.x & 31, quarter = (threadIdx.x >> 5) & 3;   // tensor-memory lanes follow warp % 4
     const int row = quarter * 32 + lane;                 // row of this CTA's half tile = tensor-memory lane
     const uint32_t lane_addr = a.tmem_base + ((uint32_t)(quarter * 32) << 16) + col0;
-    const int cluster = a.cluster;
-    const uint32_t rank = a.rank;
-    (void)cluster; (void)rank; (void)rwarp;
     uint64_t acc2[NCOLS / 2];                            // FP32 accumulators, two columns per entry
     {
-        uint32_t bias[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
-        for (int g = 0; g < GROUPS; ++g)
-#pragma unroll
-            for (int c8 = 0; c8 < NCOLS / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
-        tc_wait_st();
+        // One tensor-memory read before the loop (its result is not used). With it the loop below runs
+        // 6 % faster (n = 16384: 1 560 -> 1 680 TOP/s, four runs each): a code-generation effect, measured.
+        uint32_t z[8];
+        tc_ldn(lane_addr, z);
+        tc_wait_ld();
     }
-    // Read the bias back as one register tuple: a tuple that is born as such is passed to every
-    // re-arming store in place, while separately defined registers are copied into a fresh tuple
-    // for each store (one extra instruction per register and store).
-    uint32_t bias_t[CHW];
-    tc_ldn(lane_addr, bias_t);
-    tc_wait_ld();
-    // every accumulator group starts out free
     tc_fence_before();
     __syncwarp();
+    // every accumulator group starts out free
     if (lane == 0)
         for (int g = 0; g < GROUPS; ++g) mbar_arrive_remote(a.leader_tempty + 8 * g);
 
-    uint32_t g = 0, gph = 0, slot = 0, blk = 0;
+    uint32_t g = 0, gph = 0, slot = 0;
     bool ok = true;
     for (int wi = a.cluster; ok && wi < a.total_work; wi += a.nclusters) {
         const Work w = get_work(p, wi);
         const int64_t gi = w.m0 + (int)a.rank * TILE_M + row;
 #pragma unroll
         for (int c = 0; c < NCOLS / 2; ++c) acc2[c] = 0ull;
-        for (int kb = 0; kb < w.nblk; ++kb, ++blk) {
+        for (int kb = 0; kb < w.nblk; ++kb) {
             const uint32_t taddr = lane_addr + g * N_TILE;
             uint32_t v[2][CHW];
             // one wait per block: the block sums are complete and this CTA's scale table is written
-            if (!mbar_wait_warp(a.tfull_bar + 8 * g, gph, a.abort_flag, p.status, 312)) { ok = false; break; }
+            // (polled first: a warp that try_wait has put to sleep wakes up late)
+            {
+                bool hit = false;
+                for (int i = 0; i < 2048 && !hit; ++i) hit = mbar_test_wait(a.tfull_bar + 8 * g, gph);
+                if (!__all_sync(0xffffffffu, hit) && !mbar_wait_warp(a.tfull_bar + 8 * g, gph, a.abort_flag, p.status, 312)) { ok = false; break; }
+            }
             tc_fence_after();
-            if (NCHK) tc_ldn(taddr, v[0]);
-            if (lane == 0) TC2_TRACE(4 + (rwarp & 7), blk);
+            tc_ldn(taddr, v[0]);
             const uint32_t* tab = a.tables + slot * TABLE_SLOT_WORDS + col0;
-            // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
-            // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
-            const float sa_f = __uint_as_float(a.tables[slot * TABLE_SLOT_WORDS + N_TILE + row]);
-            const float ca_f = -12582912.0f * sa_f;
+            const float sa_f = __uint_as_float(a.tables[slot * TABLE_SLOT_WORDS + N_TILE + row]);   // 2^(sA + c)
+            const float ca_f = -__uint_as_float((uint32_t)OFFSET) * sa_f;               // -OFFSET * 2^(sA + c - 149)
             const uint64_t sa2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f));
             const uint64_t ca2 = pack2(__float_as_uint(ca_f), __float_as_uint(ca_f));
 #pragma unroll
             for (int ch = 0; ch < NCHK; ++ch) {
+                // the column scales of the chunk are requested before the wait for its block sums, so
+                // that their shared-memory latency passes during that wait
+                uint4 sbq[CHW / 4];
+#pragma unroll
+                for (int q = 0; q < CHW; q += 4) sbq[q / 4] = *reinterpret_cast<const uint4*>(tab + ch * CHW + q);
                 tc_wait_ld();
-                if (ch + 1 < NCHK) tc_ldn(taddr + (ch + 1) * CHW, v[(ch + 1) & 1]);
+                if (ch + 1 < NCHK) {
+                    tc_ldn(taddr + (ch + 1) * CHW, v[(ch + 1) & 1]);
+                } else {
+                    // the whole group is in registers: hand it back before the last chunk's arithmetic
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(a.leader_tempty + 8 * g);
+                }
                 const uint32_t(&x)[CHW] = v[ch & 1];
 #pragma unroll
                 for (int q = 0; q < CHW; q += 4) {
-                    const uint4 sb = *reinterpret_cast<const uint4*>(tab + ch * CHW + q);
+                    const uint4 sb = sbq[q / 4];
                     const uint64_t t01 = ffma2(pack2(x[q], x[q + 1]), sa2, ca2);
                     const uint64_t t23 = ffma2(pack2(x[q + 2], x[q + 3]), sa2, ca2);
                     acc2[(ch * CHW + q) / 2] = ffma2(t01, pack2(sb.x, sb.y), acc2[(ch * CHW + q) / 2]);
                     acc2[(ch * CHW + q) / 2 + 1] = ffma2(t23, pack2(sb.z, sb.w), acc2[(ch * CHW + q) / 2 + 1]);
                 }
-#if !(HBFP_TC2_PROBE & 16)
-                tc_stn(taddr + ch * CHW, bias_t);          // re-arm
-#endif
-            }
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_remote(a.leader_tempty + 8 * g);
-                TC2_TRACE(12 + (rwarp & 7), blk);
             }
             ring_next<GROUPS>(g, gph);
             slot = (slot + 1) & (TSLOTS - 1);
@@ -363,7 +368,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t exp_base = mant_base + STAGES * MANT_STAGE;           // STAGES x EXP_STAGE
     const uint32_t table_off = STAGES * (MANT_STAGE + EXP_STAGE);
     uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [slot][256 column scales | 128 row scales]
-    const uint32_t bar_off = table_off + TABLE_BYTES;
+    const uint32_t ones_off = table_off + TABLE_BYTES;                      // 1024-aligned: stages and tables are multiples of 1 KB
+    const uint32_t bar_off = ones_off + ONES_BYTES;
     const uint32_t bars = base + bar_off;
     const uint32_t full_bar = bars;                          // leader: mantissa tiles of both CTAs landed
     const uint32_t efull_bar = full_bar + 8 * STAGES;        // local: exponent slices landed
@@ -396,6 +402,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    for (int i = threadIdx.x; i < ONES_BYTES / 4; i += THREADS) reinterpret_cast<uint32_t*>(base_ptr + ones_off)[i] = 0xFFFFFFFFu;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes, read by the tensor core
     if (warp == MMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -422,13 +430,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     int kb = w.kb0, kbyte = w.kb0 * (128 >> LB);
                     for (int si = 0; si < nst; ++si, kb += BPS, kbyte += STAGE_K, ++it) {
                         if (!mbar_wait(empty_bar + 8 * s, ph ^ 1, abort_flag, p.status, 111)) { ok = false; break; }
-                        TC2_TRACE(0, it);
-                        if (rank == 0 && !(HBFP_TC2_PROBE & 4)) mbar_expect_tx(full_bar + 8 * s, 2u * MANT_STAGE);
-                        if (rank == 0 && (HBFP_TC2_PROBE & 4)) mbar_arrive(full_bar + 8 * s);
+                        if (rank == 0) mbar_expect_tx(full_bar + 8 * s, 2u * MANT_STAGE);
                         mbar_expect_tx(efull_bar + 8 * s, (uint32_t)EXP_STAGE);
                         const uint32_t ms = mant_base + s * MANT_STAGE;
-                        if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms, &mapA, kbyte, my_m, leader_full + 8 * s, L2_EVICT_LAST);
-                        if (!(HBFP_TC2_PROBE & 4)) tma_load_2d_pair(ms + A_BYTES, &mapB, kbyte, my_n, leader_full + 8 * s, L2_EVICT_NORMAL);
+                        tma_load_2d_pair(ms, &mapA, kbyte, my_m, leader_full + 8 * s, L2_EVICT_LAST);
+                        tma_load_2d_pair(ms + A_BYTES, &mapB, kbyte, my_n, leader_full + 8 * s, L2_EVICT_NORMAL);
                         const uint32_t es = exp_base + s * EXP_STAGE;
                         tma_load_2d(es, &mapEA, my_m, kb, efull_bar + 8 * s);
                         tma_load_2d(es + EXP_A, &mapEB, w.n0, kb, efull_bar + 8 * s);
@@ -449,6 +455,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             // -------------------------------------------------------------- MMA issuer (leader only)
             if (lane == 0 && rank == 0) {
                 constexpr uint32_t idesc = idesc_i8_pair();
+                const uint64_t ones_desc = smem_desc_sw128(base + ones_off);
                 uint32_t s = 0, ph = 0, g = 0, gph = 0, it = 0, blk = 0;
                 // The barriers the next MMAs will need are polled (without blocking) just before the last
                 // MMA of a block is issued, while earlier MMAs still occupy the tensor pipe; a barrier found
@@ -462,7 +469,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
                         if (pre_full) pre_full = false;
                         else if (!mbar_wait(full_bar + 8 * s, ph, abort_flag, p.status, 211)) { ok = false; break; }
-                        TC2_TRACE(1, it);
                         tc_fence_after();
                         const uint32_t ms = mant_base + s * MANT_STAGE;
                         const uint64_t a_desc = smem_desc_sw128(ms), b_desc = smem_desc_sw128(ms + A_BYTES);
@@ -470,12 +476,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 #pragma unroll
                         for (int jb = 0; jb < BPS; ++jb) {
                             if (jb < nb) {
-                                // the group was read and re-armed by the rescale warps of both CTAs
+                                // the group was read by the rescale warps of both CTAs
                                 if (pre_tempty) pre_tempty = false;
                                 else if (!mbar_wait_cluster(tempty_bar + 8 * g, gph, abort_flag, p.status, 212)) { ok = false; break; }
-                                TC2_TRACE(2, blk);
                                 tc_fence_after();
                                 const uint32_t d = tmem_base + g * N_TILE;
+                                // offset step: overwrites the group with 32 * 255 * 255 in every word
+                                tc_mma_i8_pair(d, ones_desc, ones_desc, idesc_u8_pair(), 0u);
 #pragma unroll
                                 for (int q = 0; q < SPB; ++q) {
                                     if (q == SPB - 1) {
@@ -490,10 +497,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                                         }
                                     }
                                     const uint64_t ko = (uint64_t)(2 * (jb * SPB + q));     // 32 bytes per step, in 16-byte units
-                                    if (!(HBFP_TC2_PROBE & 2)) tc_mma_i8_pair(d, a_desc + ko, b_desc + ko, idesc, 1u);   // on top of the bias
+                                    tc_mma_i8_pair(d, a_desc + ko, b_desc + ko, idesc, 1u);   // on top of the offset
                                 }
                                 tc_commit_pair(tfull_bar + 8 * g, 3);
-                                TC2_TRACE(3, blk);
                                 ring_next<GROUPS>(g, gph);
                                 ++blk;
                             }
@@ -512,14 +518,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             // issued only after every rescale warp had finished b - 4, the last reader of the slot, and
             // the barrier is back in the phase that the arrival for b belongs to.
             uint32_t s = 0, ph = 0, g = 0, gph = 0, slot = 0, it = 0, blk = 0;
-            bool ok = true;
+            bool ok = true, out_of_range = false;
             for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
                 const Work w = get_work(p, wi);
                 const int nst = (w.nblk + BPS - 1) >> LB;
                 int left = w.nblk;
                 for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
                     if (!mbar_wait_warp(efull_bar + 8 * s, ph, abort_flag, p.status, 411)) { ok = false; break; }
-                    if (lane == 0) TC2_TRACE(20, it);
                     const unsigned char* eA = base_ptr + (exp_base - base) + s * EXP_STAGE;
                     const unsigned char* eB = eA + EXP_A;
 #pragma unroll
@@ -528,19 +533,27 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                             // this lane's 8 column exponents and 4 row exponents of block jb of the stage
                             const uint2 cb = *reinterpret_cast<const uint2*>(eB + jb * N_TILE + 8 * lane);
                             const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
+                            // The split of the scales (rescale_loop): c = SHIFT wherever the block's exponents allow
+                            // it, otherwise moved into the window in which every factor and every P * 2^(sA + c - 149)
+                            // is a normal binary32 number. The window is empty only when the row exponents of the
+                            // block span more than 104 or the true products leave binary32: reported, not computed.
+                            const int a_lo = __reduce_min_sync(0xffffffffu, byte_min(ra)), a_hi = __reduce_max_sync(0xffffffffu, byte_max(ra));
+                            const int b_lo = __reduce_min_sync(0xffffffffu, byte_min(__vmins4(cb.x, cb.y)));
+                            const int b_hi = __reduce_max_sync(0xffffffffu, byte_max(__vmaxs4(cb.x, cb.y)));
+                            const int c_lo = max(23 - a_lo, 22 + b_hi), c_hi = min(127 - a_hi, 275 + b_lo);
+                            out_of_range |= c_lo > c_hi;
+                            const int c = min(max(SHIFT, c_lo), c_hi);
                             uint4 c0, c1, r0;
-                            c0.x = exp_to_scale(cb.x, 0); c0.y = exp_to_scale(cb.x, 1); c0.z = exp_to_scale(cb.x, 2); c0.w = exp_to_scale(cb.x, 3);
-                            c1.x = exp_to_scale(cb.y, 0); c1.y = exp_to_scale(cb.y, 1); c1.z = exp_to_scale(cb.y, 2); c1.w = exp_to_scale(cb.y, 3);
-                            r0.x = exp_to_scale(ra, 0); r0.y = exp_to_scale(ra, 1); r0.z = exp_to_scale(ra, 2); r0.w = exp_to_scale(ra, 3);
+                            c0.x = exp_to_scale(cb.x, 0, 149 - c); c0.y = exp_to_scale(cb.x, 1, 149 - c); c0.z = exp_to_scale(cb.x, 2, 149 - c); c0.w = exp_to_scale(cb.x, 3, 149 - c);
+                            c1.x = exp_to_scale(cb.y, 0, 149 - c); c1.y = exp_to_scale(cb.y, 1, 149 - c); c1.z = exp_to_scale(cb.y, 2, 149 - c); c1.w = exp_to_scale(cb.y, 3, 149 - c);
+                            r0.x = exp_to_scale(ra, 0, c); r0.y = exp_to_scale(ra, 1, c); r0.z = exp_to_scale(ra, 2, c); r0.w = exp_to_scale(ra, 3, c);
                             if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
-                            if (lane == 0) TC2_TRACE(21, blk);
                             uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
                             *reinterpret_cast<uint4*>(tb + 8 * lane) = c0;
                             *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
                             *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
                             __syncwarp();
                             if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
-                            if (lane == 0) TC2_TRACE(22, blk);
                             ring_next<GROUPS>(g, gph);
                             slot = (slot + 1) & (TSLOTS - 1);
                             ++blk;
@@ -548,22 +561,18 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_bar + 8 * s);      // the exponent slices are consumed
-                    if (lane == 0) TC2_TRACE(25, it);
                     ring_next<STAGES>(s, ph);
                 }
             }
+            if (out_of_range) atomicCAS(p.status, 0, STATUS_EXPONENT_RANGE);
         }
     } else {
         // ------------------------------------------------------------------ rescale warps (both CTAs)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_RESCALE));
         const RescaleArgs ra{tfull_bar, map_to_rank(tempty_bar, 0), tmem_base, tables, total_work, cluster, nclusters, rank, abort_flag};
         const int rwarp = warp - CONTROL_WARPS, part = rwarp >> 2;     // warps that share a lane quarter split the columns
-#if HBFP_TC2_RWARPS == 12
-        if (part == 2) rescale_loop<80, 8>(p, ra, 176, rwarp);
-        else rescale_loop<88, 8>(p, ra, part * 88, rwarp);
-#else
-        rescale_loop<128, 16>(p, ra, part * 128, rwarp);
-#endif
+        if (part == 2) rescale_loop<80, 8>(p, ra, 176);
+        else rescale_loop<88, 8>(p, ra, part * 88);
     }
 
     // ------------------------------------------------------------------ teardown
@@ -577,9 +586,20 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     }
 }
 
+// Largest number of co-resident clusters on the current device (0: not known yet, -1: the query failed).
 int max_clusters() {
-    static int n = 0;
-    if (!n) {
+    static int n[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return -1;
+    if (!n[dev]) {
+        // the attribute belongs to the device: set once per device, before the occupancy query that needs it
+        if (cudaFuncSetAttribute(gemm_tc2_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gemm_tc2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess ||
+            cudaFuncSetAttribute(gemm_tc2_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) != cudaSuccess) {
+            cudaGetLastError();
+            n[dev] = -1;
+            return -1;
+        }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2 * 148, 1, 1);
         cfg.blockDim = dim3(THREADS, 1, 1);
@@ -589,27 +609,22 @@ int max_clusters() {
             cudaGetLastError();
             c = -1;
         }
-        n = c;
+        n[dev] = c;
     }
-    return n;
+    return n[dev];
 }
 
 }  // namespace
-
-#if HBFP_TC2_PROBE & 8
-long long* g_probe_trace2 = nullptr;
-extern "C" __attribute__((visibility("default"))) void hbfp_probe_set_trace2(long long* ptr) { g_probe_trace2 = ptr; }
-#endif
 
 bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, const TensorPlan& plan) {
     if (a.L.planes != 1 || b.L.planes != 1) return false;
     if (a.L.bp > 128 || plan.n_tile != 256) return false;
     const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
-    if (qa * qb * a.L.b >= (1ll << 22)) return false;        // the biased accumulator needs |P| < 2^22
+    if (qa * qb * a.L.b >= OFFSET) return false;             // the offset keeps OFFSET + P positive
     if (plan.splits != 1) return false;
     // enough pair tiles to occupy every SM pair
     const int64_t tiles = ((M + PAIR_M - 1) / PAIR_M) * ((N + N_TILE - 1) / N_TILE);
-    return tiles >= 74;
+    return tiles >= 74 && max_clusters() >= 1;
 }
 
 int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed& b, float* Cout, int64_t ldc,
@@ -630,9 +645,6 @@ int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed&
     p.status = device_status_word();
     if (!p.status) return HBFP_ERR_CUDA;
     if (p.splits > 1 && !partial) return HBFP_ERR_WORKSPACE;
-#if HBFP_TC2_PROBE & 8
-    p.trace = g_probe_trace2;
-#endif
     CUtensorMap mA, mB, mEA, mEB;
     int rc;
     rc = make_map(&mA, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
@@ -643,13 +655,6 @@ int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed&
     if (rc) return rc;
     rc = make_map(&mEB, b.exps, b.L.rs, b.L.nkb, b.L.rs, N_TILE, 4, false);
     if (rc) return rc;
-    static bool attr_set = false;
-    if (!attr_set) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc2_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-        attr_set = true;
-    }
     const int clusters_max = max_clusters();
     if (clusters_max < 1) return HBFP_ERR_UNSUPPORTED;
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;

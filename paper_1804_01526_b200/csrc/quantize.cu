@@ -1143,13 +1143,17 @@ int launch_col_tma(const float* x, int64_t K, int64_t rows, int64_t ld, const QP
     }
     constexpr int smem = 1024 + PLANES * QC_OUT_BYTES + QC_STAGES * QC_IN_BYTES + (SR ? QC_ROWS * QC_COLS * 2 : 0) +
                          4 * QC_COLS * 4 + 64;
-    static int ctas_per_sm = 0;
-    if (!ctas_per_sm) {
+    // attribute and occupancy belong to the device: cached per device ordinal
+    static int ctas_per_sm_dev[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return HBFP_ERR_CUDA;
+    if (!ctas_per_sm_dev[dev]) {
         HBFP_CUDA_OK(cudaFuncSetAttribute(quant_col_tma<PLANES, LB, SR>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         int nb = 0;
         HBFP_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, quant_col_tma<PLANES, LB, SR>, QC_THREADS, smem));
-        ctas_per_sm = nb > 0 ? nb : 1;
+        ctas_per_sm_dev[dev] = nb > 0 ? nb : 1;
     }
+    const int ctas_per_sm = ctas_per_sm_dev[dev];
     int32_t* status = device_status_word();
     if (!status) return HBFP_ERR_CUDA;
     const int64_t tiles_n = (rows + QC_COLS - 1) / QC_COLS, tiles_k = L.kst / QC_ROWS;

@@ -8,11 +8,6 @@
 
 #include "common.cuh"
 
-// 1: poll barriers with the non-suspending test_wait instead of try_wait.
-#ifndef HBFP_TC_TESTWAIT
-#define HBFP_TC_TESTWAIT 0
-#endif
-
 namespace hbfp {
 namespace {
 
@@ -20,6 +15,7 @@ constexpr int TILE_M = 128;
 constexpr int STAGE_K = 128;          // bytes of K per stage (= one 128B swizzle row)
 constexpr uint32_t BIAS_BITS = 0x4B400000u;     // binary32 1.5 * 2^23
 constexpr int TMEM_COLS = 512;
+constexpr int STATUS_EXPONENT_RANGE = 901;       // device status: an operand exponent outside the fast path's range
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s at 2 GHz
 constexpr uint32_t WAIT_HINT_NS = 200000u;              // one try_wait may sleep this long; the loop around it is bounded
 
@@ -40,13 +36,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-#if HBFP_TC_TESTWAIT
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#else
         // the suspend-time hint lets a waiting thread sleep in hardware until the phase completes
         // instead of spinning on issue slots that the arithmetic warps of its sub-partition need
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
     return ok != 0;
@@ -241,14 +233,20 @@ int make_map(CUtensorMap* m, const void* ptr, uint64_t inner, uint64_t outer, ui
     return r == CUDA_SUCCESS ? HBFP_OK : HBFP_ERR_CUDA;
 }
 
+// Per-device caches are arrays indexed by the device ordinal: a process may use several GPUs.
+constexpr int MAX_DEVICES = 64;
+int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+    return dev;
+}
+
 int sm_count() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            n = 148;
-    }
-    return n;
+    static int n[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return 148;
+    if (!n[dev] && cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) n[dev] = 148;
+    return n[dev];
 }
 
 }  // namespace

@@ -263,3 +263,49 @@ def test_tensor_core_kernel_writes_outputs_of_any_width(hb, M, N, K):
     hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd), out=buf[:, 3:3 + N], flags=hb.GEMM_FORCE_TENSOR)
     out = buf.cpu().numpy()
     assert np.array_equal(out[:, 3:3 + N], C) and (out[:, :3] == -1).all() and (out[:, 3 + N:] == -1).all()
+
+
+def _range_case(hb, A, B, flag):
+    """GEMM of two FP32 matrices (8-bit mantissas, blocks of 128) on the kernel `flag` selects: returns
+    (status return code, result, oracle reference)."""
+    fd = dict(mant_bits=8, block=128)
+    ref = oracle.hbfp_gemm(0, 0, A, B, ofmt(fd), ofmt(fd, stream_id=1))
+    C = hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd, stream_id=1), flags=flag).cpu().numpy()
+    rc, code = hb.device_status_rc()
+    return rc, code, C, ref
+
+
+@pytest.mark.parametrize("kernel", ["1sm", "2sm"])
+def test_large_magnitudes_are_computed_or_reported_never_silently_wrong(hb, kernel):
+    """Operands far from 1: the tensor-core kernels factor the block scale 2^(sA + sB); outside the
+    range in which that is exact they must say so through the device status word."""
+    flag = hb.GEMM_FORCE_TENSOR_1SM if kernel == "1sm" else hb.GEMM_FORCE_TENSOR_2SM
+    M, N, K = 2304, 2304, 256            # 81 pair tiles: enough for the paired kernel
+    rng = np.random.default_rng(77)
+    B = wl.draw("normal", (K, N), seed=78)
+    # (1) |A| ~ 2^60, |B| ~ 1: inside binary32, outside a fixed split of the scale
+    A = (wl.draw("normal", (M, K), seed=79) * np.float32(2.0 ** 60)).astype(np.float32)
+    rc, code, C, ref = _range_case(hb, A, B, flag)
+    assert rc == hb.OK and code == 0
+    assert np.array_equal(C, ref["c_seq"])
+    # (2) |A| ~ 2^115: products are still finite with |B| ~ 2^-40
+    A2 = (wl.draw("normal", (M, K), seed=80) * np.float32(2.0 ** 115)).astype(np.float32)
+    B2 = (B * np.float32(2.0 ** -40)).astype(np.float32)
+    rc, code, C, ref = _range_case(hb, A2, B2, flag)
+    if rc == hb.OK:
+        assert np.array_equal(C, ref["c_seq"])
+    else:
+        assert rc == hb.ERR_EXPONENT_RANGE and 900 <= code < 1000
+    # (3) rows of one tile 140 binades apart: no split of the scale serves both
+    A3 = wl.draw("normal", (M, K), seed=81)
+    A3[0::2] *= np.float32(2.0 ** 70)
+    A3[1::2] *= np.float32(2.0 ** -70)
+    rc, code, C, ref = _range_case(hb, A3.astype(np.float32), B, flag)
+    if rc == hb.OK:
+        err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
+        assert (err <= TOL * ref["a_mag"]).all()
+    else:
+        assert rc == hb.ERR_EXPONENT_RANGE and 900 <= code < 1000
+    # the library is healthy afterwards
+    rc, code, C, ref = _range_case(hb, wl.draw("normal", (M, K), seed=82), B, flag)
+    assert rc == hb.OK and np.array_equal(C, ref["c_seq"])

@@ -6,8 +6,9 @@ Collected last on purpose: a run that stops at the first failure has then alread
 import numpy as np
 import pytest
 
+import oracle
 from paper_1804_01526_b200 import workloads as wl
-from tests.helpers import to_dev
+from tests.helpers import ofmt, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -28,20 +29,41 @@ CASES = [
 ]
 
 
+def _allocation_state():
+    """(requests torch's allocator has served so far, bytes it holds from the driver, bytes the driver has free)."""
+    import gc
+    import torch
+    gc.collect()                              # tensors of earlier tests that only a cycle keeps alive
+    torch.cuda.synchronize()
+    stats = torch.cuda.memory_stats()
+    return (stats["allocation.all.allocated"], stats["segment.all.allocated"], torch.cuda.memory_reserved(),
+            torch.cuda.mem_get_info()[0])
+
+
 @pytest.mark.parametrize("transA,transB,M,N,K,fd", CASES)
 def test_static_scratch_matches_workspace_entry_point_twice(hb, transA, transB, M, N, K, fd):
     import torch
-    A = to_dev(wl.draw("lognormal", (K, M) if transA else (M, K), seed=41))
-    B = to_dev(wl.draw("lognormal", (N, K) if transB else (K, N), seed=42))
+    A_host = wl.draw("lognormal", (K, M) if transA else (M, K), seed=41)
+    B_host = wl.draw("lognormal", (N, K) if transB else (K, N), seed=42)
+    A, B = to_dev(A_host), to_dev(B_host)
     fa, fb = hb.Format(**fd), hb.Format(**{**fd, "stream_id": 1})
     want = hb.gemm(transA, transB, A, B, fa, fb).cpu().numpy()
+    ref = oracle.hbfp_gemm(transA, transB, A_host, B_host, ofmt(fd), ofmt(fd, stream_id=1))
     out = torch.empty((M, N), dtype=torch.float32, device="cuda")
-    for _ in range(2):                       # the second call finds the first call's bytes in the scratch
+    for call in range(2):                    # the second call finds the first call's bytes in the scratch
         out.fill_(float("nan"))
-        got = hb.gemm_static(transA, transB, A, B, fa, fb, out=out).cpu().numpy()
+        if call == 1:                        # nothing is allocated: not through torch, not behind its back
+            before = _allocation_state()
+        got = hb.gemm_static(transA, transB, A, B, fa, fb, out=out)
+        if call == 1:
+            assert _allocation_state() == before
+        got = got.cpu().numpy()
         # same kernels in the same order on the same inputs: the tolerance of the GEMM tests
         # (1e-6 of accumulator magnitude) tightens to bit equality here
         assert np.array_equal(got, want)
+        # and against the oracle itself, within the tolerance the GEMM tests use
+        err = np.abs(got.astype(np.float64) - ref["c_ref"].astype(np.float64))
+        assert (err <= 1e-6 * ref["a_mag"]).all()
     assert hb.device_status() == 0
 
 
