@@ -34,9 +34,14 @@ METRIC = "bfp_gemm_effective_tops_quantize_plus_gemm"
 UNIT = "TOPS"
 INT8_OVER_BF16 = 2.0          # nominal dense int8 : bf16 tensor ratio (4.5 : 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (read + write) of one launch of the GEMM kernel at the default workload (n = 16384, m = 8,
-# b = 128), from the single-pass ncu capture summarised in profiles/bench_launch_list_n16384_m8_b128.md.
-GEMM_DRAM_TRAFFIC_BYTES = {(16384, 8, 128): 3970740224 + 1068051712}
+# DRAM bytes (read + write) of one launch of the GEMM kernel, by (kernel, n, mantissa bits, block), each
+# with the summary of the single-pass ncu capture it was read from. A workload without an entry reports
+# no traffic.
+GEMM_DRAM_TRAFFIC = {
+    ("gemm_tc2_kernel", 16384, 8, 128): {"bytes": 3970740224 + 1068051712,
+                                         "profile": "profiles/bench_launch_list_n16384_m8_b128.md"},
+}
+SUSTAINED_SECONDS = 2.5       # length of the back-to-back GEMM loop behind `gemm_sustained`
 
 
 def load_peaks():
@@ -317,6 +322,36 @@ def gpu_arm(args):
         replicas.shutdown(rep)
         return 0
 
+    # ---- which GEMM kernel the library launched for this workload (asked of the library, not re-derived)
+    hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
+    gemm_kernel = hb.last_gemm_kernel()
+
+    # ---- the GEMM back to back for a few seconds: what it does once the power cap has pulled the clock
+    # down (the timed region above is a burst of ~0.1 s). Device time by CUDA events, SM clock sampled
+    # during the loop; time x MHz compares the two regimes clock for clock.
+    sustained = None
+    if not args.no_sustained:
+        reps = max(10, int(SUSTAINED_SECONDS / max(t_gemm * 1e-3, 1e-6)))
+        sampler2 = ClockSampler(local)
+        sampler2.start()
+        time.sleep(0.25)
+        torch.cuda.synchronize()
+        tw0 = time.time()
+        s5, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s5.record()
+        for _ in range(reps):
+            hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
+        e5.record()
+        torch.cuda.synchronize()
+        tw1 = time.time()
+        clk2 = sampler2.stop(tw0 + 0.5 * (tw1 - tw0), tw1)      # second half of the loop: settled clocks
+        ms5 = s5.elapsed_time(e5) / reps
+        sustained = {"launches": reps, "seconds": (tw1 - tw0), "ms_per_launch": ms5, "tops": ops / (ms5 * 1e-3) / 1e12,
+                     "sm_mhz_median_second_half": clk2["sm_mhz"], "power_w_max": clk2.get("power_w_max"),
+                     "reasons": clk2["reasons"],
+                     "ms_x_mhz": ms5 * clk2["sm_mhz"] if clk2["sm_mhz"] else None,
+                     "burst_ms_x_mhz": t_gemm * clocks["sm_mhz"] if clocks.get("sm_mhz") else None}
+
     # ---- standalone quantiser on the 1 GiB tensor (the second half of the metric), rank 0 only
     quant = {}
     if n * n * 4 >= 2 ** 30 or args.quantize_line:
@@ -363,13 +398,12 @@ def gpu_arm(args):
     int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16
     gemm_tops = ops / (t_gemm * 1e-3) / 1e12
-    # the library takes the paired-SM kernel for one-plane operands with blocks up to 128, >= 74 tiles of
-    # 256 x 256 and at least 1 KiB of mantissas per row
-    paired = args.mant_bits <= 8 and 0 < args.block <= 128 and ((n + 255) // 256) ** 2 >= 74 and n >= 1024
-    roofline = {"bound": "tensor", "kernel": "gemm_tc2_kernel" if paired else "gemm_tc_kernel", "achieved": gemm_tops,
+    traffic = GEMM_DRAM_TRAFFIC.get((gemm_kernel, n, args.mant_bits, args.block))
+    roofline = {"bound": "tensor", "kernel": gemm_kernel, "achieved": gemm_tops,
                 "peak": int8_burst,
                 "unit": "TOP/s", "frac": gemm_tops / int8_burst,
-                "traffic": GEMM_DRAM_TRAFFIC_BYTES.get((n, args.mant_bits, args.block)),
+                "traffic": traffic["bytes"] if traffic else None,
+                "traffic_profile": traffic["profile"] if traffic else None,
                 "algorithmic_bytes": 2 * n * n * ((1 if args.mant_bits <= 8 else 2) + 1.0 / args.block) + 4 * n * n,
                 "peak_source": f"{peaks_kind} bf16 burst x {INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
                 "frac_of_sustained_peak": gemm_tops / int8_sust, "frac_of_nominal_4500": gemm_tops / 4500.0,
@@ -400,7 +434,7 @@ def gpu_arm(args):
                            "per panel) on 3 streams: copy-in, compute and copy-out overlap") if panels > 1
                           else "one hbfp_gemm call between the copies"},
            "gpu_launches": 3 * args.steps, "roofline": roofline, "cpu_baseline": cpu,
-           "breakdown": breakdown, "quantize_standalone": quant, "wide_storage": wide}
+           "breakdown": breakdown, "gemm_sustained": sustained, "quantize_standalone": quant, "wide_storage": wide}
     print(json.dumps(out), flush=True)
     replicas.shutdown(rep)
     return 0
@@ -418,6 +452,7 @@ def main():
     ap.add_argument("--rounding", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quantize-line", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the few-second back-to-back GEMM loop")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -110,8 +110,8 @@ HBFP_API int hbfp_packed_layout(int64_t rows, int64_t k, const hbfp_format* fmt,
 HBFP_API int hbfp_packed_sizes(int64_t rows, int64_t k, const hbfp_format* fmt, size_t* mant_bytes,
                                size_t* exp_bytes);
 
-/* FP32 -> BFP conversion (Sec. 4.1 "convert tensors to BFP before every dot product, using
- * the exponent of the largest tensor value"; Sec. 5.3 FP-to-BFP unit).
+/* FP32 -> BFP conversion, done ahead of each dot product with the shared exponent taken from the
+ * block's largest magnitude (Sec. 4.1; the FP-to-BFP unit of Sec. 5.3).
  * x: FP32 [d0][d1], row stride ld >= d1 (elements). Blocks run along contract_axis (1 = along
  * rows of x, 0 = down its columns). Output: packed operand with rows = the other extent and
  * k = the extent of contract_axis (so contract_axis 0 writes the transposed, contraction-major
@@ -164,6 +164,13 @@ HBFP_API int hbfp_wide_update(int16_t* wide, int8_t* wide_exps, const float* del
 HBFP_API int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1,
                               const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1,
                               int8_t* exps_c1, void* stream);
+
+/* Value of the wide copy as FP32 (Eq. 1): out[i][j] = wide[i][j] * 2^wide_exps[i/tile][j/tile], exact
+ * (16-bit mantissas fit binary32). out: FP32 [d0][d1], pitch ldo >= d1 (device). What the FP32 parts
+ * of training (the optimiser, regularisation: Sec. 4.1) see of the weights. Asynchronous on `stream`;
+ * HBFP_ERR_INVALID_ARG for null pointers, tile <= 0 or ldo < d1. */
+HBFP_API int hbfp_wide_dequantize(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1,
+                                  int32_t tile, float* out, int64_t ldo, void* stream);
 
 /* Convolution operand without the FP32 im2col matrix (the paper runs convolutions through the same
  * BFP dot products, Sec. 5.1). x is an activation tensor [n][h][w][c] (channels last) that was
@@ -294,12 +301,29 @@ HBFP_API int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbf
                                       const hbfp_operand* b, int32_t* P, uint32_t impl,
                                       void* stream);
 
+/* Host-only: name of the GEMM kernel that the calling thread's most recent hbfp_gemm, hbfp_gemm_q,
+ * hbfp_gemm_static or hbfp_gemm_block_partials call launched ("gemm_tc2_kernel": two SMs per 256 x 256
+ * tile; "gemm_tc_kernel": one SM per tile; "gemm_simt_kernel"), "" before the first launch. For
+ * measurement scripts that must name the kernel they timed (the paper has no counterpart). The
+ * string is static storage. */
+HBFP_API const char* hbfp_last_gemm_kernel(void);
+
 /* Synchronises `stream`, then returns and clears the device-side status word of the current
  * device in *status (host int): 0, or a code recorded by a kernel. Codes below 900: a bounded wait
  * on a barrier expired (the kernel then abandons its work and exits; HBFP_ERR_TIMEOUT is returned).
  * Codes 900-999: a tensor-core GEMM met block exponents outside the range in which its scaled
  * accumulation is exact (see hbfp_gemm; HBFP_ERR_EXPONENT_RANGE is returned). */
 HBFP_API int hbfp_device_status(void* stream, int32_t* status);
+
+/* Self-test of the bounded waits (the paper has no counterpart: failure behaviour of this
+ * library). Launches one warp that waits, with the same wait routine and abort protocol the GEMM
+ * kernels use, on a barrier nobody arrives on, with a budget of `limit_cycles` SM cycles (0 ..
+ * 1e8) instead of the kernels' ~2 s. The wait runs out, the warp records `code` (1 .. 899) in the
+ * device status word and returns; *outcome (device int32, may be null) receives 2 (abandoned, abort
+ * flag raised; 1 would mean the barrier completed). A following hbfp_device_status returns
+ * HBFP_ERR_TIMEOUT with `code`. Touches no tensor memory and issues no copy. Asynchronous on
+ * `stream`. */
+HBFP_API int hbfp_selftest_bounded_wait(int64_t limit_cycles, int32_t code, int32_t* outcome, void* stream);
 
 #ifdef __cplusplus
 }

@@ -82,10 +82,8 @@ class HbfpLinear(torch.nn.Module):
 
     # ---- weights
     def _refresh_fp32_copy(self) -> None:
-        """The FP32 tensor autograd sees is the value of the wide copy (plain torch bookkeeping)."""
-        t = self.tile
-        scale = torch.exp2(self.wide.exps.float()).repeat_interleave(t, 0).repeat_interleave(t, 1)
-        self.weight.data = self.wide.mant.float() * scale[: self.fin, : self.fout]
+        """The FP32 tensor autograd sees is the value of the wide copy (hbfp_wide_dequantize)."""
+        self.weight.data = hb.wide_dequantize(self.wide)
 
     def apply_update(self, delta: torch.Tensor) -> None:
         """``W <- Q16(float32(W + delta))`` in wide storage, views refreshed by the same launch."""
@@ -158,9 +156,7 @@ class HbfpConv3x3(torch.nn.Module):
         return hb.Format(mant_bits=self.mant_bits, block=self.pixel_block, stream_id=which)
 
     def _refresh_fp32_copy(self) -> None:
-        t = self.c
-        scale = torch.exp2(self.wide.exps.float()).repeat_interleave(t, 0).repeat_interleave(t, 1)
-        self.weight.data = self.wide.mant.float() * scale[: 9 * self.c, : self.fout]
+        self.weight.data = hb.wide_dequantize(self.wide)
 
     def apply_update(self, delta: torch.Tensor) -> None:
         hb.wide_update(self.wide, delta.contiguous(), self.fmt_weight(), views=self.views)

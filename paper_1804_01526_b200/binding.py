@@ -28,7 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
-    "hbfp_im2col_packed", "hbfp_im2col_packed_t",
+    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel",
 ]
 
 
@@ -104,8 +104,13 @@ def lib() -> ctypes.CDLL:
         L.hbfp_gemm_static.argtypes = [i32, i32, i64, i64, i64, p, i64, p, i64, p, i64, p, p, u32, p]
         L.hbfp_gemm_block_partials.argtypes = [i64, i64, i64, p, p, p, u32, p]
         L.hbfp_device_status.argtypes = [p, p]
+        L.hbfp_wide_dequantize.argtypes = [p, p, i64, i64, i32, p, i64, p]
+        L.hbfp_selftest_bounded_wait.argtypes = [i64, i32, p, p]
+        L.hbfp_last_gemm_kernel.restype = ctypes.c_char_p
+        L.hbfp_last_gemm_kernel.argtypes = []
         for name in EXPORTS[1:]:
-            getattr(L, name).restype = ctypes.c_int
+            if name != "hbfp_last_gemm_kernel":
+                getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -263,6 +268,25 @@ def wide_narrow(wide: Wide, fmt: Format, views: Optional[Tuple[Packed, Packed]] 
     return views
 
 
+def wide_dequantize(wide: Wide, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """hbfp_wide_dequantize: the FP32 value ``mant * 2^exps`` of the wide copy (exact)."""
+    d0, d1 = wide.mant.shape
+    if out is None:
+        out = torch.empty((d0, d1), dtype=torch.float32, device=wide.mant.device)
+    _check_f32(out, "out")
+    _check(lib().hbfp_wide_dequantize(_dptr(wide.mant), _dptr(wide.exps), d0, d1, wide.tile, _dptr(out), _ld(out),
+                                      _stream()), "hbfp_wide_dequantize")
+    return out
+
+
+def selftest_bounded_wait(limit_cycles: int = 20000, code: int = 777) -> int:
+    """hbfp_selftest_bounded_wait: one warp runs the kernels' bounded barrier wait on a barrier nobody
+    arrives on; returns the outcome word (2 = the wait was abandoned)."""
+    outcome = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().hbfp_selftest_bounded_wait(limit_cycles, code, _dptr(outcome), _stream()), "hbfp_selftest_bounded_wait")
+    return int(outcome.item())
+
+
 def im2col_packed(px: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, pad: int,
                   out: Optional[Packed] = None) -> Packed:
     """hbfp_im2col_packed: the packed convolution operand ``[n*ho*wo][kh*kw*c]`` gathered from the
@@ -401,6 +425,11 @@ def gemm_block_partials(a: Packed, b: Packed, impl: int = GEMM_FORCE_SIMT) -> to
     _check(lib().hbfp_gemm_block_partials(M, N, K, ctypes.byref(oa), ctypes.byref(ob), _dptr(P), impl, _stream()),
            "hbfp_gemm_block_partials")
     return P
+
+
+def last_gemm_kernel() -> str:
+    """hbfp_last_gemm_kernel: the GEMM kernel this thread's last GEMM call launched."""
+    return lib().hbfp_last_gemm_kernel().decode()
 
 
 def device_status() -> int:

@@ -25,6 +25,9 @@ int read_clear_device_status(cudaStream_t st, int32_t* out) {
 
 namespace {
 
+// Name of the GEMM kernel the calling thread's last hbfp_gemm* call launched (hbfp_last_gemm_kernel).
+thread_local const char* t_last_gemm_kernel = "";
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct GemmPlan {
@@ -135,11 +138,16 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
         const bool long_k = g.la.nkb * g.la.bp >= 1024;
         const bool pair_ok = !P && quad_rows && flags != HBFP_GEMM_FORCE_TENSOR_1SM && pair_gemm_eligible(M, N, pa, pb, g.tp) &&
                              (long_k || flags == HBFP_GEMM_FORCE_TENSOR_2SM);
-        if (pair_ok) return launch_gemm_tensor_pair(M, N, pa, pb, C, ldc, g.tp, ws ? ws + g.off_partial : nullptr, st);
+        if (pair_ok) {
+            t_last_gemm_kernel = "gemm_tc2_kernel";
+            return launch_gemm_tensor_pair(M, N, pa, pb, C, ldc, g.tp, ws ? ws + g.off_partial : nullptr, st);
+        }
         if (flags == HBFP_GEMM_FORCE_TENSOR_2SM) return HBFP_ERR_UNSUPPORTED;
+        t_last_gemm_kernel = "gemm_tc_kernel";
         return launch_gemm_tensor(M, N, K, pa, pb, C, ldc, P, g.tp, ws ? ws + g.off_partial : nullptr, st);
     }
     if (flags >= HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_UNSUPPORTED;
+    t_last_gemm_kernel = "gemm_simt_kernel";
     return launch_gemm_simt(M, N, K, pa, pb, C, ldc, P, st);
 }
 
@@ -149,6 +157,8 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
 using namespace hbfp;
 
 extern "C" {
+
+const char* hbfp_last_gemm_kernel(void) { return t_last_gemm_kernel; }
 
 const char* hbfp_status_string(int status) {
     switch (status) {
@@ -248,6 +258,13 @@ int hbfp_wide_narrow(const int16_t* wide, const int8_t* wide_exps, int64_t d0, i
                        static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_wide_dequantize(const int16_t* wide, const int8_t* wide_exps, int64_t d0, int64_t d1, int32_t tile, float* out,
+                         int64_t ldo, void* stream) {
+    if (d0 < 0 || d1 < 0 || tile <= 0 || ldo < d1) return HBFP_ERR_INVALID_ARG;
+    if (d0 * d1 > 0 && (!wide || !wide_exps || !out)) return HBFP_ERR_INVALID_ARG;
+    return launch_wide_dequantize(wide, wide_exps, d0, d1, tile, out, ldo, static_cast<cudaStream_t>(stream));
+}
+
 int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_t n, int64_t h, int64_t w, int64_t c, int kh,
                        int kw, int pad, const hbfp_format* fmt, void* mant_out, int8_t* exps_out, void* stream) {
     if (!fmt || n < 0 || h <= 0 || w <= 0 || c <= 0 || kh <= 0 || kw <= 0 || pad < 0) return HBFP_ERR_INVALID_ARG;
@@ -334,6 +351,10 @@ int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbfp_operand
     if (a->kind != HBFP_OPERAND_PACKED || b->kind != HBFP_OPERAND_PACKED) return HBFP_ERR_INVALID_ARG;
     if (impl != HBFP_GEMM_FORCE_SIMT && impl != HBFP_GEMM_FORCE_TENSOR) return HBFP_ERR_INVALID_ARG;
     return gemm_impl(M, N, K, a, b, nullptr, N, nullptr, 0, impl, P, static_cast<cudaStream_t>(stream));
+}
+
+int hbfp_selftest_bounded_wait(int64_t limit_cycles, int32_t code, int32_t* outcome, void* stream) {
+    return launch_wait_probe((long long)limit_cycles, (int)code, reinterpret_cast<int*>(outcome), static_cast<cudaStream_t>(stream));
 }
 
 int hbfp_device_status(void* stream, int32_t* status) {

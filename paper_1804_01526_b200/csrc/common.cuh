@@ -74,6 +74,8 @@ int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, co
 int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,
                 int16_t* wide, int8_t* wide_exps, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
                 cudaStream_t st);
+int launch_wide_dequantize(const int16_t* wide, const int8_t* exps, int64_t d0, int64_t d1, int tile, float* out,
+                           int64_t ldo, cudaStream_t st);
 // Packed convolution operand gathered from the packed per-pixel operand.
 int launch_im2col_packed(const int8_t* xm, const int8_t* xe, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
                          int pad, const hbfp_format* f, int8_t* om, int8_t* oe, cudaStream_t st);
@@ -105,6 +107,9 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
 bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, const TensorPlan& plan);
 int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed& b, float* C, int64_t ldc,
                             const TensorPlan& plan, void* partial, cudaStream_t st);
+
+// One warp running the kernels' bounded barrier wait on a barrier nobody arrives on (test hook).
+int launch_wait_probe(long long limit_cycles, int code, int* outcome, cudaStream_t st);
 
 // Device status word (bounded waits report here).
 int32_t* device_status_word();   // device address, per current device

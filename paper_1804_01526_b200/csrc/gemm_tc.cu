@@ -649,7 +649,32 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
     return launch_status();
 }
 
+// One warp waits, with the kernels' own bounded wait and a cycle budget chosen by the caller, on a
+// barrier that nobody arrives on: the wait runs out, records `code`, raises the abort flag and the
+// kernel returns. No TMA, no tensor memory: nothing that could fault or outlive the launch.
+__global__ void __launch_bounds__(32, 1) wait_probe_kernel(int32_t* status, long long limit_cycles, int code, int* outcome) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_word = 0;
+    }
+    __syncwarp();
+    const bool done = mbar_wait(smem_u32(&bar), 0, abort_flag, status, code, true, limit_cycles);
+    const bool any_done = __any_sync(0xffffffffu, done);
+    if (threadIdx.x == 0 && outcome) *outcome = (any_done ? 1 : 0) | (*abort_flag ? 2 : 0);   // expected: 2
+}
+
 }  // namespace
+
+int launch_wait_probe(long long limit_cycles, int code, int* outcome, cudaStream_t st) {
+    int32_t* status = device_status_word();
+    if (!status) return HBFP_ERR_CUDA;
+    if (limit_cycles < 0 || limit_cycles > 100000000ll || code <= 0 || code >= 900) return HBFP_ERR_INVALID_ARG;
+    wait_probe_kernel<<<1, 32, 0, st>>>(status, limit_cycles, code, outcome);
+    return launch_status();
+}
 
 TensorPlan plan_gemm_tensor(int64_t M, int64_t N, int64_t K, const Layout& la, const Layout& lb, int mant_bits_a,
                             int mant_bits_b) {

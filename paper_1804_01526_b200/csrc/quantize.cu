@@ -1427,6 +1427,25 @@ int launch_unpack(const Packed& p, int16_t* q, int8_t* s, cudaStream_t st) {
     return launch_status();
 }
 
+// Value of wide weight storage, Eq. 1: out[i][j] = q16[i][j] * 2^s16[i/t][j/t] (exact in binary32: 16-bit mantissas).
+__global__ void wide_dequant_kernel(const int16_t* __restrict__ wide, const int8_t* __restrict__ exps, int64_t d0,
+                                    int64_t d1, int t, int64_t tiles1, float* __restrict__ out, int64_t ldo) {
+    const int64_t n = d0 * d1;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / d1, c = i - r * d1;
+        const int e = exps[(r / t) * tiles1 + c / t];
+        out[r * ldo + c] = ldexpf((float)wide[i], e);
+    }
+}
+
+int launch_wide_dequantize(const int16_t* wide, const int8_t* exps, int64_t d0, int64_t d1, int tile, float* out,
+                           int64_t ldo, cudaStream_t st) {
+    if (d0 * d1 == 0) return HBFP_OK;
+    const int64_t tiles1 = (d1 + tile - 1) / tile;
+    wide_dequant_kernel<<<blocks_for(d0 * d1, 256), 256, 0, st>>>(wide, exps, d0, d1, tile, tiles1, out, ldo);
+    return launch_status();
+}
+
 int launch_dequantize(const Packed& p, float* out, int64_t ld, cudaStream_t st) {
     const Layout& L = p.L;
     if (L.rows * L.k == 0) return HBFP_OK;

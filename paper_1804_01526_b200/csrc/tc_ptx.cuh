@@ -47,13 +47,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait. Returns false when the wait was abandoned (abort flag raised by anyone, or the
 // cycle budget ran out, in which case this thread raises the flag and records `code`).
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            int32_t* status, int code, bool heed_abort) {
+                                            int32_t* status, int code, bool heed_abort, long long limit) {
     const long long t0 = clock64();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (heed_abort && *abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicCAS(status, 0, code);
             return false;
@@ -61,9 +61,10 @@ __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, vo
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status, int code, bool heed_abort = true) {
+                                          int32_t* status, int code, bool heed_abort = true,
+                                          long long limit = WAIT_LIMIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status, code, heed_abort);
+    return mbar_wait_slow(bar, parity, abort_flag, status, code, heed_abort, limit);
 }
 
 // Whole-warp variant: every lane waits and the verdict is made uniform, so that the warp never

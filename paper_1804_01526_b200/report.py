@@ -163,7 +163,7 @@ def rows_for(specs, tensors_np, peak_tops, hbm_gbs):
         t_g = _time_auto(lambda: hb.gemm_q(sp.M, sp.N, sp.K, pa, pb, out=C, workspace=ws))
         ops = sp.ops
         planes = 1 if fa.mant_bits <= 8 else 2
-        qa_bytes = A.numel() * (4 + planes + 1.0 / max(fa.block, 1))
+        qa_bytes = A.numel() * (4 + planes + 1.0 / (fa.block if fa.block > 0 else sp.K))
         tops_g = ops / (t_g * 1e-3) / 1e12
         tops_all = ops / ((t_qa + t_qb + t_g) * 1e-3) / 1e12
         fmt = f"m{fa.mant_bits} b{fa.block}" + (f" t{fb.tile}" if fb.tile else "") + (" SR" if fa.rounding else " RNE")
@@ -194,7 +194,9 @@ def main():
         if specs:
             lines += rows_for(specs, wl.materialize(specs, seed=seed), args.peak_tops, args.hbm_gbs)
     for n in args.sweep:
-        for (m, b, r) in ((8, 128, 0), (8, 64, 0), (8, 32, 0), (8, 128, 1), (12, 64, 1)):
+        # the design points of Sec. 6: 8- and 12-bit mantissas, the 4-bit end of the mantissa range, and one
+        # exponent per whole row / column (block 0: BFP without tiles)
+        for (m, b, r) in ((8, 128, 0), (8, 64, 0), (8, 32, 0), (8, 128, 1), (12, 64, 1), (4, 128, 0), (8, 0, 0)):
             specs = wl.config_sweep(n, m, b, r)
             if args.only and args.only not in specs[0].name:
                 continue

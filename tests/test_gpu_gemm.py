@@ -309,3 +309,14 @@ def test_large_magnitudes_are_computed_or_reported_never_silently_wrong(hb, kern
     # the library is healthy afterwards
     rc, code, C, ref = _range_case(hb, wl.draw("normal", (M, K), seed=82), B, flag)
     assert rc == hb.OK and np.array_equal(C, ref["c_seq"])
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable(hb):
+    """The wait routine of the GEMM kernels, on a barrier nobody arrives on, with a budget of a few
+    thousand cycles: the status word carries the code, the next read is clean, the next GEMM is right."""
+    assert hb.device_status() == 0
+    assert hb.selftest_bounded_wait(limit_cycles=5000, code=777) == 2      # abandoned, abort flag raised
+    assert hb.device_status_rc() == (hb.ERR_TIMEOUT, 777)
+    assert hb.device_status_rc() == (hb.OK, 0)
+    specs = wl.config_single_256()
+    run_spec(hb, specs[0], wl.materialize(specs, seed=0), hb.GEMM_AUTO)

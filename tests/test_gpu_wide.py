@@ -58,6 +58,9 @@ def test_wide_quantise_and_narrow_views_match_the_oracle(hb, shape, law, fd):
     # the read-only entry point writes the same views
     again = hb.wide_narrow(wide, gfmt(fd))
     check_views(hb, again, qm, sm, t)
+    # the FP32 value of the wide copy is Eq. 1 written out: mantissa times 2^(tile exponent), exact
+    val = hb.wide_dequantize(wide).cpu().numpy()
+    assert np.array_equal(val, np.ldexp(q16.astype(np.float64), np.repeat(s16, t, axis=1)[:, : shape[1]].astype(np.int64)).astype(np.float32))
     for a, b in zip(again, views):                               # and the same bytes in every documented position
         lay = hb.packed_layout(a.rows, a.k, a.fmt)
         for pl in range(lay["planes"]):

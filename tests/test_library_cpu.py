@@ -34,7 +34,7 @@ def test_struct_sizes_match_header(hb):
 
 def test_status_strings(hb):
     assert hb.status_string(0) == "ok"
-    assert len({hb.status_string(i) for i in range(8)}) == 8
+    assert len({hb.status_string(i) for i in range(9)}) == 9
 
 
 @pytest.mark.parametrize("rows,k,m,b,exp", [
