@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_quantize.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p]
         L.oracle_gemm.restype = ctypes.c_int
         L.oracle_gemm.argtypes = [i64, i64, i64, i64, p, p, p, p, p, p, p, p, ctypes.c_int]
+        L.oracle_quantize_conv_weights.restype = ctypes.c_int
+        L.oracle_quantize_conv_weights.argtypes = [p, i64, i64, i64, i64, ctypes.c_int, p, p, p]
         L.oracle_wide_narrow.restype = ctypes.c_int
         L.oracle_wide_narrow.argtypes = [p, p, i64, i64, ctypes.c_int, p, p]
         L.oracle_wide_update.restype = ctypes.c_int
@@ -211,6 +213,23 @@ def hbfp_gemm(transA: int, transB: int, A: np.ndarray, B: np.ndarray, fmtA: Form
     if rc:
         raise ValueError(f"oracle_hbfp_gemm failed: {rc}")
     return {"c_ref": c_ref, "a_mag": a_mag, "c_seq": c_seq}
+
+
+def quantize_conv_weights(w: np.ndarray, taps: int, contract_axis: int, fmt: Format):
+    """Convolution weights ``w [taps * c_in][c_out]`` with one exponent per tile of ``t`` input maps x ``t``
+    output maps across all filter taps (``fmt.tile``). Returns ``(q, s)`` laid out like ``quantize``."""
+    assert w.dtype == np.float32 and w.ndim == 2 and w.shape[0] % taps == 0
+    w = np.ascontiguousarray(w)
+    d0, d1 = w.shape
+    c_in = d0 // taps
+    k, rows = (d1, d0) if contract_axis == 1 else (d0, d1)
+    q = np.zeros((rows, k), dtype=np.int16)
+    s = np.zeros((rows, n_blocks(k, fmt.tile)), dtype=np.int8)
+    cf = fmt._c()
+    rc = lib().oracle_quantize_conv_weights(_ptr(w), taps, c_in, d1, d1, contract_axis, ctypes.byref(cf), _ptr(q), _ptr(s))
+    if rc:
+        raise ValueError(f"oracle_quantize_conv_weights failed: {rc}")
+    return q, s
 
 
 def wide_quantize(w: np.ndarray, fmt: Format):

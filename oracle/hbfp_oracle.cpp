@@ -234,6 +234,69 @@ int oracle_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int cont
 }
 
 // ---------------------------------------------------------------------------------------
+// Weights of a convolution layer (Sec. 5.1, last sentence: for convolutional layers the two outer,
+// feature-map dimensions of the weights are tiled). The weights are w[tap][ci][co], tap = (filter row,
+// filter column), stored as the matrix [taps * c_in][c_out] that the convolution GEMM multiplies by.
+// Reading taken: a tile is t input maps x t output maps and spans every filter tap, so all
+// kh * kw * t * t weights of a tile share one exponent (the filter dimensions are not tiled):
+//   E[u][v] = exponent of max |w[tap][ci][co]| over all taps, ci in [u t, (u+1) t), co in [v t, (v+1) t)
+// Every weight is then rounded on its tile's grid exactly as in oracle_quantize. Output in the
+// canonical layout of that function for the same contraction axis: axis 0 (forward: contraction over
+// (tap, ci)) q [c_out][taps * c_in], s [c_out][taps * c_in / t]; axis 1 (backward-data: contraction over
+// co) q [taps * c_in][c_out], s [taps * c_in][ceil(c_out / t)]. Needs f->tile == f->block == t > 0 and
+// c_in % t == 0 (a K-block never straddles two taps). Returns 0, -1 bad arguments, -2 bad format.
+// ---------------------------------------------------------------------------------------
+int oracle_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                                 int contract_axis, const oracle_format* f, int16_t* q, int8_t* s) {
+    if (!w || !f || !q || !s || taps <= 0 || c_in <= 0 || c_out <= 0 || ld < c_out) return -1;
+    if (contract_axis != 0 && contract_axis != 1) return -1;
+    const int m = f->mant_bits;
+    if (m < 2 || m > 16) return -2;
+    const int64_t t = f->tile;
+    if (t <= 0 || f->block != t || c_in % t != 0) return -2;
+    const int64_t nu = c_in / t, nv = (c_out + t - 1) / t;
+    const int64_t d0 = taps * c_in, d1 = c_out;
+    const int64_t idx_cols = f->idx_cols > 0 ? f->idx_cols : d1;
+    // Pass 1: one exponent per (input-map tile, output-map tile), over all taps.
+    std::vector<int> E((size_t)(nu * nv));
+    for (int64_t u = 0; u < nu; ++u)
+        for (int64_t v = 0; v < nv; ++v) {
+            double amax = 0.0;
+            const int64_t co1 = (v + 1) * t < c_out ? (v + 1) * t : c_out;
+            for (int64_t tap = 0; tap < taps; ++tap)
+                for (int64_t ci = u * t; ci < (u + 1) * t; ++ci)
+                    for (int64_t co = v * t; co < co1; ++co) {
+                        double a = std::fabs((double)w[(tap * c_in + ci) * ld + co]);
+                        if (a > amax) amax = a;
+                    }
+            E[(size_t)(u * nv + v)] = oracle_block_exponent(amax, m, f->exp_mode);
+        }
+    // Pass 2: mantissas and the canonical exponent array.
+    const int64_t nkb0 = d0 / t;
+    for (int64_t i = 0; i < d0; ++i)
+        for (int64_t j = 0; j < d1; ++j) {
+            const int64_t ci = i % c_in;
+            const int se = E[(size_t)((ci / t) * nv + j / t)];
+            const float v = w[i * ld + j];
+            int32_t qq;
+            if (f->rounding == 0) {
+                qq = oracle_round_rne(v, se, m);
+            } else {
+                uint32_t rnd = oracle_sr_draw(f->seed, f->stream_id, (uint64_t)((i + f->idx_row_off) * idx_cols + (j + f->idx_col_off)));
+                qq = oracle_round_sr(v, se, m, rnd);
+            }
+            if (contract_axis == 0) {
+                q[j * d0 + i] = (int16_t)qq;
+                s[j * nkb0 + i / t] = (int8_t)se;
+            } else {
+                q[i * d1 + j] = (int16_t)qq;
+                s[i * nv + j / t] = (int8_t)se;
+            }
+        }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------
 // BFP matrix product of two canonically quantised operands (Eq. 2 applied per block, blocks
 // accumulated in floating point):
 //   P[i][j][kb] = sum_{k in block kb} qA[i][k] * qB[j][k]                (integers, exact)
