@@ -294,6 +294,24 @@ HBFP_API int hbfp_gemm_q(int64_t M, int64_t N, int64_t K, const hbfp_operand* a,
                          const hbfp_operand* b, float* C, int64_t ldc, void* workspace,
                          size_t workspace_bytes, uint32_t flags, void* stream);
 
+/* Convolution forward pass as one implicit GEMM (Sec. 5.1: convolutions run through the same BFP dot
+ * products): Y [n*h*w][filters] = conv(x, filters), stride 1, `pad` zeros around the image, an output as
+ * large as the input (2 pad == kh - 1 == kw - 1). x: the activations [n][h][w][c] converted once per
+ * pixel - hbfp_quantize(x as [n*h*w][c], contract_axis 1, block = c, fmt_x) - given as mant_x / exps_x;
+ * filters_op: a packed operand with rows = filters, k = kh*kw*c, block = c, K ordered (filter row, filter
+ * column, channel), e.g. view c0 of hbfp_quantize_tiles / hbfp_wide_* of the [kh*kw*c][filters] matrix or
+ * hbfp_quantize of it with contract_axis 0. The kernel reads every tap's channel vectors straight from
+ * the packed pixels (one 4-D TMA box per tap and 128 output pixels; positions outside the image read as
+ * zero mantissas): the packed im2col operand of hbfp_im2col_packed is never formed. The result equals
+ * hbfp_gemm_q on that operand bit for bit (taps accumulated in ascending order, one FP32 rounding each).
+ * Y: FP32, 16-byte aligned, row stride ldy >= filters, ldy % 4 == 0. Supported: c in {64, 128}, mantissas
+ * up to 8 bits, w in {16, 32, 64, 128}, h a multiple of 128 / w, up to 256 filters, kh * kw <= 25; any
+ * other case returns HBFP_ERR_UNSUPPORTED and leaves Y untouched (use hbfp_im2col_packed + hbfp_gemm_q).
+ * Exponent range as for the paired-SM GEMM (hbfp_gemm). Asynchronous on `stream`, allocates nothing. */
+HBFP_API int hbfp_conv_forward(const void* mant_x, const int8_t* exps_x, int64_t n, int64_t h, int64_t w, int64_t c,
+                               int kh, int kw, int pad, const hbfp_format* fmt_x, const hbfp_operand* filters_op,
+                               int64_t filters, float* Y, int64_t ldy, void* stream);
+
 /* Inspection hook: the exact per-block integer sums P [M][N][nkb] (int32) of two packed
  * operands (Eq. 2's fixed-point dot product), for small shapes. `impl` selects the kernel that
  * produces them: HBFP_GEMM_FORCE_SIMT or HBFP_GEMM_FORCE_TENSOR. */
@@ -303,7 +321,8 @@ HBFP_API int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbf
 
 /* Host-only: name of the GEMM kernel that the calling thread's most recent hbfp_gemm, hbfp_gemm_q,
  * hbfp_gemm_static or hbfp_gemm_block_partials call launched ("gemm_tc2_kernel": two SMs per 256 x 256
- * tile; "gemm_tc_kernel": one SM per tile; "gemm_simt_kernel"), "" before the first launch. For
+ * tile; "gemm_tc_kernel": one SM per tile; "gemm_simt_kernel"; "conv_fwd_kernel" after hbfp_conv_forward),
+ * "" before the first launch. For
  * measurement scripts that must name the kernel they timed (the paper has no counterpart). The
  * string is static storage. */
 HBFP_API const char* hbfp_last_gemm_kernel(void);

@@ -28,7 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
-    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel",
+    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel", "hbfp_conv_forward",
 ]
 
 
@@ -104,6 +104,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_gemm_static.argtypes = [i32, i32, i64, i64, i64, p, i64, p, i64, p, i64, p, p, u32, p]
         L.hbfp_gemm_block_partials.argtypes = [i64, i64, i64, p, p, p, u32, p]
         L.hbfp_device_status.argtypes = [p, p]
+        L.hbfp_conv_forward.argtypes = [p, p, i64, i64, i64, i64, i32, i32, i32, p, p, i64, p, i64, p]
         L.hbfp_wide_dequantize.argtypes = [p, p, i64, i64, i32, p, i64, p]
         L.hbfp_selftest_bounded_wait.argtypes = [i64, i32, p, p]
         L.hbfp_last_gemm_kernel.restype = ctypes.c_char_p
@@ -297,6 +298,22 @@ def im2col_packed(px: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, 
     f = px.fmt.c()
     _check(lib().hbfp_im2col_packed(_dptr(px.mant), _dptr(px.exps), n, h, w, c, kh, kw, pad, ctypes.byref(f),
                                     _dptr(out.mant), _dptr(out.exps), _stream()), "hbfp_im2col_packed")
+    return out
+
+
+def conv_forward(px: Packed, filters: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, pad: int,
+                 out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """hbfp_conv_forward: the convolution ``[n*h*w][filters]`` of packed pixels ``px`` (block = c) with the
+    packed filters ``filters`` (rows = filters, k = kh*kw*c) as one implicit GEMM. Raises ``HbfpError``
+    (ERR_UNSUPPORTED) for shapes the kernel does not cover."""
+    nf = filters.rows
+    if out is None:
+        out = torch.empty((n * h * w, nf), dtype=torch.float32, device=px.mant.device)
+    _check_f32(out, "out")
+    fx = px.fmt.c()
+    op = filters.operand()
+    _check(lib().hbfp_conv_forward(_dptr(px.mant), _dptr(px.exps), n, h, w, c, kh, kw, pad, ctypes.byref(fx), ctypes.byref(op),
+                                   nf, _dptr(out), _ld(out), _stream()), "hbfp_conv_forward")
     return out
 
 

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhbfp.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_static.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_conv.cu", "gemm_static.cu"]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo",

@@ -276,6 +276,33 @@ int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_t n, int6
                                 static_cast<int8_t*>(mant_out), exps_out, static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_conv_forward(const void* mant_x, const int8_t* exps_x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
+                      int pad, const hbfp_format* fmt_x, const hbfp_operand* filters_op, int64_t filters, float* Y,
+                      int64_t ldy, void* stream) {
+    if (!fmt_x || !filters_op || n < 0 || h <= 0 || w <= 0 || c <= 0 || kh <= 0 || kw <= 0 || pad < 0 || filters <= 0)
+        return HBFP_ERR_INVALID_ARG;
+    if (!mant_x || !exps_x || !Y || ldy < filters) return HBFP_ERR_INVALID_ARG;
+    if (filters_op->struct_size != sizeof(hbfp_operand) || filters_op->kind != HBFP_OPERAND_PACKED || !filters_op->data ||
+        !filters_op->exps)
+        return HBFP_ERR_INVALID_ARG;
+    if (fmt_x->block != c || fmt_x->tile != 0 || filters_op->fmt.block != c) return HBFP_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(mant_x) & 255) || (reinterpret_cast<uintptr_t>(filters_op->data) & 255)) return HBFP_ERR_ALIGNMENT;
+    Packed px, pw;
+    int rc = make_layout(n * h * w, c, fmt_x, &px.L);
+    if (rc) return rc;
+    rc = make_layout(filters, (int64_t)kh * kw * c, &filters_op->fmt, &pw.L);
+    if (rc) return rc;
+    px.mant = static_cast<const int8_t*>(mant_x);
+    px.exps = exps_x;
+    px.mant_bits = fmt_x->mant_bits;
+    pw.mant = static_cast<const int8_t*>(filters_op->data);
+    pw.exps = static_cast<const int8_t*>(filters_op->exps);
+    pw.mant_bits = filters_op->fmt.mant_bits;
+    if (n == 0) return HBFP_OK;
+    t_last_gemm_kernel = "conv_fwd_kernel";
+    return launch_conv_forward(px, pw, n, h, w, c, kh, kw, pad, filters, Y, ldy, static_cast<cudaStream_t>(stream));
+}
+
 int hbfp_im2col_packed_t(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw, int pad,
                          const hbfp_format* fmt, void* mant, int8_t* exps, void* stream) {
     if (!fmt || n < 0 || h <= 0 || w <= 0 || c <= 0 || kh <= 0 || kw <= 0 || pad < 0) return HBFP_ERR_INVALID_ARG;

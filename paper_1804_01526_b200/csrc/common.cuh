@@ -108,6 +108,10 @@ bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, 
 int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed& b, float* C, int64_t ldc,
                             const TensorPlan& plan, void* partial, cudaStream_t st);
 
+// Convolution forward as an implicit GEMM over the packed pixels (gemm_conv.cu).
+int launch_conv_forward(const Packed& x, const Packed& wt, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw,
+                        int pad, int64_t filters, float* Y, int64_t ldy, cudaStream_t st);
+
 // One warp running the kernels' bounded barrier wait on a barrier nobody arrives on (test hook).
 int launch_wait_probe(long long limit_cycles, int code, int* outcome, cudaStream_t st);
 

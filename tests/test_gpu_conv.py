@@ -137,3 +137,51 @@ def test_backward_weight_operand_is_nearest_even_only(hb):
     with pytest.raises(hb.HbfpError) as e:
         hb.im2col_packed_t(x, 3, 3, 1, hb.Format(mant_bits=8, block=16, rounding=1))
     assert e.value.code == hb.ERR_UNSUPPORTED
+
+
+IMPLICIT_CASES = [
+    # n, h, w, c, filters, kh, pad, weight law: shapes the implicit-GEMM kernel covers
+    (4, 32, 32, 64, 64, 3, 1),        # the 64 -> 64 convolution of the ResNet configuration (four images)
+    (3, 16, 16, 128, 128, 3, 1),      # the 128 -> 128 one; an odd number of 128-pixel row tiles
+    (5, 8, 16, 64, 12, 3, 1),         # few filters; a last super tile that is only partly there
+    (2, 16, 16, 128, 200, 5, 2),      # 5 x 5 filter, 200 filters (256-wide tile)
+    (1, 4, 128, 64, 96, 1, 0),        # 1 x 1 filter, an image row as long as a row tile
+    (7, 4, 64, 64, 132, 3, 1),
+]
+
+
+@pytest.mark.parametrize("n,h,w,c,f,k,pad", IMPLICIT_CASES)
+def test_implicit_gemm_convolution_equals_oracle_and_the_gather_path(hb, n, h, w, c, f, k, pad):
+    """hbfp_conv_forward reads the taps straight from the packed pixels: same numbers as the oracle's GEMM
+    on the im2col matrix in its sequential order, and what gather + GEMM gives."""
+    x = wl.draw("half_normal", (n * h * w, c), seed=75).reshape(n, h, w, c)
+    x *= np.exp(2 * wl.draw("normal", (n * h * w, 1), seed=76)).reshape(n, h, w, 1).astype(np.float32)
+    wt = wl.draw("he_weight", (k * k * c, f), seed=77, fan_in=k * k * c)
+    fd = dict(mant_bits=8, block=c, rounding=0, seed=0)
+    px = hb.quantize(to_dev(x.reshape(n * h * w, c)), 1, gfmt(fd))
+    pw = hb.quantize(to_dev(wt), 0, gfmt(fd, stream_id=1))
+    Y = hb.conv_forward(px, pw, n, h, w, c, k, k, pad).cpu().numpy()
+    assert hb.device_status() == 0
+    assert hb.last_gemm_kernel() == "conv_fwd_kernel"
+    cols = oracle.im2col(x, k, k, pad)
+    ref = oracle.hbfp_gemm(0, 0, cols, wt, ofmt(fd), ofmt(fd, stream_id=1))
+    err = np.abs(Y.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all(), float((err / np.maximum(ref["a_mag"], 1e-300)).max())
+    assert np.array_equal(Y, ref["c_seq"])            # taps in ascending order, one rounding each
+    # the gather + GEMM path computes the same product (it may split K for a small output, so its order of
+    # accumulation can differ: the tolerance of the GEMM tests)
+    pa = hb.im2col_packed(px, n, h, w, c, k, k, pad)
+    Y2 = hb.gemm_q(n * h * w, f, k * k * c, pa, pw).cpu().numpy()
+    assert (np.abs(Y.astype(np.float64) - Y2.astype(np.float64)) <= 2 * TOL * ref["a_mag"]).all()
+
+
+def test_implicit_gemm_convolution_says_what_it_does_not_cover(hb):
+    n, h, w, c, f = 1, 9, 7, 24, 8
+    x = wl.draw("half_normal", (n * h * w, c), seed=78)
+    wt = wl.draw("he_weight", (9 * c, f), seed=79, fan_in=9 * c)
+    fd = dict(mant_bits=8, block=c)
+    px = hb.quantize(to_dev(x), 1, gfmt(fd))
+    pw = hb.quantize(to_dev(wt), 0, gfmt(fd))
+    with pytest.raises(hb.HbfpError) as e:
+        hb.conv_forward(px, pw, n, h, w, c, 3, 3, 1)
+    assert e.value.code == hb.ERR_UNSUPPORTED
