@@ -132,6 +132,20 @@ HBFP_API int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t
                                  const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0,
                                  void* mant_c1, int8_t* exps_c1, int8_t* tile_exps, void* stream);
 
+/* Weights of a convolution layer with tiled feature-map dimensions (Sec. 5.1, last sentence). w: FP32
+ * [taps * c_in][c_out] (taps = filter rows x filter columns, row index (tap, input map); pitch ld >=
+ * c_out) - the matrix the convolution GEMM multiplies by. A tile is t input maps x t output maps and
+ * spans every filter tap (fmt->tile == fmt->block == t, c_in % t == 0): the kh * kw * t * t weights of a
+ * tile share one exponent, taken from their largest magnitude; the filter dimensions themselves are not
+ * tiled. Writes view c0 (rows = c_out, k = taps * c_in: forward, hbfp_conv_forward) and / or view c1 (rows
+ * = taps * c_in, k = c_out: backward-data) in the packed layout - either pair of pointers may be NULL -
+ * and, if tile_exps is given, the grid [c_in / t][ceil(c_out / t)] of tile exponents (int8). Rounding,
+ * seed and stream id as in hbfp_quantize (stochastic draws keyed by the index in w). Two passes over w
+ * (weights are converted once per step). HBFP_ERR_UNSUPPORTED when c_in % t != 0. */
+HBFP_API int hbfp_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                                        const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1,
+                                        int8_t* exps_c1, int8_t* tile_exps, void* stream);
+
 /* Wide weight storage (Sec. 4.2 "Wide weight storage": weights are kept with wider mantissas, only
  * weight updates use them, and the forward and backward passes read only the most significant bits).
  * The long-lived copy of w [d0][d1] is `wide`: int16 mantissas, row-major with pitch d1 (device,

@@ -103,8 +103,15 @@ class _HbfpConv3x3Fn(torch.autograd.Function):
         ctx.save_for_backward(x)
         x = x.contiguous()
         px = hb.quantize(x.view(n * h * w, c), 1, layer.fmt_pixels(0))
-        pa = hb.im2col_packed(px, n, h, w, c, 3, 3, 1)
-        y = hb.gemm_q(n * h * w, layer.fout, 9 * c, pa, layer.views[0])
+        try:
+            # the implicit GEMM reads the taps straight from the packed pixels
+            y = hb.conv_forward(px, layer.views[0], n, h, w, c, 3, 3, 1)
+        except hb.HbfpError as e:
+            if e.code != hb.ERR_UNSUPPORTED:
+                raise
+            # shapes it does not cover: gather the packed operand, then the ordinary GEMM (same product)
+            pa = hb.im2col_packed(px, n, h, w, c, 3, 3, 1)
+            y = hb.gemm_q(n * h * w, layer.fout, 9 * c, pa, layer.views[0])
         return y.view(n, h, w, layer.fout)
 
     @staticmethod

@@ -218,6 +218,18 @@ int hbfp_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, cons
                                  static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                               const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1,
+                               int8_t* tile_exps, void* stream) {
+    if (!w || !fmt || taps <= 0 || c_in <= 0 || c_out <= 0 || ld < c_out) return HBFP_ERR_INVALID_ARG;
+    if ((mant_c0 && !exps_c0) || (mant_c1 && !exps_c1) || (!mant_c0 && !mant_c1 && !tile_exps)) return HBFP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(mant_c0) & 255) || (reinterpret_cast<uintptr_t>(mant_c1) & 255) ||
+        (reinterpret_cast<uintptr_t>(exps_c0) & 127) || (reinterpret_cast<uintptr_t>(exps_c1) & 127))
+        return HBFP_ERR_ALIGNMENT;
+    return launch_quantize_conv_weights(w, taps, c_in, c_out, ld, fmt, static_cast<int8_t*>(mant_c0), exps_c0,
+                                        static_cast<int8_t*>(mant_c1), exps_c1, tile_exps, static_cast<cudaStream_t>(stream));
+}
+
 static int wide_views_ok(void* mant_c0, int8_t* exps_c0, void* mant_c1, int8_t* exps_c1) {
     if (!mant_c0 && !mant_c1 && !exps_c0 && !exps_c1) return HBFP_OK;        // wide storage only
     if (!mant_c0 || !exps_c0 || !mant_c1 || !exps_c1) return HBFP_ERR_INVALID_ARG;

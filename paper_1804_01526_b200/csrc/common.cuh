@@ -69,6 +69,9 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int cont
 int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, const hbfp_format* f,
                           int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
                           int8_t* tile_exps, cudaStream_t st);
+int launch_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                                 const hbfp_format* f, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                                 int8_t* tile_exps, cudaStream_t st);
 // Wide weight storage: mode 0 quantise FP32 weights, 1 apply an FP32 update in place, 2 read only; in every
 // mode the packed narrow views are written when their pointers are given.
 int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,

@@ -646,6 +646,35 @@ __global__ void exps_tiles(const float* __restrict__ x, int64_t d0, int64_t d1, 
     else for (int64_t j = v * t + lane; j < j1; j += 32) exps[u * rs + j] = s;
 }
 
+// Pass 1d, convolution weights [taps * c_in][c_out] (Sec. 5.1: the two feature-map dimensions are tiled, the
+// filter taps are not): one warp per (input-map tile u, output-map tile v) takes the maximum over every tap
+// and repeats the tile's exponent for every line and K-block of the view that crosses the tile.
+__global__ void exps_conv_tiles(const float* __restrict__ x, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                                int64_t t, QParams p, int axis, int8_t* __restrict__ exps, int64_t rs, int64_t nu,
+                                int64_t nv, int8_t* __restrict__ tile_exps) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (warp >= nu * nv) return;
+    const int64_t u = warp / nv, v = warp % nv;
+    const int64_t j1 = min(c_out, (v + 1) * t);
+    uint32_t am = 0;
+    for (int64_t tap = 0; tap < taps; ++tap)
+        for (int64_t ci = u * t; ci < (u + 1) * t; ++ci)
+            for (int64_t j = v * t + lane; j < j1; j += 32) am = max(am, abs_bits(x[(tap * c_in + ci) * ld + j]));
+    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    const int8_t s = (int8_t)block_exponent(am, p.m, p.exp_mode);
+    if (tile_exps && lane == 0) tile_exps[u * nv + v] = s;
+    if (!exps) return;
+    // axis 0 (forward view): lines are output maps, K-block (tap, u). axis 1: lines are (tap, ci), K-block v.
+    if (axis == 0) {
+        for (int64_t tap = 0; tap < taps; ++tap)
+            for (int64_t j = v * t + lane; j < j1; j += 32) exps[(tap * nu + u) * rs + j] = s;
+    } else {
+        for (int64_t tap = 0; tap < taps; ++tap)
+            for (int64_t ci = u * t + lane; ci < (u + 1) * t; ci += 32) exps[v * rs + tap * c_in + ci] = s;
+    }
+}
+
 // Pass 2: one thread per 4 output bytes of a line; reads the exponent written by pass 1.
 template <int PLANES>
 __global__ void mant_generic(const float* __restrict__ x, int64_t d1, int64_t rows, int64_t K, int64_t ld,
@@ -1340,6 +1369,41 @@ int launch_quantize_tiles(const float* w, int64_t d0, int64_t d1, int64_t ld, co
                           int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
                           int8_t* tile_exps, cudaStream_t st) {
     return launch_tiles<3>(w, ld, d0, d1, f, nullptr, tile_exps, mant_c0, exps_c0, mant_c1, exps_c1, st);
+}
+
+// Convolution weights w [taps * c_in][c_out] with one exponent per (t input maps) x (t output maps) tile over
+// all taps: view c0 (rows = c_out, k = taps * c_in) and / or view c1 (rows = taps * c_in, k = c_out).
+int launch_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
+                                 const hbfp_format* f, int8_t* mant_c0, int8_t* exps_c0, int8_t* mant_c1, int8_t* exps_c1,
+                                 int8_t* tile_exps, cudaStream_t st) {
+    const int64_t t = f->tile;
+    if (t <= 0 || f->block != t || taps <= 0 || c_in <= 0 || c_out <= 0) return HBFP_ERR_INVALID_ARG;
+    if (c_in % t != 0) return HBFP_ERR_UNSUPPORTED;               // a K-block must not straddle two taps
+    const int64_t d0 = taps * c_in, d1 = c_out, nu = c_in / t, nv = (c_out + t - 1) / t;
+    const QParams p = make_params(f);
+    for (int axis = 0; axis < 2; ++axis) {
+        int8_t* mant = axis == 0 ? mant_c0 : mant_c1;
+        int8_t* exps = axis == 0 ? exps_c0 : exps_c1;
+        if (!mant) continue;
+        Layout L;
+        const int64_t rows = axis == 0 ? d1 : d0, K = axis == 0 ? d0 : d1;
+        int rc = make_layout(rows, K, f, &L);
+        if (rc) return rc;
+        HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        exps_conv_tiles<<<blocks_for(nu * nv * 32, 256), 256, 0, st>>>(w, taps, c_in, c_out, ld, t, p, axis, exps, L.rs, nu, nv,
+                                                                      tile_exps);
+        if (launch_status()) return HBFP_ERR_CUDA;
+        if (L.planes == 1)
+            mant_generic<1><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(w, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
+        else
+            mant_generic<2><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(w, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
+        if (launch_status()) return HBFP_ERR_CUDA;
+    }
+    if (!mant_c0 && !mant_c1 && tile_exps) {
+        exps_conv_tiles<<<blocks_for(nu * nv * 32, 256), 256, 0, st>>>(w, taps, c_in, c_out, ld, t, p, 0, nullptr, 0, nu, nv, tile_exps);
+        return launch_status();
+    }
+    return HBFP_OK;
 }
 
 int launch_wide(int mode, const float* src, int64_t ld, int64_t d0, int64_t d1, const hbfp_format* f,

@@ -111,8 +111,8 @@ def conv_lines():
     """Forward GEMM operand of the two 3x3 convolutions: converting the FP32 im2col matrix against
     converting the activations once per pixel and gathering the packed operand."""
     out = ["", "| convolution | im2col matrix FP32 MB | forward: convert im2col matrix µs | convert pixels µs | gather packed operand µs | GEMM µs | "
-           "backward-weight: convert im2col matrix (column blocks) µs | operand from the activations µs |",
-           "|---|---|---|---|---|---|---|---|"]
+           "implicit GEMM (`hbfp_conv_forward`) µs (GB/s of output) | backward-weight: convert im2col matrix (column blocks) µs | operand from the activations µs |",
+           "|---|---|---|---|---|---|---|---|---|"]
     for name, n, hw, c, f in (("c2.conv64", 128, 32, 64, 64), ("c2.conv128", 128, 16, 128, 128)):
         fmt = hb.Format(mant_bits=8, block=c)          # one block per pixel; the configuration's 64 for the first
         x = torch.from_numpy(wl.draw("half_normal", (n * hw * hw, c), seed=5)).cuda()
@@ -129,13 +129,14 @@ def conv_lines():
         C = torch.empty((M, f), dtype=torch.float32, device="cuda")
         ws = torch.empty(max(hb.gemm_q_workspace(M, f, K, pa, pw), 1), dtype=torch.int8, device="cuda")
         t_m = _time_auto(lambda: hb.gemm_q(M, f, K, pa, pw, out=C, workspace=ws))
+        t_i = _time_auto(lambda: hb.conv_forward(px, pw, n, hw, hw, c, 3, 3, 1, out=C))
         fb = hb.Format(mant_bits=8, block=64)           # backward-weight: blocks of 64 output pixels
         pt = hb.quantize(cols, 0, fb)
         t_ct = _time_auto(lambda: hb.quantize(cols, 0, fb, out=pt))
         x4 = x.view(n, hw, hw, c)
         pt2 = hb.im2col_packed_t(x4, 3, 3, 1, fb)
         t_t = _time_auto(lambda: hb.im2col_packed_t(x4, 3, 3, 1, fb, out=pt2))
-        out.append(f"| {name} {M}x{f}x{K} | {M*K*4/1e6:.0f} | {t_c*1e3:.1f} | {t_p*1e3:.1f} | {t_g*1e3:.1f} | {t_m*1e3:.1f} | {t_ct*1e3:.1f} | {t_t*1e3:.1f} |")
+        out.append(f"| {name} {M}x{f}x{K} | {M*K*4/1e6:.0f} | {t_c*1e3:.1f} | {t_p*1e3:.1f} | {t_g*1e3:.1f} | {t_m*1e3:.1f} | {t_i*1e3:.1f} ({M*f*4/(t_i*1e-3)/1e9:.0f}) | {t_ct*1e3:.1f} | {t_t*1e3:.1f} |")
         del x, x4, wt, px, pa, pw, cols, pc, C, ws, pt, pt2
     torch.cuda.empty_cache()
     return out

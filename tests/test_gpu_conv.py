@@ -185,3 +185,40 @@ def test_implicit_gemm_convolution_says_what_it_does_not_cover(hb):
     with pytest.raises(hb.HbfpError) as e:
         hb.conv_forward(px, pw, n, h, w, c, 3, 3, 1)
     assert e.value.code == hb.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("taps,c_in,c_out,t,m,rounding", [(9, 64, 64, 64, 8, 0), (9, 128, 96, 32, 8, 1), (25, 24, 40, 24, 6, 0),
+                                                          (1, 64, 130, 64, 12, 1)])
+def test_convolution_weights_tiled_on_the_feature_map_dimensions(hb, taps, c_in, c_out, t, m, rounding):
+    """hbfp_quantize_conv_weights against the oracle: one exponent per (t input maps x t output maps) tile over
+    every filter tap, both views bit-exact."""
+    w = wl.draw("he_weight", (taps * c_in, c_out), seed=83, fan_in=taps * c_in)
+    w *= np.exp(wl.draw("normal", (taps * c_in, 1), seed=84)).astype(np.float32)
+    fd = dict(mant_bits=m, block=t, tile=t, rounding=rounding, seed=9, stream_id=2)
+    c0, c1, grid = hb.quantize_conv_weights(to_dev(w), taps, gfmt(fd), want_grid=True)
+    assert hb.device_status() == 0
+    q0, s0 = oracle.quantize_conv_weights(w, taps, 0, ofmt(fd))
+    q1, s1 = oracle.quantize_conv_weights(w, taps, 1, ofmt(fd))
+    g0, e0 = decode_packed(c0, hb.packed_layout(c0.rows, c0.k, c0.fmt))
+    g1, e1 = decode_packed(c1, hb.packed_layout(c1.rows, c1.k, c1.fmt))
+    assert np.array_equal(g0, q0) and np.array_equal(e0, s0)
+    assert np.array_equal(g1, q1) and np.array_equal(e1, s1)
+    assert np.array_equal(grid.cpu().numpy(), s1[:c_in:t, :])
+
+
+def test_convolution_with_tiled_weights_end_to_end(hb):
+    """Pixels converted once, weights tiled over the feature maps, implicit GEMM: the oracle's GEMM on the
+    oracle's operands, bit for bit."""
+    n, h, w_, c, f = 2, 32, 32, 64, 64
+    x = wl.draw("half_normal", (n * h * w_, c), seed=85).reshape(n, h, w_, c)
+    wt = wl.draw("he_weight", (9 * c, f), seed=86, fan_in=9 * c)
+    fx = dict(mant_bits=8, block=c)
+    fw = dict(mant_bits=8, block=c, tile=c, stream_id=1)
+    px = hb.quantize(to_dev(x.reshape(n * h * w_, c)), 1, gfmt(fx))
+    c0, c1, _ = hb.quantize_conv_weights(to_dev(wt), 9, gfmt(fw))
+    Y = hb.conv_forward(px, c0, n, h, w_, c, 3, 3, 1).cpu().numpy()
+    assert hb.device_status() == 0
+    qa, sa = oracle.quantize(oracle.im2col(x, 3, 3, 1), 1, ofmt(fx))
+    qb, sb = oracle.quantize_conv_weights(wt, 9, 0, ofmt(fw))
+    ref = oracle.gemm(qa, sa, qb, sb, c)
+    assert np.array_equal(Y, ref["c_seq"])
