@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_quantize.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p]
         L.oracle_gemm.restype = ctypes.c_int
         L.oracle_gemm.argtypes = [i64, i64, i64, i64, p, p, p, p, p, p, p, p, ctypes.c_int]
+        L.oracle_quantize_indexed.restype = ctypes.c_int
+        L.oracle_quantize_indexed.argtypes = [p, i64, i64, i64, ctypes.c_int, p, p, p, p]
         L.oracle_quantize_conv_weights.restype = ctypes.c_int
         L.oracle_quantize_conv_weights.argtypes = [p, i64, i64, i64, i64, ctypes.c_int, p, p, p]
         L.oracle_wide_narrow.restype = ctypes.c_int
@@ -215,6 +217,23 @@ def hbfp_gemm(transA: int, transB: int, A: np.ndarray, B: np.ndarray, fmtA: Form
     return {"c_ref": c_ref, "a_mag": a_mag, "c_seq": c_seq}
 
 
+def quantize_indexed(x: np.ndarray, contract_axis: int, fmt: Format, index: np.ndarray):
+    """``quantize`` with the stochastic-rounding draw of element ``(i, j)`` taken at ``index[i, j]`` (its
+    position in the tensor it is a copy of; negative = structural zero, no draw)."""
+    assert x.dtype == np.float32 and x.ndim == 2 and index.shape == x.shape
+    x = np.ascontiguousarray(x)
+    index = np.ascontiguousarray(index, dtype=np.int64)
+    d0, d1 = x.shape
+    k, rows = (d1, d0) if contract_axis == 1 else (d0, d1)
+    q = np.zeros((rows, k), dtype=np.int16)
+    s = np.zeros((rows, n_blocks(k, fmt.block)), dtype=np.int8)
+    cf = fmt._c()
+    rc = lib().oracle_quantize_indexed(_ptr(x), d0, d1, d1, contract_axis, ctypes.byref(cf), _ptr(index), _ptr(q), _ptr(s))
+    if rc:
+        raise ValueError(f"oracle_quantize_indexed failed: {rc}")
+    return q, s
+
+
 def quantize_conv_weights(w: np.ndarray, taps: int, contract_axis: int, fmt: Format):
     """Convolution weights ``w [taps * c_in][c_out]`` with one exponent per tile of ``t`` input maps x ``t``
     output maps across all filter taps (``fmt.tile``). Returns ``(q, s)`` laid out like ``quantize``."""
@@ -284,3 +303,10 @@ def im2col(x: np.ndarray, kh: int, kw: int, pad: int) -> np.ndarray:
                     if 0 <= ix < w:
                         out[:, oy, ox, i, j, :] = x[:, iy, ix, :]
     return out.reshape(n * ho * wo, kh * kw * c)
+
+
+def im2col_index(n: int, h: int, w: int, c: int, kh: int, kw: int, pad: int) -> np.ndarray:
+    """For every element of ``im2col(x, kh, kw, pad)`` the row-major index in ``x [n][h][w][c]`` of the
+    activation it is a copy of, -1 for the zeros outside the image (int64, same shape as the im2col matrix)."""
+    ids = np.arange(1, n * h * w * c + 1, dtype=np.int64).reshape(n, h, w, c)
+    return im2col(ids, kh, kw, pad) - 1

@@ -234,6 +234,33 @@ int oracle_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int cont
 }
 
 // ---------------------------------------------------------------------------------------
+// oracle_quantize for a matrix whose elements are copies of the elements of another tensor (the im2col
+// matrix of a convolution, Sec. 5.1): exactly the same two passes, but under stochastic rounding element
+// (i, j) takes the draw of index[i * d1 + j] - its position in the tensor it was copied from - so that every
+// copy of an activation uses that activation's draw; a negative index marks a structural zero (padding),
+// which needs no draw. With index[i * d1 + j] = i * d1 + j this is oracle_quantize.
+// ---------------------------------------------------------------------------------------
+int oracle_quantize_indexed(const float* x, int64_t d0, int64_t d1, int64_t ld, int contract_axis,
+                            const oracle_format* f, const int64_t* index, int16_t* q, int8_t* s) {
+    if (!index) return -1;
+    oracle_format g = *f;
+    g.rounding = 0;                                   // pass 1 (exponents) does not depend on the rounding mode
+    int rc = oracle_quantize(x, d0, d1, ld, contract_axis, &g, q, s);
+    if (rc || f->rounding == 0) return rc;
+    const int m = f->mant_bits;
+    const int64_t k = contract_axis == 1 ? d1 : d0, rows = contract_axis == 1 ? d0 : d1;
+    const int64_t b = f->block == 0 ? (k > 0 ? k : 1) : f->block, nkb = (k + b - 1) / b;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t kk = 0; kk < k; ++kk) {
+            const int64_t i = contract_axis == 1 ? r : kk, j = contract_axis == 1 ? kk : r;
+            const int64_t L = index[i * d1 + j];
+            const uint32_t rnd = L < 0 ? 0u : oracle_sr_draw(f->seed, f->stream_id, (uint64_t)L);
+            q[r * k + kk] = (int16_t)oracle_round_sr(x[i * ld + j], s[r * nkb + kk / b], m, rnd);
+        }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------------------
 // Weights of a convolution layer (Sec. 5.1, last sentence: for convolutional layers the two outer,
 // feature-map dimensions of the weights are tiled). The weights are w[tap][ci][co], tap = (filter row,
 // filter column), stored as the matrix [taps * c_in][c_out] that the convolution GEMM multiplies by.

@@ -51,3 +51,41 @@ def test_blocks_of_the_gathered_matrix_are_blocks_of_the_pixels():
                         assert np.array_equal(qc[:, oy, ox, i, j], qp[:, iy, ix]) and np.array_equal(sc[:, oy, ox, i, j], sp[:, iy, ix])
                     else:
                         assert not qc[:, oy, ox, i, j].any() and (sc[:, oy, ox, i, j] == -63).all()
+
+
+def test_indexed_quantiser_reduces_to_the_plain_one_and_draws_by_the_given_index():
+    """oracle.quantize_indexed: with the identity index it is oracle.quantize; otherwise every element is
+    rounded with the draw of the index it names (the scalar functions are pinned on their own)."""
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal((12, 20)) * np.exp(rng.standard_normal((12, 20)))).astype(np.float32)
+    fmt = oracle.Format(mant_bits=8, block=4, rounding=1, seed=21, stream_id=5)
+    ident = np.arange(x.size, dtype=np.int64).reshape(x.shape)
+    for axis in (0, 1):
+        q, s = oracle.quantize_indexed(x, axis, fmt, ident)
+        q_ref, s_ref = oracle.quantize(x, axis, fmt)
+        assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
+    perm = rng.permutation(x.size).astype(np.int64).reshape(x.shape)
+    perm[0, 0] = -1
+    x[0, 0] = 0.0                                         # a structural zero: no draw, stays zero
+    q, s = oracle.quantize_indexed(x, 0, fmt, perm)       # q [20][12], blocks of 4 down the columns of x
+    _, s_plain = oracle.quantize(x, 0, fmt)
+    assert np.array_equal(s, s_plain)                     # exponents do not depend on the draws
+    assert q[0, 0] == 0
+    for (i, j) in ((3, 7), (11, 19), (5, 0)):
+        r = oracle.sr_draw(21, 5, int(perm[i, j]))
+        assert q[j, i] == oracle.round_sr(x[i, j], int(s[j, i // 4]), 8, r)
+
+
+def test_im2col_index_names_the_activation_each_entry_copies():
+    n, h, w, c = 2, 5, 4, 3
+    x = np.random.default_rng(4).standard_normal((n, h, w, c)).astype(np.float32)
+    cols = oracle.im2col(x, 3, 3, 1)
+    idx = oracle.im2col_index(n, h, w, c, 3, 3, 1)
+    assert idx.shape == cols.shape
+    flat = x.reshape(-1)
+    inside = idx >= 0
+    assert np.array_equal(cols[inside], flat[idx[inside]])
+    assert (cols[~inside] == 0).all() and (~inside).sum() > 0
+    # every interior activation appears once per tap
+    counts = np.bincount(idx[inside], minlength=flat.size).reshape(n, h, w, c)
+    assert (counts[:, 1:-1, 1:-1, :] == 9).all()
