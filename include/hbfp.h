@@ -207,7 +207,9 @@ HBFP_API int hbfp_im2col_packed(const void* mant_x, const int8_t* exps_x, int64_
  * the n*h*w output pixels, so the A operand is cols^T with blocks of fmt->block consecutive pixels
  * along each (tap, channel) row. This call converts it straight from the FP32 activations x
  * [n][h][w][c] (16-byte aligned, c % 4 == 0): rows = kh*kw*c, k = n*h*w, bit-identical to
- * hbfp_quantize(im2col matrix, contract_axis 0). Supported: nearest-even rounding, an output as
+ * hbfp_quantize(im2col matrix, contract_axis 0) under nearest-even rounding; under stochastic rounding
+ * every entry takes the draw of the activation it is a copy of (keyed by its index in x, as in
+ * hbfp_im2col_packed). Supported: an output as
  * large as the input (2 pad == kh - 1 == kw - 1), blocks of whole image rows (block in {16, 32, 64,
  * 128}, block % w == 0, h*w % block == 0), w a power of two >= 4; anything else returns
  * HBFP_ERR_UNSUPPORTED (convert the im2col matrix instead). mant / exps: buffers of the

@@ -1441,10 +1441,8 @@ int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t 
                        const hbfp_format* f, int8_t* mant, int8_t* exps, cudaStream_t st) {
     if (f->tile != 0 || f->block <= 0) return HBFP_ERR_INVALID_ARG;
     const int64_t b = f->block;
-    // Nearest-even only: the oracle numbers stochastic-rounding draws by the position in the matrix it is
-    // given, and this operand's matrix never exists (the kernel's SR instantiation, which would draw by the
-    // position in the activation tensor, is not launched).
-    if (f->rounding != 0) return HBFP_ERR_UNSUPPORTED;
+    // Under stochastic rounding every entry takes the draw of the activation it is a copy of (its index in
+    // x [n][h][w][c]): the matrix this operand is the conversion of never exists.
     // same-size output, blocks of whole image rows that do not straddle images
     if (2 * pad != kh - 1 || 2 * pad != kw - 1) return HBFP_ERR_UNSUPPORTED;
     if (!(b == 16 || b == 32 || b == 64 || b == 128) || b % w != 0 || w < 4 || (w & (w - 1)) != 0 || (h * w) % b != 0 ||
@@ -1470,7 +1468,8 @@ int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t 
     } while (0)
 #define HBFP_COLS_LAUNCH(PL, NPX)                                                 \
     do {                                                                          \
-        HBFP_COLS_LAUNCH2(PL, NPX, false);                                        \
+        if (p.rounding) HBFP_COLS_LAUNCH2(PL, NPX, true);                         \
+        else HBFP_COLS_LAUNCH2(PL, NPX, false);                                   \
     } while (0)
     if (L.planes == 1) {
         if (b == 16) HBFP_COLS_LAUNCH(1, 4); else if (b == 32) HBFP_COLS_LAUNCH(1, 8); else if (b == 64) HBFP_COLS_LAUNCH(1, 16); else HBFP_COLS_LAUNCH(1, 32);

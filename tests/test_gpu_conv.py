@@ -131,12 +131,19 @@ def test_backward_weight_operand_refuses_what_it_does_not_cover(hb):
     assert e.value.code == hb.ERR_UNSUPPORTED
 
 
-def test_backward_weight_operand_is_nearest_even_only(hb):
-    import torch
-    x = torch.zeros((1, 8, 8, 16), device="cuda")
-    with pytest.raises(hb.HbfpError) as e:
-        hb.im2col_packed_t(x, 3, 3, 1, hb.Format(mant_bits=8, block=16, rounding=1))
-    assert e.value.code == hb.ERR_UNSUPPORTED
+@pytest.mark.parametrize("n,hw,c,b,m", [(2, 32, 64, 64, 8), (3, 16, 32, 128, 12), (2, 8, 16, 16, 8), (1, 16, 128, 32, 6)])
+def test_backward_weight_operand_under_stochastic_rounding(hb, n, hw, c, b, m):
+    """Every entry of the operand is a copy of an activation and is rounded with that activation's draw
+    (index in x): the oracle's indexed quantiser on the im2col matrix, bit for bit."""
+    x = wl.draw("half_normal", (n * hw * hw, c), seed=87).reshape(n, hw, hw, c)
+    x *= np.exp(wl.draw("normal", (n * hw * hw, 1), seed=88)).reshape(n, hw, hw, 1).astype(np.float32)
+    fd = dict(mant_bits=m, block=b, rounding=1, seed=13, stream_id=4)
+    pa = hb.im2col_packed_t(to_dev(x), 3, 3, 1, gfmt(fd))
+    assert hb.device_status() == 0
+    cols = oracle.im2col(x, 3, 3, 1)
+    q_ref, s_ref = oracle.quantize_indexed(cols, 0, ofmt(fd), oracle.im2col_index(n, hw, hw, c, 3, 3, 1))
+    q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
+    assert np.array_equal(s, s_ref) and np.array_equal(q, q_ref)
 
 
 IMPLICIT_CASES = [
@@ -222,3 +229,16 @@ def test_convolution_with_tiled_weights_end_to_end(hb):
     qb, sb = oracle.quantize_conv_weights(wt, 9, 0, ofmt(fw))
     ref = oracle.gemm(qa, sa, qb, sb, c)
     assert np.array_equal(Y, ref["c_seq"])
+
+
+def test_gathered_operand_under_stochastic_rounding_takes_each_activations_draw(hb):
+    """Forward operand under stochastic rounding: the pixels were converted with draws keyed by their index in
+    the activation tensor, so the gathered operand is the oracle's indexed conversion of the im2col matrix."""
+    n, h, w, c = 2, 8, 8, 32
+    x = wl.draw("half_normal", (n * h * w, c), seed=89).reshape(n, h, w, c)
+    fd = dict(mant_bits=8, block=c, rounding=1, seed=17, stream_id=6)
+    px = hb.quantize(to_dev(x.reshape(n * h * w, c)), 1, gfmt(fd))
+    pa = hb.im2col_packed(px, n, h, w, c, 3, 3, 1)
+    q_ref, s_ref = oracle.quantize_indexed(oracle.im2col(x, 3, 3, 1), 1, ofmt(fd), oracle.im2col_index(n, h, w, c, 3, 3, 1))
+    q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
+    assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
