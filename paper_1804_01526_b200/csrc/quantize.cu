@@ -591,6 +591,213 @@ tile_kernel(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, i
     write_tile_views<PLANES>(qt, tp, hi, wj, i0, j0, u, v, s + sh, sh, tv, tid);
 }
 
+// Full tiles of 32, 64 or 128 (the tile is its own padded width), aligned rows: the same arithmetic as
+// tile_kernel with far fewer instructions per weight. A thread keeps its groups of eight weights in registers
+// between the maximum and the rounding pass (no FP32 tile in shared memory); the rounded words go to a 16-bit
+// tile in shared memory once, from which view c1 leaves as 8-byte pieces cut by byte permutes and view c0 as
+// the byte-transposes of 4 x 4 blocks (eight permutes per block) instead of one shared-memory load, shift and
+// mask per byte. ROWS4 = 4 x 4 blocks stacked per thread for view c0 (wider stores per output row).
+template <int MODE, int PLANES, int TP>
+__global__ void __launch_bounds__(256)
+tile_kernel_full(const float* __restrict__ src, int64_t ld, int64_t d0, int64_t d1, QParams p,
+                 int16_t* __restrict__ wide, int8_t* __restrict__ grid, int64_t grid_ld, TileViews tv) {
+    constexpr int G = TP / 8;                          // groups of eight per tile row
+    constexpr int NITEMS = TP * G;                     // groups per tile
+    constexpr int ITEMS = (NITEMS + 255) / 256;        // per thread
+    constexpr int QP = TP + 8;                         // halfword pitch of qt: rows stay 16-byte aligned
+    __shared__ __align__(16) int16_t qt[TP * QP];
+    __shared__ uint32_t s_am[8];
+    __shared__ int s_exp;
+    const int tid = threadIdx.x, lane = tid & 31, wrow = tid >> 5;
+    const int64_t u = blockIdx.y, v = blockIdx.x;
+    const int64_t i0 = u * TP, j0 = v * TP;
+    const int wbits = MODE == 3 ? p.m : 16, wqmax = MODE == 3 ? p.qmax : 32767;
+    const int sh = MODE == 3 ? 0 : 16 - p.m;
+    const int half = sh > 0 ? 1 << (sh - 1) : 0;
+    const int w_hi = ((p.qmax + 1) << sh) - half - 1, w_lo = -(p.qmax << sh) - half;
+    const uint32_t w_hi2 = ((uint32_t)w_hi & 0xFFFFu) * 0x10001u, w_lo2 = ((uint32_t)w_lo & 0xFFFFu) * 0x10001u;
+    const uint32_t half2 = (uint32_t)half * 0x10001u;
+    auto stored_pair = [&](uint32_t h) { return MODE == 3 ? h : __vadd2(__vmaxs2(__vmins2(h, w_hi2), w_lo2), half2); };
+    int s;
+    if (MODE == 2) {
+        s = grid[u * grid_ld + v];
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            const int item = tid + 256 * k;
+            if (NITEMS % 256 == 0 || item < NITEMS) {
+                const int ii = item / G, gj = item - ii * G;
+                const uint4 q8 = *reinterpret_cast<const uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj);
+                *reinterpret_cast<uint4*>(qt + ii * QP + 8 * gj) = make_uint4(stored_pair(q8.x), stored_pair(q8.y), stored_pair(q8.z), stored_pair(q8.w));
+            }
+        }
+    } else {
+        const float old_scale = MODE == 1 ? pow2f(grid[u * grid_ld + v]) : 0.f;
+        // the FP32 groups of the tile are requested before anything waits for them; for an update the wide
+        // words follow, combined as fl32(wide * 2^s + delta) with one rounding
+        float4 a[ITEMS], b[ITEMS];
+        uint32_t am = 0;
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            const int item = tid + 256 * k;
+            a[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            b[k] = a[k];
+            if (NITEMS % 256 == 0 || item < NITEMS) {
+                const int ii = item / G, gj = item - ii * G;
+                const float4* sp = reinterpret_cast<const float4*>(src + (i0 + ii) * ld + j0 + 8 * gj);
+                a[k] = __ldcs(sp);
+                b[k] = __ldcs(sp + 1);
+            }
+        }
+        if (MODE == 1) {
+#pragma unroll
+            for (int k = 0; k < ITEMS; ++k) {
+                const int item = tid + 256 * k;
+                if (NITEMS % 256 == 0 || item < NITEMS) {
+                    const int ii = item / G, gj = item - ii * G;
+                    const uint4 q8 = *reinterpret_cast<const uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj);
+                    a[k].x = __fadd_rn(__fmul_rn((float)(int16_t)(q8.x & 0xFFFFu), old_scale), a[k].x);
+                    a[k].y = __fadd_rn(__fmul_rn((float)(int16_t)(q8.x >> 16), old_scale), a[k].y);
+                    a[k].z = __fadd_rn(__fmul_rn((float)(int16_t)(q8.y & 0xFFFFu), old_scale), a[k].z);
+                    a[k].w = __fadd_rn(__fmul_rn((float)(int16_t)(q8.y >> 16), old_scale), a[k].w);
+                    b[k].x = __fadd_rn(__fmul_rn((float)(int16_t)(q8.z & 0xFFFFu), old_scale), b[k].x);
+                    b[k].y = __fadd_rn(__fmul_rn((float)(int16_t)(q8.z >> 16), old_scale), b[k].y);
+                    b[k].z = __fadd_rn(__fmul_rn((float)(int16_t)(q8.w & 0xFFFFu), old_scale), b[k].z);
+                    b[k].w = __fadd_rn(__fmul_rn((float)(int16_t)(q8.w >> 16), old_scale), b[k].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            const float e8[8] = {a[k].x, a[k].y, a[k].z, a[k].w, b[k].x, b[k].y, b[k].z, b[k].w};
+            am = max(am, amax8_bits(e8));
+        }
+        for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        if (lane == 0) s_am[wrow] = am;
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t m8 = 0;
+            for (int i = 0; i < 8; ++i) m8 = max(m8, s_am[i]);
+            s_exp = block_exponent(m8, wbits, p.exp_mode);
+            if (grid) grid[u * grid_ld + v] = (int8_t)s_exp;
+        }
+        __syncthreads();
+        s = s_exp;
+        const uint32_t qm = qmax_pair(wqmax), nqm = neg_qmax_pair(wqmax);
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            const int item = tid + 256 * k;
+            if (NITEMS % 256 == 0 || item < NITEMS) {
+                const int ii = item / G, gj = item - ii * G;
+                const float e8[8] = {a[k].x, a[k].y, a[k].z, a[k].w, b[k].x, b[k].y, b[k].z, b[k].w};
+                uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                if (p.rounding == 1) w = draws_of_group(p, (uint64_t)((i0 + ii) * d1 + j0 + 8 * gj) >> 3);
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+                uint32_t h[4];
+                if (MODE == 3) {
+                    const float sc = pow2f(p.rounding == 1 ? 16 - s : -s);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        h[j] = p.rounding == 1 ? round_sr_pair(e8[2 * j], e8[2 * j + 1], sc, ww[j], qm, nqm)
+                                               : round_rne_pair(e8[2 * j], e8[2 * j + 1], sc, qm, nqm);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        int q0, q1;
+                        if (p.rounding == 0) {
+                            q0 = round_rne(e8[2 * j], s, 32767);
+                            q1 = round_rne(e8[2 * j + 1], s, 32767);
+                        } else {
+                            q0 = round_sr_wide(e8[2 * j], s, ww[j] & 0xFFFFu);
+                            q1 = round_sr_wide(e8[2 * j + 1], s, ww[j] >> 16);
+                        }
+                        h[j] = ((uint32_t)q0 & 0xFFFFu) | ((uint32_t)q1 << 16);
+                    }
+                }
+                *reinterpret_cast<uint4*>(qt + ii * QP + 8 * gj) = make_uint4(stored_pair(h[0]), stored_pair(h[1]), stored_pair(h[2]), stored_pair(h[3]));
+                if (MODE != 3) *reinterpret_cast<uint4*>(wide + (i0 + ii) * d1 + j0 + 8 * gj) = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+        }
+    }
+    if (tv.mant_c0 == nullptr && tv.mant_c1 == nullptr) return;
+    __syncthreads();
+    // Bytes of the views from pairs of stored halfwords: plane 0 takes bits [sh + 4 (PLANES - 1), + 8) of each
+    // halfword, plane 1 the four bits below; the masks remove what a 32-bit shift drags across the halfwords.
+    const int sh_hi = sh + (PLANES == 2 ? 4 : 0);
+    auto bytes4 = [&](uint32_t w0, uint32_t w1, int k, uint32_t mask) {
+        return __byte_perm((w0 >> k) & mask, (w1 >> k) & mask, 0x6420);
+    };
+    const int s_view = s + sh;
+    // view c1: row i0 + ii, bytes [v TP + 8 gj, + 8)
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        const int item = tid + 256 * k;
+        if (NITEMS % 256 == 0 || item < NITEMS) {
+            const int ii = item / G, gj = item - ii * G;
+            const uint4 q8 = *reinterpret_cast<const uint4*>(qt + ii * QP + 8 * gj);
+            int8_t* dst = tv.mant_c1 + (i0 + ii) * tv.kst1 + v * TP + 8 * gj;
+            *reinterpret_cast<uint2*>(dst) = make_uint2(bytes4(q8.x, q8.y, sh_hi, 0x00ff00ffu), bytes4(q8.z, q8.w, sh_hi, 0x00ff00ffu));
+            if (PLANES == 2)
+                *reinterpret_cast<uint2*>(dst + tv.ps1) = make_uint2(bytes4(q8.x, q8.y, sh, 0x000f000fu), bytes4(q8.z, q8.w, sh, 0x000f000fu));
+        }
+    }
+    // view c0: row j0 + jj, bytes [u TP + g, ...): blocks of 4 columns x (4 ROWS4) rows of qt, byte-transposed
+    constexpr int ROWS4 = TP >= 64 ? 4 : 1;                            // 16- or 4-byte stores
+    constexpr int NBLK = (TP / 4) * (TP / (4 * ROWS4));
+#pragma unroll
+    for (int k = 0; k < (NBLK + 255) / 256; ++k) {
+        const int e = tid + 256 * k;
+        if (NBLK % 256 == 0 || e < NBLK) {
+            const int jj = (e % (TP / 4)) * 4, g = (e / (TP / 4)) * 4 * ROWS4;
+            uint32_t out[PLANES][4][ROWS4];
+#pragma unroll
+            for (int rb = 0; rb < ROWS4; ++rb) {
+                uint2 r[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r[i] = *reinterpret_cast<const uint2*>(qt + (g + 4 * rb + i) * QP + jj);
+#pragma unroll
+                for (int pl = 0; pl < PLANES; ++pl) {
+                    const int kk = pl == 0 ? sh_hi : sh;
+                    const uint32_t mask = pl == 0 ? 0x00ff00ffu : 0x000f000fu;
+                    const uint32_t R0 = bytes4(r[0].x, r[0].y, kk, mask), R1 = bytes4(r[1].x, r[1].y, kk, mask);
+                    const uint32_t R2 = bytes4(r[2].x, r[2].y, kk, mask), R3 = bytes4(r[3].x, r[3].y, kk, mask);
+                    const uint32_t t0 = __byte_perm(R0, R1, 0x5140), t1 = __byte_perm(R2, R3, 0x5140);
+                    const uint32_t t2 = __byte_perm(R0, R1, 0x7362), t3 = __byte_perm(R2, R3, 0x7362);
+                    out[pl][0][rb] = __byte_perm(t0, t1, 0x5410);
+                    out[pl][1][rb] = __byte_perm(t0, t1, 0x7632);
+                    out[pl][2][rb] = __byte_perm(t2, t3, 0x5410);
+                    out[pl][3][rb] = __byte_perm(t2, t3, 0x7632);
+                }
+            }
+#pragma unroll
+            for (int pl = 0; pl < PLANES; ++pl)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    int8_t* dst = tv.mant_c0 + pl * tv.ps0 + (j0 + jj + c) * tv.kst0 + u * TP + g;
+                    if (ROWS4 == 4) *reinterpret_cast<uint4*>(dst) = make_uint4(out[pl][c][0], out[pl][c][1], out[pl][c][2 % ROWS4], out[pl][c][3 % ROWS4]);
+                    else if (ROWS4 == 2) *reinterpret_cast<uint2*>(dst) = make_uint2(out[pl][c][0], out[pl][c][1 % ROWS4]);
+                    else *reinterpret_cast<uint32_t*>(dst) = out[pl][c][0];
+                }
+        }
+    }
+    // replicated exponents, and the row tails beyond the last tile
+    if (tid < TP) {
+        tv.exps_c1[v * tv.rs1 + i0 + tid] = (int8_t)s_view;
+        tv.exps_c0[u * tv.rs0 + j0 + tid] = (int8_t)s_view;
+    }
+    if (v == tv.nkb1 - 1)
+        for (int64_t e = tid; e < (int64_t)TP * ((tv.kst1 - tv.nkb1 * TP) / 4); e += 256) {
+            const int64_t per = (tv.kst1 - tv.nkb1 * TP) / 4, ii = e / per, o = tv.nkb1 * TP + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(tv.mant_c1 + (i0 + ii) * tv.kst1 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(tv.mant_c1 + tv.ps1 + (i0 + ii) * tv.kst1 + o) = 0;
+        }
+    if (u == tv.nkb0 - 1)
+        for (int64_t e = tid; e < (int64_t)TP * ((tv.kst0 - tv.nkb0 * TP) / 4); e += 256) {
+            const int64_t per = (tv.kst0 - tv.nkb0 * TP) / 4, jj = e / per, o = tv.nkb0 * TP + (e % per) * 4;
+            *reinterpret_cast<uint32_t*>(tv.mant_c0 + (j0 + jj) * tv.kst0 + o) = 0;
+            if (PLANES == 2) *reinterpret_cast<uint32_t*>(tv.mant_c0 + tv.ps0 + (j0 + jj) * tv.kst0 + o) = 0;
+        }
+}
+
 // ------------------------------------------------------------------------------ generic two-pass path
 
 // Element (r, kk) of the operand view: r = line, kk = position along the contraction axis.
@@ -1349,6 +1556,17 @@ int launch_tiles(const float* src, int64_t ld, int64_t d0, int64_t d1, const hbf
                       (MODE == 3 || (reinterpret_cast<uintptr_t>(wide) & 15) == 0);
     const size_t smem = (size_t)t * (t + 4) * sizeof(float) + (size_t)tp * (tp + 2) * sizeof(int16_t);
     const dim3 grid_dim((unsigned)nv, (unsigned)nu);
+    // full tiles of 32 / 64 / 128, both views or none, narrow bits cut by 32-bit shifts (see tile_kernel_full)
+    const int sh_full = MODE == 3 ? 0 : 16 - p.m;
+    const bool full = fast && t == tp && (d0 % t) == 0 && (d1 % t) == 0 && ((mant_c0 != nullptr) == (mant_c1 != nullptr)) &&
+                      (!mant_c0 || (exps_c0 && exps_c1)) && sh_full + (L0.planes == 2 ? 4 : 0) <= 8;
+    if (full) {
+#define HBFP_TILE_FULL(PLANES, TP) tile_kernel_full<MODE, PLANES, TP><<<grid_dim, 256, 0, st>>>(src, ld, d0, d1, p, wide, grid, nv, tv)
+        if (L0.planes == 1) { if (t == 32) HBFP_TILE_FULL(1, 32); else if (t == 64) HBFP_TILE_FULL(1, 64); else HBFP_TILE_FULL(1, 128); }
+        else { if (t == 32) HBFP_TILE_FULL(2, 32); else if (t == 64) HBFP_TILE_FULL(2, 64); else HBFP_TILE_FULL(2, 128); }
+#undef HBFP_TILE_FULL
+        return launch_status();
+    }
 #define HBFP_TILE_LAUNCH(PLANES, FAST)                                                                                       \
     do {                                                                                                                     \
         HBFP_CUDA_OK(cudaFuncSetAttribute(tile_kernel<MODE, PLANES, FAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
