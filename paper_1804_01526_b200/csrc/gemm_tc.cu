@@ -53,7 +53,9 @@ constexpr int THREADS = 32 * (CONTROL_WARPS + RESCALE_WARPS);
 constexpr int REGS_RESCALE = 216, REGS_CONTROL = 72;
 static_assert(128 * REGS_CONTROL + 32 * RESCALE_WARPS * REGS_RESCALE <= 384 * 168, "register split");
 
-template <int N_TILE, int PLANES>
+// TSTORE: the output tile leaves through shared memory and TMA stores (one 32 x 32 FP32 box per rescale warp
+// and 32 columns, double-buffered) instead of per-lane stores from registers; takes 64 KB from the stages.
+template <int N_TILE, int PLANES, bool TSTORE = false>
 struct Cfg {
     // accumulator parts per group; two planes: [hi.hi | hi.lo + lo.hi | lo.lo], each N_TILE columns
     static constexpr int PARTS = PLANES == 1 ? 1 : 3;
@@ -68,9 +70,11 @@ struct Cfg {
     static constexpr int TABLE_SLOTS = 2 * GROUPS;
     static constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
     static constexpr int TABLE_BYTES = 4 * TABLE_SLOTS * TABLE_SLOT_WORDS;
-    static constexpr int STAGES_RAW = (232448 - 2048 - TABLE_BYTES) / (MANT_STAGE + EXP_STAGE);
+    static constexpr int OUT_BUF = 32 * 32 * 4;                    // one 32-row x 32-column FP32 box
+    static constexpr int OUT_BYTES = TSTORE ? RESCALE_WARPS * 2 * OUT_BUF : 0;
+    static constexpr int STAGES_RAW = (232448 - 2048 - TABLE_BYTES - OUT_BYTES - (TSTORE ? 1024 : 0)) / (MANT_STAGE + EXP_STAGE);
     static constexpr int STAGES = STAGES_RAW > 8 ? 8 : STAGES_RAW;
-    static constexpr int SMEM = 1024 /*align slack*/ + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + 1024 /*barriers*/;
+    static constexpr int SMEM = 1024 /*align slack*/ + STAGES * (MANT_STAGE + EXP_STAGE) + (TSTORE ? 1024 : 0) + OUT_BYTES + TABLE_BYTES + 1024 /*barriers*/;
     static constexpr uint32_t TX_BYTES = MANT_STAGE + EXP_STAGE;
     static_assert(GROUPS >= 2, "need two accumulator groups to overlap MMA and rescale");
     static_assert(STAGES >= 3, "pipeline too shallow");
@@ -170,9 +174,9 @@ struct MmaArgs {
 
 // The loop of the single MMA-issuing thread. LNG: blocks of 128 bytes or more (one block step set per
 // stage, SPB = 4); otherwise 128 / (32 SPB) blocks of SPB steps share a stage.
-template <int N_TILE, int PLANES, bool MAGIC, bool LNG, int SPB>
+template <int N_TILE, int PLANES, bool MAGIC, bool LNG, int SPB, bool TSTORE>
 __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh, const MmaArgs& a) {
-    using C = Cfg<N_TILE, PLANES>;
+    using C = Cfg<N_TILE, PLANES, TSTORE>;      // the kernel's configuration: same ring sizes
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS;
     constexpr int BPS = LNG ? 1 : 4 / SPB;
     // Two planes: the hi and lo planes of B lie back to back in a stage, so one MMA of twice the width
@@ -264,13 +268,13 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
 
 // ------------------------------------------------------------------------------ kernel
 
-template <int N_TILE, int PLANES, bool MAGIC, bool DUMP>
+template <int N_TILE, int PLANES, bool MAGIC, bool DUMP, bool TSTORE>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
                const __grid_constant__ CUtensorMap mapEA, const __grid_constant__ CUtensorMap mapEB,
-               const Problem p) {
-    using C = Cfg<N_TILE, PLANES>;
+               const __grid_constant__ CUtensorMap mapC, const Problem p) {
+    using C = Cfg<N_TILE, PLANES, TSTORE>;
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS, TSLOTS = C::TABLE_SLOTS;
     constexpr int COLS_PER_WARP = N_TILE / COL_GROUPS;  // warps that share a lane quarter split the columns
     static_assert(!(MAGIC && PLANES != 1), "the biased-accumulator path is for one-plane operands");
@@ -280,7 +284,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
     const uint32_t mant_base = base;                                        // STAGES x MANT_STAGE, 1024-aligned
     const uint32_t exp_base = mant_base + STAGES * C::MANT_STAGE;           // STAGES x EXP_STAGE
-    const uint32_t table_off = STAGES * (C::MANT_STAGE + C::EXP_STAGE);
+    const uint32_t out_off = (STAGES * (C::MANT_STAGE + C::EXP_STAGE) + 1023u) & ~1023u;   // output boxes (TSTORE), 1024-aligned
+    const uint32_t table_off = out_off + C::OUT_BYTES;
     uint32_t* tables = reinterpret_cast<uint32_t*>(base_ptr + table_off);   // [slot][N_TILE column scales | 128 row scales]
     const uint32_t bar_off = table_off + C::TABLE_BYTES;
     const uint32_t bars = base + bar_off;
@@ -367,9 +372,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             // -------------------------------------------------------------- MMA issuer
             if (lane == 0) {
                 const MmaArgs ma{full_bar, empty_bar, tfull_bar, tempty_bar, done_bar, mant_base, tmem_base, total_work, abort_flag};
-                if (sh.lng) mma_issue_loop<N_TILE, PLANES, MAGIC, true, 4>(p, sh, ma);
-                else if (sh.spb == 2) mma_issue_loop<N_TILE, PLANES, MAGIC, false, 2>(p, sh, ma);
-                else mma_issue_loop<N_TILE, PLANES, MAGIC, false, 1>(p, sh, ma);
+                if (sh.lng) mma_issue_loop<N_TILE, PLANES, MAGIC, true, 4, TSTORE>(p, sh, ma);
+                else if (sh.spb == 2) mma_issue_loop<N_TILE, PLANES, MAGIC, false, 2, TSTORE>(p, sh, ma);
+                else mma_issue_loop<N_TILE, PLANES, MAGIC, false, 1, TSTORE>(p, sh, ma);
             }
         } else if (warp == TABLE_WARP) {
             // -------------------------------------------------------------- scale-table builder
@@ -464,7 +469,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
         if (lane == 0)
             for (int g = 0; g < GROUPS; ++g) mbar_arrive(tempty_bar + 8 * g);
 
-        uint32_t g = 0, gph = 0, slot = 0, blk = 0;
+        uint32_t g = 0, gph = 0, slot = 0, blk = 0, out_turn = 0;
         bool ok = true;
         for (int wi = blockIdx.x; ok && wi < total_work; wi += gridDim.x) {
             const Work w = get_work(p, wi);
@@ -564,7 +569,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             // ---- store the tile (or this split's partial tile)
             float* dst = p.splits > 1 ? p.partial + (int64_t)w.split * p.M * p.ldp : p.C;
             const int64_t ldd = p.splits > 1 ? p.ldp : p.ldc;
-            if (dst != nullptr && gi < p.M) {
+            if (TSTORE) {
+                // Each lane writes its row's 32 columns into a 128B-swizzled box (16-byte piece j of row r at
+                // piece j ^ (r & 7): conflict-free), one lane hands the box to the copy engine, and the warp goes
+                // on; a box is reused once the copy engine has read the one sent two boxes earlier. The copy
+                // clips what lies beyond M or N.
+#pragma unroll
+                for (int cb = 0; cb < COLS_PER_WARP / 32; ++cb) {
+                    const uint32_t buf = base + out_off + (uint32_t)((rwarp * 2 + (out_turn & 1)) * C::OUT_BUF);
+                    if (out_turn >= 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t at = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v2.b64 [%0], {%1, %2};" ::"r"(at), "l"(acc2[cb * 16 + 2 * j]), "l"(acc2[cb * 16 + 2 * j + 1]) : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                                     ::"l"(reinterpret_cast<uint64_t>(&mapC)), "r"(buf), "r"(n0 + col0 + 32 * cb), "r"(w.m0 + quarter * 32) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    ++out_turn;
+                }
+            } else if (dst != nullptr && gi < p.M) {
                 float* rowp = dst + gi * ldd + n0 + col0;
                 // full 32-byte sectors per lane where the row pitch allows it (each lane owns a row)
                 const bool wide = (ldd & 7) == 0 && (reinterpret_cast<uintptr_t>(dst) & 31) == 0;
@@ -593,6 +622,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     }
 
     // ------------------------------------------------------------------ teardown
+    if (TSTORE) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // this thread's output boxes have been written
     tc_fence_before();
     __syncthreads();
     if (warp == MMA_WARP) {
@@ -614,10 +644,23 @@ __global__ void splitk_reduce(const float* __restrict__ partial, int splits, int
 
 // ------------------------------------------------------------------------------ host side
 
-template <int N_TILE, int PLANES, bool MAGIC, bool DUMP>
+// 2-D FP32 tensor [rows][cols] with pitch ld (elements); box = 32 columns x 32 rows, 128B-swizzled.
+int make_map_out(CUtensorMap* m, float* ptr, uint64_t cols, uint64_t rows, uint64_t ld) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return HBFP_ERR_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, ptr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? HBFP_OK : HBFP_ERR_CUDA;
+}
+
+template <int N_TILE, int PLANES, bool MAGIC, bool DUMP, bool TSTORE = false>
 int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t st) {
-    using C = Cfg<N_TILE, PLANES>;
-    CUtensorMap mA0, mA1, mB0, mB1, mEA, mEB;
+    using C = Cfg<N_TILE, PLANES, TSTORE>;
+    CUtensorMap mA0, mA1, mB0, mB1, mEA, mEB, mC;
     int rc;
     rc = make_map(&mA0, a.mant, a.L.kst, a.L.rows, a.L.kst, STAGE_K, TILE_M, true);
     if (rc) return rc;
@@ -635,17 +678,22 @@ int launch_cfg(const Problem& p, const Packed& a, const Packed& b, cudaStream_t 
     if (rc) return rc;
     rc = make_map(&mEB, b.exps, b.L.rs, b.L.nkb, b.L.rs, N_TILE, 4, false);
     if (rc) return rc;
+    mC = mEB;                                                  // unused unless TSTORE
+    if (TSTORE) {
+        rc = make_map_out(&mC, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.ldc);
+        if (rc) return rc;
+    }
     // the attribute belongs to the device: set once per device, not once per process
     static bool attr_set[MAX_DEVICES] = {};
     const int dev = current_device();
     if (dev < 0) return HBFP_ERR_CUDA;
     if (!attr_set[dev]) {
-        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP, TSTORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM));
         attr_set[dev] = true;
     }
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     const int grid = (int)(work < sm_count() ? work : sm_count());
-    gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, p);
+    gemm_tc_kernel<N_TILE, PLANES, MAGIC, DUMP, TSTORE><<<grid, THREADS, C::SMEM, st>>>(mA0, mA1, mB0, mB1, mEA, mEB, mC, p);
     return launch_status();
 }
 
@@ -742,11 +790,16 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     // the biased-accumulator path needs every |P| < 2^22
     const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
     const bool magic = a.L.planes == 1 && qa * qb * a.L.b < (1ll << 22);
+    // Short contractions are bound by the write of C: the tile then leaves through shared memory and TMA stores,
+    // which the copy engine writes as whole lines while the warps go on with the next tile.
+    const bool tstore = p.splits == 1 && !P && a.L.nkb * a.L.bp <= 1024 && (reinterpret_cast<uintptr_t>(Cout) & 15) == 0 && (ldc % 4) == 0;
     if (P) {   // the inspection build of the kernel: 64-column tiles, writes the block sums
         p.tiles_n = (int)((N + 63) / 64);
         if (a.L.planes == 2) rc = launch_cfg<64, 2, false, true>(p, a, b, st);
         else rc = magic ? launch_cfg<64, 1, true, true>(p, a, b, st) : launch_cfg<64, 1, false, true>(p, a, b, st);
     } else if (a.L.planes == 2) rc = launch_cfg<64, 2, false, false>(p, a, b, st);
+    else if (magic && tstore && plan.n_tile == 256) rc = launch_cfg<256, 1, true, false, true>(p, a, b, st);
+    else if (magic && tstore && plan.n_tile == 128) rc = launch_cfg<128, 1, true, false, true>(p, a, b, st);
     else if (plan.n_tile == 256) rc = magic ? launch_cfg<256, 1, true, false>(p, a, b, st) : launch_cfg<256, 1, false, false>(p, a, b, st);
     else if (plan.n_tile == 128) rc = magic ? launch_cfg<128, 1, true, false>(p, a, b, st) : launch_cfg<128, 1, false, false>(p, a, b, st);
     else rc = magic ? launch_cfg<64, 1, true, false>(p, a, b, st) : launch_cfg<64, 1, false, false>(p, a, b, st);
