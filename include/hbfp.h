@@ -153,10 +153,10 @@ HBFP_API int hbfp_quantize_conv_weights(const float* w, int64_t taps, int64_t c_
  * tile x tile square, [ceil(d0/t)][ceil(d1/t)] (device). fmt->tile == fmt->block = t in 1..128;
  * fmt->rounding, seed, stream_id and exp_mode govern the conversion to 16 bits (stochastic rounding
  * draws by the element's row-major index in w); fmt->mant_bits = m in 3..12 is the width of the narrow
- * copy: its mantissas are the top m bits of the stored words, a stored word being the mantissa plus
- * half a narrow unit, i.e. clamp(floor((q16 + 2^(15-m)) / 2^(16-m)), +-(2^(m-1) - 1)): the wide value
- * rounded to nearest, ties upward (plain truncation would leave every narrow weight half a narrow ULP
- * low, a bias that adds up over a dot product), under the exponent s16 + 16 - m. The narrow copy is
+ * copy: its mantissas are the top m bits of the wide mantissa after half a narrow unit has been added,
+ * clamp(floor((q16 + 2^(15-m)) / 2^(16-m)), +-(2^(m-1) - 1)): the wide value rounded to nearest, ties
+ * upward (plain truncation would leave every narrow weight half a narrow ULP low, a bias that adds up
+ * over a dot product), under the exponent s16 + 16 - m. `wide` itself holds the bare mantissas q16. The narrow copy is
  * written as the two packed views of
  * hbfp_quantize_tiles (`*_c0`: rows = d1, k = d0; `*_c1`: rows = d0, k = d1; buffers of the sizes
  * hbfp_packed_sizes returns, fully overwritten); both mant_c0 and mant_c1 may be NULL to skip it, one

@@ -1,5 +1,6 @@
 """Pins of the oracle's wide weight storage (Sec. 4.2): 16-bit quantisation against exact rational
-rounding, the narrow copy as the top bits (a floor, bracketed in exact rationals), and the weight
+rounding, the narrow copy as the top bits after half a narrow unit was added (nearest narrow value, ties
+upward, checked in exact rationals), and the weight
 update against a binary32 numpy restatement, its fixed point and exact integer steps."""
 from fractions import Fraction
 import math
