@@ -7,16 +7,17 @@
 // rescale work as a 128 x 256 tile on one SM, but only half of the B panel crosses from L2 into
 // each SM, which is what limits the single-SM kernel on large problems.
 //
-// Roles per CTA (16 warps) as in the single-SM kernel: warp 0 TMA producer, warp 1 MMA issuer
-// (only in the cluster's first CTA, the leader) and tensor-memory owner, warp 2 scale-table
-// builder, warps 4-15 rescale (Eq. 2 per block, blocks accumulated in FP32, Sec. 4): three per
+// Roles per CTA (16 warps): warp 0 TMA producer, warp 1 MMA issuer (only in the cluster's first
+// CTA, the leader) and tensor-memory owner, warps 2 and 3 scale-table builders (even / odd
+// K-blocks), warps 4-15 rescale (Eq. 2 per block, blocks accumulated in FP32, Sec. 4): three per
 // lane quarter of tensor memory, which split the 256 columns 88 + 88 + 80.
 //
 // Barriers. Mantissa tiles of both CTAs complete on the leader's full[s]; exponent slices on a
-// local efull[s]; the leader's MMA thread commits to tfull[g] and empty[s] of both CTAs; the
+// local efull[s]; the leader's MMA thread commits to tfull[g] of both CTAs (one commit per
+// K-block and no other); the table builders hand the stages back to the producer (empty[s]); the
 // rescale warps of both CTAs arrive on the leader's tempty[g]. A rescale warp does one wait and
-// one arrival per K-block: the table warp's "scales written" arrival is counted on tfull[g]
-// together with the MMA commit, and the table warp learns that a table slot is free again from
+// one arrival per K-block: the builder's "scales written" arrival is counted on tfull[g]
+// together with the MMA commit, and the builder learns that a table slot is free again from
 // the completion of tfull two blocks back (the MMAs of that block were issued only after every
 // rescale warp had finished the slot's last reader). Every wait is bounded: when one expires the
 // CTA records a code in the device status word, raises its abort flag, drains what it can wait
@@ -55,7 +56,7 @@ constexpr int EXP_STAGE = EXP_A + EXP_B;
 constexpr int TSLOTS = 4;
 constexpr int TABLE_SLOT_WORDS = N_TILE + TILE_M;
 constexpr int TABLE_BYTES = 4 * TSLOTS * TABLE_SLOT_WORDS;
-constexpr int STAGES = 6;
+constexpr int STAGES = 5;      // measured: 5 stages 2.6 % fewer cycles than 6 (n = 16384), 4 as many as 6, 3 far more
 constexpr int ONES_BYTES = TILE_M * STAGE_K;   // 128 rows of 0xFF bytes: both operands of the offset step
 constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + ONES_BYTES + 1024;
 static_assert(SMEM <= 232448, "shared memory");
@@ -373,7 +374,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const uint32_t bars = base + bar_off;
     const uint32_t full_bar = bars;                          // leader: mantissa tiles of both CTAs landed
     const uint32_t efull_bar = full_bar + 8 * STAGES;        // local: exponent slices landed
-    const uint32_t empty_bar = efull_bar + 8 * STAGES;       // local: stage consumed (MMA commit + table warp)
+    const uint32_t empty_bar = efull_bar + 8 * STAGES;       // local: stage consumed (both table builders)
     const uint32_t tfull_bar = empty_bar + 8 * STAGES;       // local: block sums complete (MMA commit) and scale table written
     const uint32_t tempty_bar = tfull_bar + 8 * GROUPS;      // leader: group read and re-armed by the rescale warps of both CTAs
     const uint32_t done_bar = tempty_bar + 8 * GROUPS;
@@ -391,10 +392,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(full_bar + 8 * s, 1);
             mbar_init(efull_bar + 8 * s, 1);
-            mbar_init(empty_bar + 8 * s, 2);
+            mbar_init(empty_bar + 8 * s, 2);               // this CTA's two table builders, once the stage's MMAs are complete
         }
         for (int g = 0; g < GROUPS; ++g) {
-            mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + this CTA's table warp
+            mbar_init(tfull_bar + 8 * g, 2);                 // MMA commit + this CTA's table builder of the group
             mbar_init(tempty_bar + 8 * g, 2 * RESCALE_WARPS);
         }
         mbar_init(done_bar, 1);
@@ -504,63 +505,79 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                                 ++blk;
                             }
                         }
-                        tc_commit_pair(empty_bar + 8 * s, 3);        // the stage is free in both CTAs
                         ring_next<STAGES>(s, ph);
                     }
                 }
                 tc_commit_pair(done_bar, 1);
                 mbar_wait(done_bar, 0, abort_flag, p.status, 213, false);
             }
-        } else if (warp == TABLE_WARP) {
-            // -------------------------------------------------------------- scale-table builder
-            // The table of block b goes to slot b % 4 and its arrival counts on tfull[b % 2]. It is
-            // written once the phase of block b - 2 on that barrier is complete: the MMAs of b - 2 were
-            // issued only after every rescale warp had finished b - 4, the last reader of the slot, and
-            // the barrier is back in the phase that the arrival for b belongs to.
-            uint32_t s = 0, ph = 0, g = 0, gph = 0, slot = 0, it = 0, blk = 0;
+        } else {
+            // -------------------------------------------------------------- scale-table builders (warps 2 and 3)
+            // Warp 2 builds the tables of the even blocks (accumulator group 0), warp 3 those of the odd blocks
+            // (group 1): a single builder made the rescale warps of its sub-partition the last to hand every
+            // group back. The table of block b goes to slot b % 4 and its arrival counts on tfull[b % 2]. It is
+            // written once the phase of block b - 2 on that barrier is complete: the MMAs of b - 2 were issued
+            // only after every rescale warp had finished b - 4, the last reader of the slot, and the barrier is
+            // back in the phase that the arrival for b belongs to.
+            //
+            // Stage hand-back. A commit costs the MMA thread several hundred cycles, so it issues one per block
+            // (tfull) and none per stage: each builder arrives once per stage on empty[s] (count 2). A builder
+            // with blocks in the stage does so when it sees the tfull phase of its last block there complete,
+            // which it waits for anyway at its next block (MMAs complete in order); a builder without a block
+            // in the stage arrives at once. Both wait for the stage's exponent slices first: their arrival shows
+            // that the producer has consumed the previous phase of empty[s], so an arrival can never fall into it.
+            const uint32_t me = (uint32_t)(warp - TABLE_WARP);
+            uint32_t s = 0, ph = 0, g = 0, own_ph = 0, slot = me;
+            int pend = -1;                 // stage to hand back at this builder's next block
             bool ok = true, out_of_range = false;
             for (int wi = cluster; ok && wi < total_work; wi += nclusters) {
                 const Work w = get_work(p, wi);
                 const int nst = (w.nblk + BPS - 1) >> LB;
                 int left = w.nblk;
-                for (int si = 0; ok && si < nst; ++si, left -= BPS, ++it) {
+                for (int si = 0; ok && si < nst; ++si, left -= BPS) {
                     if (!mbar_wait_warp(efull_bar + 8 * s, ph, abort_flag, p.status, 411)) { ok = false; break; }
                     const unsigned char* eA = base_ptr + (exp_base - base) + s * EXP_STAGE;
                     const unsigned char* eB = eA + EXP_A;
+                    bool own_any = false;
 #pragma unroll
                     for (int jb = 0; jb < BPS; ++jb) {
                         if (jb < left) {
-                            // this lane's 8 column exponents and 4 row exponents of block jb of the stage
-                            const uint2 cb = *reinterpret_cast<const uint2*>(eB + jb * N_TILE + 8 * lane);
-                            const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
-                            // The split of the scales (rescale_loop): c = SHIFT wherever the block's exponents allow
-                            // it, otherwise moved into the window in which every factor and every P * 2^(sA + c - 149)
-                            // is a normal binary32 number. The window is empty only when the row exponents of the
-                            // block span more than 104 or the true products leave binary32: reported, not computed.
-                            const int a_lo = __reduce_min_sync(0xffffffffu, byte_min(ra)), a_hi = __reduce_max_sync(0xffffffffu, byte_max(ra));
-                            const int b_lo = __reduce_min_sync(0xffffffffu, byte_min(__vmins4(cb.x, cb.y)));
-                            const int b_hi = __reduce_max_sync(0xffffffffu, byte_max(__vmaxs4(cb.x, cb.y)));
-                            const int c_lo = max(23 - a_lo, 22 + b_hi), c_hi = min(127 - a_hi, 275 + b_lo);
-                            out_of_range |= c_lo > c_hi;
-                            const int c = min(max(SHIFT, c_lo), c_hi);
-                            uint4 c0, c1, r0;
-                            c0.x = exp_to_scale(cb.x, 0, 149 - c); c0.y = exp_to_scale(cb.x, 1, 149 - c); c0.z = exp_to_scale(cb.x, 2, 149 - c); c0.w = exp_to_scale(cb.x, 3, 149 - c);
-                            c1.x = exp_to_scale(cb.y, 0, 149 - c); c1.y = exp_to_scale(cb.y, 1, 149 - c); c1.z = exp_to_scale(cb.y, 2, 149 - c); c1.w = exp_to_scale(cb.y, 3, 149 - c);
-                            r0.x = exp_to_scale(ra, 0, c); r0.y = exp_to_scale(ra, 1, c); r0.z = exp_to_scale(ra, 2, c); r0.w = exp_to_scale(ra, 3, c);
-                            if (!mbar_wait_warp(tfull_bar + 8 * g, gph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
-                            uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
-                            *reinterpret_cast<uint4*>(tb + 8 * lane) = c0;
-                            *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
-                            *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(tfull_bar + 8 * g);
-                            ring_next<GROUPS>(g, gph);
-                            slot = (slot + 1) & (TSLOTS - 1);
-                            ++blk;
+                            if (g == me) {
+                                own_any = true;
+                                // this lane's 8 column exponents and 4 row exponents of block jb of the stage
+                                const uint2 cb = *reinterpret_cast<const uint2*>(eB + jb * N_TILE + 8 * lane);
+                                const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
+                                // The split of the scales (rescale_loop): c = SHIFT wherever the block's exponents allow
+                                // it, otherwise moved into the window in which every factor and every P * 2^(sA + c - 149)
+                                // is a normal binary32 number. The window is empty only when the row exponents of the
+                                // block span more than 104 or the true products leave binary32: reported, not computed.
+                                const int a_lo = __reduce_min_sync(0xffffffffu, byte_min(ra)), a_hi = __reduce_max_sync(0xffffffffu, byte_max(ra));
+                                const int b_lo = __reduce_min_sync(0xffffffffu, byte_min(__vmins4(cb.x, cb.y)));
+                                const int b_hi = __reduce_max_sync(0xffffffffu, byte_max(__vmaxs4(cb.x, cb.y)));
+                                const int c_lo = max(23 - a_lo, 22 + b_hi), c_hi = min(127 - a_hi, 275 + b_lo);
+                                out_of_range |= c_lo > c_hi;
+                                const int c = min(max(SHIFT, c_lo), c_hi);
+                                uint4 c0, c1, r0;
+                                c0.x = exp_to_scale(cb.x, 0, 149 - c); c0.y = exp_to_scale(cb.x, 1, 149 - c); c0.z = exp_to_scale(cb.x, 2, 149 - c); c0.w = exp_to_scale(cb.x, 3, 149 - c);
+                                c1.x = exp_to_scale(cb.y, 0, 149 - c); c1.y = exp_to_scale(cb.y, 1, 149 - c); c1.z = exp_to_scale(cb.y, 2, 149 - c); c1.w = exp_to_scale(cb.y, 3, 149 - c);
+                                r0.x = exp_to_scale(ra, 0, c); r0.y = exp_to_scale(ra, 1, c); r0.z = exp_to_scale(ra, 2, c); r0.w = exp_to_scale(ra, 3, c);
+                                if (!mbar_wait_warp(tfull_bar + 8 * me, own_ph ^ 1, abort_flag, p.status, 412)) { ok = false; break; }
+                                if (pend >= 0 && lane == 0) mbar_arrive(empty_bar + 8 * pend);   // this builder's previous block is complete
+                                pend = (jb + 2 >= BPS || jb + 2 >= left) ? (int)s : -1;          // its last block of this stage?
+                                uint32_t* tb = tables + slot * TABLE_SLOT_WORDS;
+                                *reinterpret_cast<uint4*>(tb + 8 * lane) = c0;
+                                *reinterpret_cast<uint4*>(tb + 8 * lane + 4) = c1;
+                                *reinterpret_cast<uint4*>(tb + N_TILE + 4 * lane) = r0;
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(tfull_bar + 8 * me);
+                                own_ph ^= 1u;
+                                slot = (slot + 2) & (TSLOTS - 1);
+                            }
+                            g ^= 1u;
                         }
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(empty_bar + 8 * s);      // the exponent slices are consumed
+                    if (!ok) break;
+                    if (!own_any && lane == 0) mbar_arrive(empty_bar + 8 * s);     // nothing of this builder's in the stage
                     ring_next<STAGES>(s, ph);
                 }
             }
