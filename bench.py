@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # with the summary of the single-pass ncu capture it was read from. A workload without an entry reports
 # no traffic.
 GEMM_DRAM_TRAFFIC = {
-    ("gemm_tc2_kernel", 16384, 8, 128): {"bytes": 4416503296 + 1075157504,
+    ("gemm_tc2_kernel", 16384, 8, 128): {"bytes": 6233750016 + 1080012288,
                                          "profile": "profiles/bench_launch_list_n16384_m8_b128.md"},
 }
 SUSTAINED_SECONDS = 2.5       # length of the back-to-back GEMM loop behind `gemm_sustained`
@@ -325,6 +325,21 @@ def gpu_arm(args):
     # ---- which GEMM kernel the library launched for this workload (asked of the library, not re-derived)
     hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
     gemm_kernel = hb.last_gemm_kernel()
+    # ---- the clock the SMs really ran at: the paired-SM kernel stamps its length in SM cycles, and cycles / device
+    # time is the effective clock of that launch (under the power cap it is below what nvidia-smi shows)
+    eff = None
+    if gemm_kernel == "gemm_tc2_kernel":
+        s6, e6 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
+        s6.record()
+        hb.gemm_q(n, n, n, pa, pb, out=C, workspace=ws)
+        e6.record()
+        torch.cuda.synchronize()
+        cyc = hb.last_gemm_cycles()
+        ms6 = s6.elapsed_time(e6)
+        if cyc > 0 and ms6 > 0:
+            eff = {"gemm_cycles": cyc, "gemm_ms": ms6, "sm_mhz_effective": cyc / ms6 / 1e3}
 
     # ---- the GEMM back to back for a few seconds: what it does once the power cap has pulled the clock
     # down (the timed region above is a burst of ~0.1 s). Device time by CUDA events, SM clock sampled
@@ -349,6 +364,7 @@ def gpu_arm(args):
         sustained = {"launches": reps, "seconds": (tw1 - tw0), "ms_per_launch": ms5, "tops": ops / (ms5 * 1e-3) / 1e12,
                      "sm_mhz_median_second_half": clk2["sm_mhz"], "power_w_max": clk2.get("power_w_max"),
                      "reasons": clk2["reasons"],
+                     "cycles_per_launch": hb.last_gemm_cycles() if gemm_kernel == "gemm_tc2_kernel" else None,
                      "ms_x_mhz": ms5 * clk2["sm_mhz"] if clk2["sm_mhz"] else None,
                      "burst_ms_x_mhz": t_gemm * clocks["sm_mhz"] if clocks.get("sm_mhz") else None}
 
@@ -394,6 +410,11 @@ def gpu_arm(args):
         wide["update_8192x8192_m8_t64_rne"] = {"ms": ms, "gbs": nw * nw * 10 / (ms * 1e-3) / 1e9}
         del Wm, dW, wst, views
 
+    if eff:
+        clocks["gemm_sm_mhz_effective"] = eff["sm_mhz_effective"]      # cycles counted by the kernel / its device time
+        clocks["gemm_cycles"] = eff["gemm_cycles"]
+    if sustained and sustained.get("cycles_per_launch"):
+        sustained["sm_mhz_effective"] = sustained["cycles_per_launch"] / sustained["ms_per_launch"] / 1e3
     peaks, peaks_kind = load_peaks()
     int8_burst = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_sust = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * INT8_OVER_BF16

@@ -343,6 +343,15 @@ HBFP_API int hbfp_gemm_block_partials(int64_t M, int64_t N, int64_t K, const hbf
  * string is static storage. */
 HBFP_API const char* hbfp_last_gemm_kernel(void);
 
+/* Synchronises the current device, then writes to *cycles (host) the length, in SM clock cycles, of the
+ * most recent launch of the paired-SM GEMM kernel ("gemm_tc2_kernel") on that device: every CTA reads the
+ * cycle counter when it starts and when it ends, and the largest difference is reported (0 before the
+ * first such launch). Cycles divided by the launch's duration is the clock the SMs really ran at, which
+ * under the board's power cap is lower than the clock the driver reports; measurement scripts use it to
+ * tell a change of the code from a change of the clock (the paper has no counterpart). Returns
+ * HBFP_ERR_INVALID_ARG for a null pointer, HBFP_ERR_CUDA if the copy fails. */
+HBFP_API int hbfp_last_gemm_cycles(uint64_t* cycles);
+
 /* Synchronises `stream`, then returns and clears the device-side status word of the current
  * device in *status (host int): 0, or a code recorded by a kernel. Codes below 900: a bounded wait
  * on a barrier expired (the kernel then abandons its work and exits; HBFP_ERR_TIMEOUT is returned).

@@ -28,7 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
-    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel", "hbfp_conv_forward", "hbfp_quantize_conv_weights",
+    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel", "hbfp_last_gemm_cycles", "hbfp_conv_forward", "hbfp_quantize_conv_weights",
 ]
 
 
@@ -108,6 +108,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_conv_forward.argtypes = [p, p, i64, i64, i64, i64, i32, i32, i32, p, p, i64, p, i64, p]
         L.hbfp_wide_dequantize.argtypes = [p, p, i64, i64, i32, p, i64, p]
         L.hbfp_selftest_bounded_wait.argtypes = [i64, i32, p, p]
+        L.hbfp_last_gemm_cycles.argtypes = [p]
         L.hbfp_last_gemm_kernel.restype = ctypes.c_char_p
         L.hbfp_last_gemm_kernel.argtypes = []
         for name in EXPORTS[1:]:
@@ -459,6 +460,13 @@ def gemm_block_partials(a: Packed, b: Packed, impl: int = GEMM_FORCE_SIMT) -> to
     _check(lib().hbfp_gemm_block_partials(M, N, K, ctypes.byref(oa), ctypes.byref(ob), _dptr(P), impl, _stream()),
            "hbfp_gemm_block_partials")
     return P
+
+
+def last_gemm_cycles() -> int:
+    """hbfp_last_gemm_cycles: SM cycles of the longest CTA of the most recent paired-SM GEMM launch (synchronises)."""
+    out = ctypes.c_uint64(0)
+    _check(lib().hbfp_last_gemm_cycles(ctypes.byref(out)), "hbfp_last_gemm_cycles")
+    return int(out.value)
 
 
 def last_gemm_kernel() -> str:

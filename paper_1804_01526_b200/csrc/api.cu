@@ -396,6 +396,11 @@ int hbfp_selftest_bounded_wait(int64_t limit_cycles, int32_t code, int32_t* outc
     return launch_wait_probe((long long)limit_cycles, (int)code, reinterpret_cast<int*>(outcome), static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_last_gemm_cycles(uint64_t* cycles) {
+    if (!cycles) return HBFP_ERR_INVALID_ARG;
+    return pair_gemm_cycles(cycles);
+}
+
 int hbfp_device_status(void* stream, int32_t* status) {
     if (!status) return HBFP_ERR_INVALID_ARG;
     return read_clear_device_status(static_cast<cudaStream_t>(stream), status);

@@ -117,6 +117,7 @@ int launch_conv_forward(const Packed& x, const Packed& wt, int64_t n, int64_t h,
 
 // One warp running the kernels' bounded barrier wait on a barrier nobody arrives on (test hook).
 int launch_wait_probe(long long limit_cycles, int code, int* outcome, cudaStream_t st);
+int pair_gemm_cycles(uint64_t* cycles);   // longest CTA of the last paired-SM GEMM launch on the current device, in SM cycles
 
 // Device status word (bounded waits report here).
 int32_t* device_status_word();   // device address, per current device

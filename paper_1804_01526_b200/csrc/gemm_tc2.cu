@@ -61,6 +61,11 @@ constexpr int ONES_BYTES = TILE_M * STAGE_K;   // 128 rows of 0xFF bytes: both o
 constexpr int SMEM = 1024 + STAGES * (MANT_STAGE + EXP_STAGE) + TABLE_BYTES + ONES_BYTES + 1024;
 static_assert(SMEM <= 232448, "shared memory");
 
+// Length of the last launch in SM cycles, per CTA (hbfp_last_gemm_cycles): cycles ÷ event time is the clock the
+// SMs really ran at, which under the power cap is well below the one the driver reports.
+constexpr int MAX_CTAS = 2 * 148 * 2;
+__device__ unsigned long long g_cta_cycles[MAX_CTAS];
+
 struct Problem {
     int64_t M, N;
     int64_t nkb;
@@ -384,6 +389,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long cycles_start = clock64();
     const uint32_t rank = cluster_ctarank();                 // 0 = leader
     const int cluster = (int)cluster_id_x(), nclusters = (int)cluster_count_x();
     const int total_work = p.tiles_m * p.tiles_n * p.splits;
@@ -596,6 +602,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     // Neither CTA may leave while the other can still signal its barriers or read its shared memory.
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0 && blockIdx.x < MAX_CTAS) g_cta_cycles[blockIdx.x] = (unsigned long long)(clock64() - cycles_start);
     cluster_barrier();
     if (warp == MMA_WARP) {
         tc_fence_after();
@@ -631,7 +638,23 @@ int max_clusters() {
     return n[dev];
 }
 
+int g_last_ctas[MAX_DEVICES] = {};     // CTAs of the last launch, per device
+
 }  // namespace
+
+int pair_gemm_cycles(uint64_t* cycles) {
+    unsigned long long host[MAX_CTAS];
+    const int dev = current_device();
+    const int n = dev >= 0 ? g_last_ctas[dev] : 0;
+    *cycles = 0;
+    if (n <= 0) return HBFP_OK;
+    HBFP_CUDA_OK(cudaDeviceSynchronize());
+    HBFP_CUDA_OK(cudaMemcpyFromSymbol(host, g_cta_cycles, sizeof(unsigned long long) * n));
+    unsigned long long m = 0;
+    for (int i = 0; i < n; ++i) m = host[i] > m ? host[i] : m;
+    *cycles = m;
+    return HBFP_OK;
+}
 
 bool pair_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, const TensorPlan& plan) {
     if (a.L.planes != 1 || b.L.planes != 1) return false;
@@ -676,6 +699,12 @@ int launch_gemm_tensor_pair(int64_t M, int64_t N, const Packed& a, const Packed&
     if (clusters_max < 1) return HBFP_ERR_UNSUPPORTED;
     const int64_t work = (int64_t)p.tiles_m * p.tiles_n * p.splits;
     const int clusters = (int)(work < clusters_max ? work : clusters_max);
+    static_assert(2 * 148 <= MAX_CTAS, "cycle stamps");
+    if (2 * clusters > MAX_CTAS) return HBFP_ERR_UNSUPPORTED;
+    {
+        const int dev = current_device();
+        if (dev >= 0) g_last_ctas[dev] = 2 * clusters;     // the stamps that pair_gemm_cycles may read
+    }
     if (p.bp == 128) gemm_tc2_kernel<0><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);
     else if (p.bp == 64) gemm_tc2_kernel<1><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);
     else gemm_tc2_kernel<2><<<2 * clusters, THREADS, SMEM, st>>>(mA, mB, mEA, mEB, p);

@@ -320,3 +320,27 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable(
     assert hb.device_status_rc() == (hb.OK, 0)
     specs = wl.config_single_256()
     run_spec(hb, specs[0], wl.materialize(specs, seed=0), hb.GEMM_AUTO)
+
+
+def test_last_gemm_cycles_reports_the_paired_kernel_length(hb):
+    """hbfp_last_gemm_cycles: the paired-SM kernel's length in SM cycles (longest CTA), a plausible number of them."""
+    import torch
+    n = 4096
+    f = hb.Format(8, 128)
+    A = to_dev(wl.draw("lognormal", (n, n), seed=71))
+    pa, pb = hb.quantize(A, 1, f), hb.quantize(A, 0, f)
+    ws = torch.empty(max(hb.gemm_q_workspace(n, n, n, pa, pb), 1), dtype=torch.int8, device="cuda")
+    out = torch.empty((n, n), dtype=torch.float32, device="cuda")
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    hb.gemm_q(n, n, n, pa, pb, out=out, workspace=ws, flags=hb.GEMM_FORCE_TENSOR_2SM)
+    s.record()
+    hb.gemm_q(n, n, n, pa, pb, out=out, workspace=ws, flags=hb.GEMM_FORCE_TENSOR_2SM)
+    e.record()
+    torch.cuda.synchronize()
+    assert hb.last_gemm_kernel() == "gemm_tc2_kernel"
+    cycles = hb.last_gemm_cycles()
+    mhz = cycles / s.elapsed_time(e) / 1e3
+    # 32 K-blocks x 4 tiles per cluster at several hundred cycles each; a clock between 0.5 and 2.2 GHz
+    assert 32 * 4 * 300 < cycles < 32 * 4 * 20000
+    assert 500 < mhz < 2200
+    assert hb.device_status() == 0
