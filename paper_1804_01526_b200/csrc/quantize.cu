@@ -1245,7 +1245,10 @@ template <int PLANES, int LB, bool SR>      // b = 128 >> LB
 __global__ void __launch_bounds__(QC_THREADS)
 quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapM0,
               const __grid_constant__ CUtensorMap mapM1, QParams p, int8_t* __restrict__ exps, int64_t rs,
-              int64_t nkb, int64_t K, int64_t R, int tiles_n, int total_tiles, int32_t* status) {
+              int64_t nkb, int64_t K, int64_t R, int tiles_n, int total_tiles, int32_t* status,
+              const int8_t* __restrict__ given) {
+    // given != nullptr: one exponent per column for the whole axis, computed beforehand (blocks longer than a
+    // tile); the kernel then only rounds and packs
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
@@ -1317,9 +1320,9 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
         }
         if (LB == 0) am = max(max(pmax[n], pmax[QC_COLS + n]), max(pmax[2 * QC_COLS + n], pmax[3 * QC_COLS + n]));
         if (LB == 1) am = max(pmax[(q & 2) * QC_COLS + n], pmax[((q & 2) + 1) * QC_COLS + n]);
-        const int sexp = block_exponent(am, p.m, p.exp_mode);
+        const int sexp = given ? (col < R ? (int)given[col] : -63) : block_exponent(am, p.m, p.exp_mode);
         const int64_t kb = ((int64_t)kt << LB) + (q >> (2 - LB));
-        if ((q & ((4 >> LB) - 1)) == 0 && kb < nkb && col < R) exps[kb * rs + col] = (int8_t)sexp;
+        if (!given && (q & ((4 >> LB) - 1)) == 0 && kb < nkb && col < R) exps[kb * rs + col] = (int8_t)sexp;
 
         uint32_t hi[8], lo[8];
         const uint16_t* rnd16 = reinterpret_cast<const uint16_t*>(rnd);
@@ -1364,9 +1367,27 @@ quant_col_tma(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
     if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
+// Whole-axis blocks down the columns (one exponent per column of the stored matrix): pass 1 of 2. Each CTA takes
+// 256 columns and a band of rows, reads rows coalesced and folds its band's maxima into one word per column.
+constexpr int CMAX_ROWS = 128;
+__global__ void __launch_bounds__(256)
+col_amax_kernel(const float* __restrict__ x, int64_t K, int64_t R, int64_t ld, uint32_t* __restrict__ amax) {
+    const int64_t col = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (col >= R) return;
+    const int64_t k0 = (int64_t)blockIdx.y * CMAX_ROWS, k1 = min(K, k0 + CMAX_ROWS);
+    uint32_t am = 0;
+#pragma unroll 8
+    for (int64_t k = k0; k < k1; ++k) am = max(am, abs_bits(__ldg(x + k * ld + col)));
+    atomicMax(amax + col, am);
+}
+__global__ void col_exps_kernel(const uint32_t* __restrict__ amax, int64_t R, QParams p, int8_t* __restrict__ exps) {
+    const int64_t col = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (col < R) exps[col] = (int8_t)block_exponent(amax[col], p.m, p.exp_mode);
+}
+
 template <int PLANES, int LB, bool SR>
 int launch_col_tma(const float* x, int64_t K, int64_t rows, int64_t ld, const QParams& p, const Layout& L,
-                   int8_t* mant, int8_t* exps, cudaStream_t st) {
+                   int8_t* mant, int8_t* exps, cudaStream_t st, const int8_t* given = nullptr) {
     CUtensorMap mX, mM0, mM1;
     int rc = make_map(&mX, x, (uint64_t)rows * 4, (uint64_t)K, (uint64_t)ld * 4, QC_COLS * 4, QC_ROWS, false);
     if (rc) return rc;
@@ -1397,7 +1418,7 @@ int launch_col_tma(const float* x, int64_t K, int64_t rows, int64_t ld, const QP
     const int64_t cap = (int64_t)sm_count() * ctas_per_sm;
     const int grid = (int)(total < cap ? total : cap);
     quant_col_tma<PLANES, LB, SR><<<grid, QC_THREADS, smem, st>>>(mX, mM0, mM1, p, exps, L.rs, L.nkb, K, rows, (int)tiles_n,
-                                                              (int)total, status);
+                                                              (int)total, status, given);
     return launch_status();
 }
 
@@ -1471,6 +1492,24 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
             case 256: return launch_row_fast<32>(x, rows, K, ld, p, L, mant, exps, st);
             default: break;
         }
+    }
+    // one block per column over the whole axis: column maxima first (scratch: the head of the mantissa buffer, which
+    // the second pass overwrites), then the tile kernel with the exponents given
+    if (f->tile == 0 && axis == 0 && aligned && L.nkb == 1 && L.b == K && K % QC_ROWS == 0 && L.kst == K && K > 128 &&
+        (p.rounding == 0 || rows % 8 == 0) && (reinterpret_cast<uintptr_t>(mant) & 127) == 0 && rows < (1ll << 29) &&
+        K < (1ll << 31) && (K + CMAX_ROWS - 1) / CMAX_ROWS <= 65535 && (int64_t)rows * 4 <= (int64_t)rows * L.kst &&
+        ((rows + QC_COLS - 1) / QC_COLS) * (L.kst / QC_ROWS) < (1ll << 31)) {
+        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        uint32_t* amax = reinterpret_cast<uint32_t*>(mant);
+        HBFP_CUDA_OK(cudaMemsetAsync(amax, 0, (size_t)rows * 4, st));
+        const dim3 g1((unsigned)((rows + 255) / 256), (unsigned)((K + CMAX_ROWS - 1) / CMAX_ROWS));
+        col_amax_kernel<<<g1, 256, 0, st>>>(x, K, rows, ld, amax);
+        col_exps_kernel<<<(unsigned)((rows + 255) / 256), 256, 0, st>>>(amax, rows, p, exps);
+        if (launch_status()) return HBFP_ERR_CUDA;
+#define HBFP_QCOL_GIVEN(PL) (p.rounding ? launch_col_tma<PL, 0, true>(x, K, rows, ld, p, L, mant, exps, st, exps) \
+                                        : launch_col_tma<PL, 0, false>(x, K, rows, ld, p, L, mant, exps, st, exps))
+        return L.planes == 1 ? HBFP_QCOL_GIVEN(1) : HBFP_QCOL_GIVEN(2);
+#undef HBFP_QCOL_GIVEN
     }
     if (f->tile == 0 && axis == 0 && aligned && L.b == L.bp && L.b <= 128 && (p.rounding == 0 || rows % 8 == 0) &&
         (reinterpret_cast<uintptr_t>(mant) & 127) == 0 && rows < (1ll << 29) && K < (1ll << 31) &&

@@ -108,6 +108,21 @@ def test_column_blocks_streaming_kernel(hb, shape, law, fd):
     _check(hb, wl.draw(law, shape, seed=14), 0, fd)
 
 
+# One exponent per column over the whole axis (block 0) with a column length that is a multiple of 128: column maxima
+# in a first pass (scratch in the mantissa buffer), then the streaming kernel with the exponents given.
+COL_WHOLE_AXIS_CASES = [
+    ((1024, 200), "lognormal", F(8, 0, rounding=1, seed=6, sid=3)),         # ragged columns, stochastic
+    ((2048, 1000), "outliers", F(8, 0, exp_mode=1)),                        # several bands of rows per column
+    ((384, 72), "grad", F(12, 0, rounding=1, seed=2)),                      # two planes
+    ((256, 8), "normal", F(4, 0)),                                          # eight output rows
+]
+
+
+@pytest.mark.parametrize("shape,law,fd", COL_WHOLE_AXIS_CASES)
+def test_column_blocks_over_the_whole_axis(hb, shape, law, fd):
+    _check(hb, wl.draw(law, shape, seed=16), 0, fd)
+
+
 def test_column_blocks_of_a_pitched_view(hb):
     # a 16-byte aligned column window of a wider matrix: the pitch differs from the logical width,
     # and the stochastic stream follows the logical index of the window
