@@ -177,7 +177,9 @@ template <int LPB, bool SR, int PLANES>
 __global__ void __launch_bounds__(256)
 quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, QParams p,
                int8_t* __restrict__ mant, int64_t kst, int64_t plane_stride,
-               int8_t* __restrict__ exps, int64_t rs, int64_t nkb) {
+               int8_t* __restrict__ exps, int64_t rs, int64_t nkb, const int8_t* __restrict__ given = nullptr) {
+    // given != nullptr: one exponent per row for the whole axis, computed beforehand (a block longer than the
+    // tile); the kernel then only rounds and packs
     constexpr int B = 8 * LPB;
     constexpr int KB_PER_SPAN = 256 / B;            // blocks in one warp span of 256 columns
     constexpr int KB_PER_TILE = 512 / B;
@@ -222,7 +224,7 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
             uint32_t am = amax8_bits(e8);
 #pragma unroll
             for (int off = 1; off < LPB; off <<= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
-            const int s = block_exponent(am, p.m, p.exp_mode);
+            const int s = given ? (r < rows ? (int)given[r] : -63) : block_exponent(am, p.m, p.exp_mode);
             const uint4 w = wd[i];
             uint2 hi, lo;
             quantize_pack8<SR, PLANES>(e8, s, p, w, hi, lo);
@@ -235,6 +237,7 @@ quant_row_fast(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld,
         }
     }
     __syncthreads();
+    if (given) return;
     // exponents: [kb][row], 32 rows of one block are 32 contiguous bytes.
     const int64_t kb0 = c0 / B;
     for (int i = tid; i < KB_PER_TILE * 8; i += 256) {
@@ -1482,6 +1485,20 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
             case 128: return launch_row_flat<16>(x, rows, K, ld, p, L, mant, exps, st);
             default: break;
         }
+    }
+    // one block per row over the whole axis, longer than the fast kernel's tile: row maxima first (one warp per row),
+    // then the fast kernel with the exponents given
+    if (f->tile == 0 && axis == 1 && aligned && d1 % 8 == 0 && L.nkb == 1 && L.b == K && K > 256) {
+        if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        const int64_t want = (rows * 32 + 255) / 256;
+        exps_axis1<<<(unsigned)(want < 148 * 16 ? want : 148 * 16), 256, 0, st>>>(x, rows, K, ld, L.b, L.nkb, p, exps, L.rs);
+        if (launch_status()) return HBFP_ERR_CUDA;
+        dim3 grid((unsigned)((L.kst + 511) / 512), (unsigned)((rows + 31) / 32));
+#define HBFP_QROW_GIVEN(SRV, PL) quant_row_fast<16, SRV, PL><<<grid, 256, 0, st>>>(x, rows, K, ld, p, mant, L.kst, L.plane_stride, exps, L.rs, L.nkb, exps)
+        if (p.rounding == 1) { if (L.planes == 1) HBFP_QROW_GIVEN(true, 1); else HBFP_QROW_GIVEN(true, 2); }
+        else { if (L.planes == 1) HBFP_QROW_GIVEN(false, 1); else HBFP_QROW_GIVEN(false, 2); }
+#undef HBFP_QROW_GIVEN
+        return launch_status();
     }
     if (f->tile == 0 && axis == 1 && aligned && d1 % 8 == 0 && L.b == L.bp && L.b <= 256 &&
         rows <= 32ll * 65535) {

@@ -123,6 +123,21 @@ def test_column_blocks_over_the_whole_axis(hb, shape, law, fd):
     _check(hb, wl.draw(law, shape, seed=16), 0, fd)
 
 
+# The same for rows: one exponent per row over more than 256 columns (row maxima first, then the fast row kernel with
+# the exponents given).
+ROW_WHOLE_AXIS_CASES = [
+    ((200, 1032), "lognormal", F(8, 0, rounding=1, seed=6, sid=3)),         # ragged last column tile, stochastic
+    ((1000, 2048), "outliers", F(8, 0, exp_mode=1)),
+    ((72, 384), "grad", F(12, 0, rounding=1, seed=2)),                      # two planes
+    ((33, 264), "normal", F(4, 0)),                                         # ragged last row tile
+]
+
+
+@pytest.mark.parametrize("shape,law,fd", ROW_WHOLE_AXIS_CASES)
+def test_row_blocks_over_the_whole_axis(hb, shape, law, fd):
+    _check(hb, wl.draw(law, shape, seed=17), 1, fd)
+
+
 def test_column_blocks_of_a_pitched_view(hb):
     # a 16-byte aligned column window of a wider matrix: the pitch differs from the logical width,
     # and the stochastic stream follows the logical index of the window
