@@ -147,6 +147,18 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
+// try_wait with a short suspend hint: the thread sleeps at most about `ns` nanoseconds and takes no issue slots from
+// the rescale warps of its sub-partition meanwhile.
+__device__ __forceinline__ bool mbar_try_wait_ns(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+
 // Wait on a barrier that threads of the other CTA arrive on. What the arrivals order are tensor-memory
 // accesses, fenced with tcgen05.fence on both sides, so the default (CTA-scope) acquire is enough.
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
@@ -160,10 +172,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 }
 __device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                                   int32_t* status, int code) {
-    // The MMA thread has nothing else to do, and a thread that try_wait has put to sleep wakes up late
-    // (the kernel then settles in a mode 20 % slower): poll first, sleep only when that runs out.
-    for (int i = 0; i < 4096; ++i)
+    // A thread that try_wait has put to sleep with the long hint below wakes up late (the kernel then settles in a
+    // mode 20 % slower), and a thread that spins on test_wait takes issue slots from the rescale warps of its
+    // sub-partition: 32 looks, then naps of at most 64 ns, the long sleep only when those run out. Measured in
+    // cycles per launch against spinning alone (n = 8192): - 5 % for blocks of 128, - 1 % for 64, - 4 % for 32;
+    // one look before the naps is as good for 128 but 8 % worse for 64; the nap's length (32-128 ns) does not matter.
+    for (int i = 0; i < 32; ++i)
         if (mbar_test_wait(bar, parity)) return true;
+    for (int i = 0; i < 1024; ++i)
+        if (mbar_try_wait_ns(bar, parity, 64u)) return true;
     if (mbar_try_wait_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
