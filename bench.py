@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # with the summary of the single-pass ncu capture it was read from. A workload without an entry reports
 # no traffic.
 GEMM_DRAM_TRAFFIC = {
-    ("gemm_tc2_kernel", 16384, 8, 128): {"bytes": 4854548480 + 1078018048,
+    ("gemm_tc2_kernel", 16384, 8, 128): {"bytes": 4891126016 + 1062103040,
                                          "profile": "profiles/bench_launch_list_n16384_m8_b128.md"},
 }
 SUSTAINED_SECONDS = 2.5       # length of the back-to-back GEMM loop behind `gemm_sustained`
