@@ -14,6 +14,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhbfp.so")
 SOURCES = ["api.cu", "quantize.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_conv.cu", "gemm_static.cu"]
+# (object name, source, extra flags): quantize.cu is compiled a second time for the full-tile kernel of small tiles
+EXTRA_OBJECTS = [("quantize_tiles_small.o", "quantize.cu", ["-DHBFP_QUANT_PART=2", "-Xptxas", "-O1"])]
 # Per-file additions. The paired-SM GEMM is built with ptxas -O1: measured in SM cycles per launch (16384^3, b = 128)
 # 8.57 M against 8.86 M at the default level, and 12 % / 9 % fewer cycles for blocks of 64 / 32; the other files were
 # measured too and are a toss-up kernel by kernel (single-SM GEMM: 8-bit + 9 %, 12-bit - 6 %), so they keep the default.
@@ -51,6 +53,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    for obj_name, src, flags in EXTRA_OBJECTS:
+        obj = os.path.join(objdir, obj_name)
+        objs.append(obj)
+        cmd = ["nvcc", *NVCC_FLAGS, *flags, "-c", os.path.join(CSRC, src), "-o", obj]
+        procs.append((obj_name, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
     failed = False
     for src, p in procs:
         out, _ = p.communicate()
