@@ -251,7 +251,7 @@ def gpu_arm(args):
     # to the single call (row panels are independent); stochastic rounding keys its draws to the index inside
     # the matrix as passed, so there the single hbfp_gemm call is timed instead.
     e2e_steps = max(1, min(args.steps, 3))
-    panels = 8 if (args.rounding == 0 and n % (8 * 256) == 0) else 1
+    panels = args.e2e_panels if (args.rounding == 0 and n % (args.e2e_panels * 256) == 0) else 1
     rows_p = n // panels
     if panels > 1:
         s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
@@ -474,6 +474,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quantize-line", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the few-second back-to-back GEMM loop")
+    ap.add_argument("--e2e-panels", type=int, default=8, help="row panels of A in the end-to-end leg")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
