@@ -146,6 +146,24 @@ HBFP_API int hbfp_quantize_conv_weights(const float* w, int64_t taps, int64_t c_
                                         const hbfp_format* fmt, void* mant_c0, int8_t* exps_c0, void* mant_c1,
                                         int8_t* exps_c1, int8_t* tile_exps, void* stream);
 
+/* Filter operand of the backward-data convolution (Sec. 5.1: the backward pass of a convolution runs through
+ * the same BFP dot products; Sec. 4.2: the weight tiles are shared between the passes). For a kh x kw filter,
+ * stride 1, the gradient with respect to the input is the convolution of the output gradient with the
+ * filters turned by 180 degrees and with the roles of input and output maps swapped:
+ *   dX[p][ci] = sum over taps and co of dY[p + (pad' - tap')][co] * w[(taps - 1 - tap'), ci, co],  pad' = k - 1 - pad.
+ * This call builds that operand, rows = c_in, contraction = taps x c_out, from view c1 of
+ * hbfp_quantize_conv_weights (mant_c1 / exps_c1: rows = taps * c_in, contraction = c_out; device, 256-byte
+ * aligned mantissas) by copying packed bytes and tile exponents: no value is converted again, so forward and
+ * backward-data use the same mantissas. fmt: the format the weights were converted with (tile == block = t).
+ * mant_out / exps_out: device buffers of the sizes hbfp_packed_sizes(c_in, taps * c_out, fmt) returns, mantissas
+ * 256-byte aligned, fully overwritten. hbfp_conv_forward on the packed output gradient (block = c_out) with this
+ * operand, `filters` = c_in and padding pad' then yields dX without the FP32 matrix of im2col-shaped gradients.
+ * One launch, asynchronous on `stream`. Errors: HBFP_ERR_INVALID_ARG (null pointers, tile != block, sizes <= 0),
+ * HBFP_ERR_UNSUPPORTED (t not 32, 64 or 128, or c_in or c_out not a multiple of t), HBFP_ERR_ALIGNMENT. */
+HBFP_API int hbfp_conv_dgrad_filters(const void* mant_c1, const int8_t* exps_c1, int kh, int kw, int64_t c_in,
+                                     int64_t c_out, const hbfp_format* fmt, void* mant_out, int8_t* exps_out,
+                                     void* stream);
+
 /* Wide weight storage (Sec. 4.2 "Wide weight storage": weights are kept with wider mantissas, only
  * weight updates use them, and the forward and backward passes read only the most significant bits).
  * The long-lived copy of w [d0][d1] is `wide`: int16 mantissas, row-major with pitch d1 (device,

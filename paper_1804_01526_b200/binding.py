@@ -28,7 +28,7 @@ EXPORTS = [
     "hbfp_quantize_tiles", "hbfp_unpack", "hbfp_dequantize", "hbfp_gemm_workspace",
     "hbfp_gemm_q_workspace", "hbfp_gemm", "hbfp_gemm_q", "hbfp_gemm_block_partials",
     "hbfp_device_status", "hbfp_gemm_static", "hbfp_wide_quantize", "hbfp_wide_update", "hbfp_wide_narrow",
-    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel", "hbfp_last_gemm_cycles", "hbfp_conv_forward", "hbfp_quantize_conv_weights",
+    "hbfp_im2col_packed", "hbfp_im2col_packed_t", "hbfp_wide_dequantize", "hbfp_selftest_bounded_wait", "hbfp_last_gemm_kernel", "hbfp_last_gemm_cycles", "hbfp_conv_forward", "hbfp_quantize_conv_weights", "hbfp_conv_dgrad_filters",
 ]
 
 
@@ -106,6 +106,7 @@ def lib() -> ctypes.CDLL:
         L.hbfp_device_status.argtypes = [p, p]
         L.hbfp_quantize_conv_weights.argtypes = [p, i64, i64, i64, i64, p, p, p, p, p, p, p]
         L.hbfp_conv_forward.argtypes = [p, p, i64, i64, i64, i64, i32, i32, i32, p, p, i64, p, i64, p]
+        L.hbfp_conv_dgrad_filters.argtypes = [p, p, i32, i32, i64, i64, p, p, p, p]
         L.hbfp_wide_dequantize.argtypes = [p, p, i64, i64, i32, p, i64, p]
         L.hbfp_selftest_bounded_wait.argtypes = [i64, i32, p, p]
         L.hbfp_last_gemm_cycles.argtypes = [p]
@@ -303,13 +304,13 @@ def im2col_packed(px: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, 
     return out
 
 
-def quantize_conv_weights(w: torch.Tensor, taps: int, fmt: Format, want_grid: bool = False):
+def quantize_conv_weights(w: torch.Tensor, taps: int, fmt: Format, want_grid: bool = False, out=None):
     """hbfp_quantize_conv_weights: convolution weights ``w [taps * c_in][c_out]`` with one exponent per tile of
     ``t`` input maps x ``t`` output maps over all taps. Returns ``(c0, c1, grid or None)``."""
     _check_f32(w, "w")
     d0, d1 = w.shape
     c_in = d0 // taps
-    c0, c1 = _alloc_views(d0, d1, fmt, w.device)
+    c0, c1 = out if out is not None else _alloc_views(d0, d1, fmt, w.device)
     t = fmt.tile
     grid = torch.empty((c_in // t, -(-d1 // t)), dtype=torch.int8, device=w.device) if want_grid else None
     f = fmt.c()
@@ -317,6 +318,17 @@ def quantize_conv_weights(w: torch.Tensor, taps: int, fmt: Format, want_grid: bo
                                             _dptr(c1.mant), _dptr(c1.exps), _dptr(grid) if grid is not None else None,
                                             _stream()), "hbfp_quantize_conv_weights")
     return c0, c1, grid
+
+
+def conv_dgrad_filters(c1: Packed, kh: int, kw: int, c_in: int, c_out: int, out: Optional[Packed] = None) -> Packed:
+    """hbfp_conv_dgrad_filters: the filter operand of the backward-data convolution (rows = c_in, k = kh*kw*c_out)
+    from view ``c1`` of ``quantize_conv_weights``: the forward pass's mantissas and tile exponents, taps reversed."""
+    if out is None:
+        out = alloc_packed(c_in, kh * kw * c_out, c1.fmt, c1.mant.device)
+    f = c1.fmt.c()
+    _check(lib().hbfp_conv_dgrad_filters(_dptr(c1.mant), _dptr(c1.exps), kh, kw, c_in, c_out, ctypes.byref(f), _dptr(out.mant),
+                                         _dptr(out.exps), _stream()), "hbfp_conv_dgrad_filters")
+    return out
 
 
 def conv_forward(px: Packed, filters: Packed, n: int, h: int, w: int, c: int, kh: int, kw: int, pad: int,

@@ -315,6 +315,29 @@ int hbfp_conv_forward(const void* mant_x, const int8_t* exps_x, int64_t n, int64
     return launch_conv_forward(px, pw, n, h, w, c, kh, kw, pad, filters, Y, ldy, static_cast<cudaStream_t>(stream));
 }
 
+int hbfp_conv_dgrad_filters(const void* mant_c1, const int8_t* exps_c1, int kh, int kw, int64_t c_in, int64_t c_out,
+                            const hbfp_format* fmt, void* mant_out, int8_t* exps_out, void* stream) {
+    if (!fmt || kh <= 0 || kw <= 0 || c_in < 0 || c_out <= 0) return HBFP_ERR_INVALID_ARG;
+    if (!mant_c1 || !exps_c1 || !mant_out || !exps_out) return HBFP_ERR_INVALID_ARG;
+    const int64_t t = fmt->tile;
+    if (t <= 0 || fmt->block != t) return HBFP_ERR_INVALID_ARG;
+    // whole 16-byte pieces of unpadded blocks: tiles of 32, 64 or 128 output maps
+    if ((t != 32 && t != 64 && t != 128) || c_out % t != 0 || c_in % t != 0) return HBFP_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(mant_c1) & 255) || (reinterpret_cast<uintptr_t>(mant_out) & 255)) return HBFP_ERR_ALIGNMENT;
+    const int64_t taps = (int64_t)kh * kw;
+    Packed c1;
+    Layout Lo;
+    int rc = make_layout(taps * c_in, c_out, fmt, &c1.L);
+    if (rc) return rc;
+    rc = make_layout(c_in, taps * c_out, fmt, &Lo);
+    if (rc) return rc;
+    c1.mant = static_cast<const int8_t*>(mant_c1);
+    c1.exps = exps_c1;
+    c1.mant_bits = fmt->mant_bits;
+    return launch_conv_dgrad_filters(c1, (int)taps, c_in, c_out, (int)t, static_cast<int8_t*>(mant_out), exps_out, Lo,
+                                     static_cast<cudaStream_t>(stream));
+}
+
 int hbfp_im2col_packed_t(const float* x, int64_t n, int64_t h, int64_t w, int64_t c, int kh, int kw, int pad,
                          const hbfp_format* fmt, void* mant, int8_t* exps, void* stream) {
     if (!fmt || n < 0 || h <= 0 || w <= 0 || c <= 0 || kh <= 0 || kw <= 0 || pad < 0) return HBFP_ERR_INVALID_ARG;

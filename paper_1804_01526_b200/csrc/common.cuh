@@ -117,6 +117,8 @@ int launch_conv_forward(const Packed& x, const Packed& wt, int64_t n, int64_t h,
 
 // One warp running the kernels' bounded barrier wait on a barrier nobody arrives on (test hook).
 int launch_wait_probe(long long limit_cycles, int code, int* outcome, cudaStream_t st);
+int launch_conv_dgrad_filters(const Packed& c1, int taps, int64_t c_in, int64_t c_out, int t, int8_t* mant_out,
+                              int8_t* exps_out, const Layout& Lo, cudaStream_t st);
 int pair_gemm_cycles(uint64_t* cycles);   // longest CTA of the last paired-SM GEMM launch on the current device, in SM cycles
 
 // Device status word (bounded waits report here).

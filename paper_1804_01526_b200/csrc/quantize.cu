@@ -865,32 +865,48 @@ __global__ void exps_tiles(const float* __restrict__ x, int64_t d0, int64_t d1, 
 }
 
 // Pass 1d, convolution weights [taps * c_in][c_out] (Sec. 5.1: the two feature-map dimensions are tiled, the
-// filter taps are not): one warp per (input-map tile u, output-map tile v) takes the maximum over every tap
-// and repeats the tile's exponent for every line and K-block of the view that crosses the tile.
-__global__ void exps_conv_tiles(const float* __restrict__ x, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld,
-                                int64_t t, QParams p, int axis, int8_t* __restrict__ exps, int64_t rs, int64_t nu,
-                                int64_t nv, int8_t* __restrict__ tile_exps) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (warp >= nu * nv) return;
-    const int64_t u = warp / nv, v = warp % nv;
+// filter taps are not): one CTA per (input-map tile u, output-map tile v) takes the maximum over every tap
+// (a warp per weight row, lanes along the output maps) and repeats the tile's exponent for every line and
+// K-block of the two views that cross the tile.
+constexpr int CONVW_THREADS = 512;
+__global__ void __launch_bounds__(CONVW_THREADS)
+exps_conv_tiles(const float* __restrict__ x, int64_t taps, int64_t c_in, int64_t c_out, int64_t ld, int64_t t, QParams p,
+                int8_t* __restrict__ exps0, int64_t rs0, int8_t* __restrict__ exps1, int64_t rs1, int64_t nu, int64_t nv,
+                int8_t* __restrict__ tile_exps, uint32_t* __restrict__ amax, bool fill) {
+    __shared__ uint32_t part[CONVW_THREADS / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t u = blockIdx.x / nv, v = blockIdx.x % nv;
     const int64_t j1 = min(c_out, (v + 1) * t);
     uint32_t am = 0;
-    for (int64_t tap = 0; tap < taps; ++tap)
-        for (int64_t ci = u * t; ci < (u + 1) * t; ++ci)
-            for (int64_t j = v * t + lane; j < j1; j += 32) am = max(am, abs_bits(x[(tap * c_in + ci) * ld + j]));
-    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
-    const int8_t s = (int8_t)block_exponent(am, p.m, p.exp_mode);
-    if (tile_exps && lane == 0) tile_exps[u * nv + v] = s;
-    if (!exps) return;
-    // axis 0 (forward view): lines are output maps, K-block (tap, u). axis 1: lines are (tap, ci), K-block v.
-    if (axis == 0) {
-        for (int64_t tap = 0; tap < taps; ++tap)
-            for (int64_t j = v * t + lane; j < j1; j += 32) exps[(tap * nu + u) * rs + j] = s;
-    } else {
-        for (int64_t tap = 0; tap < taps; ++tap)
-            for (int64_t ci = u * t + lane; ci < (u + 1) * t; ci += 32) exps[v * rs + tap * c_in + ci] = s;
+    // with `amax` the rows are split over gridDim.y CTAs that merge their maxima there (exponents come from a
+    // second launch with `fill`); without it this CTA scans the whole tile
+    for (int64_t r = (int64_t)blockIdx.y * (CONVW_THREADS / 32) + warp; !fill && r < taps * t; r += (int64_t)gridDim.y * (CONVW_THREADS / 32)) {
+        const int64_t tap = r / t, ci = u * t + r % t;
+        for (int64_t j = v * t + lane; j < j1; j += 32) am = max(am, abs_bits(x[(tap * c_in + ci) * ld + j]));
     }
+    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    if (lane == 0) part[warp] = am;
+    __syncthreads();
+    am = part[0];
+    for (int i = 1; i < CONVW_THREADS / 32; ++i) am = max(am, part[i]);
+    if (amax && !fill) {
+        if (threadIdx.x == 0) atomicMax(amax + blockIdx.x, am);
+        return;
+    }
+    if (fill) am = amax[blockIdx.x];
+    const int8_t s = (int8_t)block_exponent(am, p.m, p.exp_mode);
+    if (tile_exps && threadIdx.x == 0) tile_exps[u * nv + v] = s;
+    // view c0 (forward): lines are output maps, K-block (tap, u). view c1: lines are (tap, ci), K-block v.
+    if (exps0)
+        for (int64_t i = threadIdx.x; i < taps * (j1 - v * t); i += CONVW_THREADS) {
+            const int64_t tap = i / (j1 - v * t), j = v * t + i % (j1 - v * t);
+            exps0[(tap * nu + u) * rs0 + j] = s;
+        }
+    if (exps1)
+        for (int64_t i = threadIdx.x; i < taps * t; i += CONVW_THREADS) {
+            const int64_t tap = i / t, ci = u * t + i % t;
+            exps1[v * rs1 + tap * c_in + ci] = s;
+        }
 }
 
 // Pass 2: one thread per 4 output bytes of a line; reads the exponent written by pass 1.
@@ -1112,6 +1128,32 @@ im2col_cols(const float* __restrict__ x, int h, int w, int lg_w, int c, int kh, 
             }
         }
     }
+}
+
+// Filter operand of the backward-data convolution from view c1 of tiled convolution weights: row ci of the result
+// is, tap by tap in reversed order, the c_out packed bytes of c1's row (tap, ci) (Sec. 5.1: backward-data is the
+// convolution of the output gradient with the filters turned by 180 degrees and their feature-map roles swapped;
+// the mantissas and tile exponents are the forward pass's own). One warp per (ci, tap), 16 bytes per lane.
+__global__ void __launch_bounds__(256)
+conv_dgrad_filters_kernel(const int8_t* __restrict__ m1, const int8_t* __restrict__ e1, int64_t kst1, int64_t ps1,
+                          int64_t rs1, int taps, int64_t c_in, int64_t c_out, int t, int planes,
+                          int8_t* __restrict__ mo, int8_t* __restrict__ eo, int64_t ksto, int64_t pso, int64_t rso) {
+    const int lane = threadIdx.x & 31;
+    const int64_t item = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (item >= c_in * taps) return;
+    const int64_t ci = item / taps;
+    const int tap = (int)(item - ci * taps);
+    const int64_t src_row = (int64_t)(taps - 1 - tap) * c_in + ci;
+    for (int pl = 0; pl < planes; ++pl)
+        for (int64_t o = 16 * lane; o < c_out; o += 512)
+            *reinterpret_cast<uint4*>(mo + pl * pso + ci * ksto + (int64_t)tap * c_out + o) =
+                *reinterpret_cast<const uint4*>(m1 + pl * ps1 + src_row * kst1 + o);
+    const int cb_n = (int)(c_out / t);
+    for (int cb = lane; cb < cb_n; cb += 32) eo[((int64_t)tap * cb_n + cb) * rso + ci] = e1[(int64_t)cb * rs1 + src_row];
+    // bytes of the row beyond the last tap (the row pitch is a multiple of 128)
+    if (tap == taps - 1)
+        for (int64_t o = (int64_t)taps * c_out + 16 * lane; o < ksto; o += 512)
+            for (int pl = 0; pl < planes; ++pl) *reinterpret_cast<uint4*>(mo + pl * pso + ci * ksto + o) = make_uint4(0u, 0u, 0u, 0u);
 }
 
 // ------------------------------------------------------------------------------ inverse helpers
@@ -1699,27 +1741,43 @@ int launch_quantize_conv_weights(const float* w, int64_t taps, int64_t c_in, int
     if (c_in % t != 0) return HBFP_ERR_UNSUPPORTED;               // a K-block must not straddle two taps
     const int64_t d0 = taps * c_in, d1 = c_out, nu = c_in / t, nv = (c_out + t - 1) / t;
     const QParams p = make_params(f);
+    if (nu * nv >= (1ll << 31)) return HBFP_ERR_UNSUPPORTED;
+    Layout L[2];
     for (int axis = 0; axis < 2; ++axis) {
-        int8_t* mant = axis == 0 ? mant_c0 : mant_c1;
         int8_t* exps = axis == 0 ? exps_c0 : exps_c1;
-        if (!mant) continue;
-        Layout L;
-        const int64_t rows = axis == 0 ? d1 : d0, K = axis == 0 ? d0 : d1;
-        int rc = make_layout(rows, K, f, &L);
+        if (!(axis == 0 ? mant_c0 : mant_c1)) continue;
+        int rc = make_layout(axis == 0 ? d1 : d0, axis == 0 ? d0 : d1, f, &L[axis]);
         if (rc) return rc;
-        HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
-        exps_conv_tiles<<<blocks_for(nu * nv * 32, 256), 256, 0, st>>>(w, taps, c_in, c_out, ld, t, p, axis, exps, L.rs, nu, nv,
-                                                                      tile_exps);
-        if (launch_status()) return HBFP_ERR_CUDA;
-        if (L.planes == 1)
-            mant_generic<1><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(w, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
-        else
-            mant_generic<2><<<blocks_for(rows * (L.kst / 4), 256), 256, 0, st>>>(w, d1, rows, K, ld, axis, L.b, L.bp, L.nkb, p, exps, L.rs, mant, L.kst, L.plane_stride);
+        if (L[axis].rs != L[axis].rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L[axis].exp_bytes, st));   // padding lines are zero
+    }
+    if (!mant_c0 && !mant_c1 && !tile_exps) return HBFP_OK;
+    // few tiles: split each tile's rows over several CTAs, maxima merged in the head of a mantissa buffer (the
+    // mantissa pass that follows overwrites it)
+    int8_t* const scratch_buf = mant_c1 ? mant_c1 : mant_c0;
+    const int64_t scratch_room = !scratch_buf ? 0 : (mant_c1 ? L[1].mant_bytes : L[0].mant_bytes);
+    int64_t splits = (2 * 148 + nu * nv - 1) / (nu * nv);
+    splits = std::min<int64_t>(splits, (taps * t + CONVW_THREADS / 32 - 1) / (CONVW_THREADS / 32));
+    for (int pass = 0; pass < 2; ++pass) {
+        uint32_t* amax = nullptr;
+        if (splits > 1 && nu * nv * 4 <= scratch_room) amax = reinterpret_cast<uint32_t*>(scratch_buf);
+        if (pass == 1 && !amax) break;
+        if (pass == 0 && amax) HBFP_CUDA_OK(cudaMemsetAsync(amax, 0, (size_t)(nu * nv * 4), st));
+        const dim3 grid((unsigned)(nu * nv), pass == 0 && amax ? (unsigned)splits : 1u);
+        exps_conv_tiles<<<grid, CONVW_THREADS, 0, st>>>(w, taps, c_in, c_out, ld, t, p, mant_c0 ? exps_c0 : nullptr,
+                                                        mant_c0 ? L[0].rs : 0, mant_c1 ? exps_c1 : nullptr,
+                                                        mant_c1 ? L[1].rs : 0, nu, nv, tile_exps, amax, pass == 1);
         if (launch_status()) return HBFP_ERR_CUDA;
     }
-    if (!mant_c0 && !mant_c1 && tile_exps) {
-        exps_conv_tiles<<<blocks_for(nu * nv * 32, 256), 256, 0, st>>>(w, taps, c_in, c_out, ld, t, p, 0, nullptr, 0, nu, nv, tile_exps);
-        return launch_status();
+    for (int axis = 0; axis < 2; ++axis) {
+        int8_t* mant = axis == 0 ? mant_c0 : mant_c1;
+        const int8_t* exps = axis == 0 ? exps_c0 : exps_c1;
+        if (!mant) continue;
+        const Layout& A = L[axis];
+        if (A.planes == 1)
+            mant_generic<1><<<blocks_for(A.rows * (A.kst / 4), 256), 256, 0, st>>>(w, d1, A.rows, A.k, ld, axis, A.b, A.bp, A.nkb, p, exps, A.rs, mant, A.kst, A.plane_stride);
+        else
+            mant_generic<2><<<blocks_for(A.rows * (A.kst / 4), 256), 256, 0, st>>>(w, d1, A.rows, A.k, ld, axis, A.b, A.bp, A.nkb, p, exps, A.rs, mant, A.kst, A.plane_stride);
+        if (launch_status()) return HBFP_ERR_CUDA;
     }
     return HBFP_OK;
 }
@@ -1796,6 +1854,17 @@ int launch_im2col_cols(const float* x, int64_t n, int64_t h, int64_t w, int64_t 
     }
 #undef HBFP_COLS_LAUNCH2
 #undef HBFP_COLS_LAUNCH
+    return launch_status();
+}
+
+int launch_conv_dgrad_filters(const Packed& c1, int taps, int64_t c_in, int64_t c_out, int t, int8_t* mant_out,
+                              int8_t* exps_out, const Layout& Lo, cudaStream_t st) {
+    if (c_in == 0) return HBFP_OK;
+    if (Lo.rs != c_in) HBFP_CUDA_OK(cudaMemsetAsync(exps_out, 0, (size_t)Lo.exp_bytes, st));   // padding lines are zero
+    const int64_t warps = c_in * taps;
+    conv_dgrad_filters_kernel<<<blocks_for(warps * 32, 256), 256, 0, st>>>(c1.mant, c1.exps, c1.L.kst, c1.L.plane_stride, c1.L.rs,
+                                                                          taps, c_in, c_out, t, (int)c1.L.planes, mant_out, exps_out,
+                                                                          Lo.kst, Lo.plane_stride, Lo.rs);
     return launch_status();
 }
 

@@ -139,6 +139,30 @@ def conv_lines():
         out.append(f"| {name} {M}x{f}x{K} | {M*K*4/1e6:.0f} | {t_c*1e3:.1f} | {t_p*1e3:.1f} | {t_g*1e3:.1f} | {t_m*1e3:.1f} | {t_i*1e3:.1f} ({M*f*4/(t_i*1e-3)/1e9:.0f}) | {t_ct*1e3:.1f} | {t_t*1e3:.1f} |")
         del x, x4, wt, px, pa, pw, cols, pc, C, ws, pt, pt2
     torch.cuda.empty_cache()
+    # backward-data: the product dY x W^T in the im2col shape (its FP32 result still has to be folded back onto the
+    # pixels) against the convolution of the packed dY with the regrouped forward weights, which yields dX itself
+    out += ["", "| convolution | convert dY (one block per pixel) µs | weights tiled over the feature maps µs | dY·Wᵀ GEMM, im2col-shaped FP32 result µs (MB written) | "
+            "regroup filters (`hbfp_conv_dgrad_filters`) µs | implicit backward-data µs (MB written) |", "|---|---|---|---|---|---|"]
+    for name, n, hw, c, f in (("c2.conv64", 128, 32, 64, 64), ("c2.conv128", 128, 16, 128, 128)):
+        M = n * hw * hw
+        fg = hb.Format(mant_bits=8, block=f, rounding=1, seed=3)
+        fw = hb.Format(mant_bits=8, block=f, tile=f)
+        dy = torch.from_numpy(wl.draw("normal", (M, f), seed=7)).cuda()
+        wt = torch.from_numpy(wl.draw("he_weight", (9 * c, f), seed=6, fan_in=9 * c)).cuda()
+        pg = hb.quantize(dy, 1, fg)
+        t_g = _time_auto(lambda: hb.quantize(dy, 1, fg, out=pg))
+        c0, c1, _ = hb.quantize_conv_weights(wt, 9, fw)
+        t_w = _time_auto(lambda: hb.quantize_conv_weights(wt, 9, fw, out=(c0, c1)))
+        dcols = torch.empty((M, 9 * c), dtype=torch.float32, device="cuda")
+        ws = torch.empty(max(hb.gemm_q_workspace(M, 9 * c, f, pg, c1), 1), dtype=torch.int8, device="cuda")
+        t_m = _time_auto(lambda: hb.gemm_q(M, 9 * c, f, pg, c1, out=dcols, workspace=ws))
+        d = hb.conv_dgrad_filters(c1, 3, 3, c, f)
+        t_d = _time_auto(lambda: hb.conv_dgrad_filters(c1, 3, 3, c, f, out=d))
+        dx = torch.empty((M, c), dtype=torch.float32, device="cuda")
+        t_i = _time_auto(lambda: hb.conv_forward(pg, d, n, hw, hw, f, 3, 3, 1, out=dx))
+        out.append(f"| {name} dX {M}x{c}, K = {9*f} | {t_g*1e3:.1f} | {t_w*1e3:.1f} | {t_m*1e3:.1f} ({M*9*c*4/1e6:.0f}) | {t_d*1e3:.1f} | {t_i*1e3:.1f} ({M*c*4/1e6:.0f}) |")
+        del dy, wt, pg, c0, c1, dcols, ws, d, dx
+    torch.cuda.empty_cache()
     return out
 
 

@@ -39,3 +39,13 @@ def decode_packed(p, lay):
     e = exps[: nkb * rs].reshape(nkb, rs)
     assert not e[:, rows:].any(), "exponent padding must be zero"
     return q.astype(np.int16), np.ascontiguousarray(e[:, :rows].T)
+
+
+def dgrad_filters_view(q1: np.ndarray, s1: np.ndarray, taps: int, c_in: int) -> tuple:
+    """Regroup a ``[taps * c_in][c_out]`` array (and its per-row block array) into the filter operand of the
+    backward-data convolution, ``[c_in][taps * c_out]``: row ci holds, tap by tap, the row (taps - 1 - tap, ci)
+    of the input (filters turned by 180 degrees, feature-map roles swapped). Pure index movement."""
+    c_out, nb = q1.shape[1], s1.shape[1]
+    q = q1.reshape(taps, c_in, c_out)[::-1].transpose(1, 0, 2).reshape(c_in, taps * c_out)
+    s = s1.reshape(taps, c_in, nb)[::-1].transpose(1, 0, 2).reshape(c_in, taps * nb)
+    return np.ascontiguousarray(q), np.ascontiguousarray(s)

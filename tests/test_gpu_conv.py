@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 from paper_1804_01526_b200 import workloads as wl
-from tests.helpers import decode_packed, gfmt, ofmt, to_dev
+from tests.helpers import decode_packed, dgrad_filters_view, gfmt, ofmt, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -195,7 +195,7 @@ def test_implicit_gemm_convolution_says_what_it_does_not_cover(hb):
 
 
 @pytest.mark.parametrize("taps,c_in,c_out,t,m,rounding", [(9, 64, 64, 64, 8, 0), (9, 128, 96, 32, 8, 1), (25, 24, 40, 24, 6, 0),
-                                                          (1, 64, 130, 64, 12, 1)])
+                                                          (1, 64, 130, 64, 12, 1), (4, 576, 560, 32, 8, 0)])
 def test_convolution_weights_tiled_on_the_feature_map_dimensions(hb, taps, c_in, c_out, t, m, rounding):
     """hbfp_quantize_conv_weights against the oracle: one exponent per (t input maps x t output maps) tile over
     every filter tap, both views bit-exact."""
@@ -242,3 +242,64 @@ def test_gathered_operand_under_stochastic_rounding_takes_each_activations_draw(
     q_ref, s_ref = oracle.quantize_indexed(oracle.im2col(x, 3, 3, 1), 1, ofmt(fd), oracle.im2col_index(n, h, w, c, 3, 3, 1))
     q, s = decode_packed(pa, hb.packed_layout(pa.rows, pa.k, pa.fmt))
     assert np.array_equal(q, q_ref) and np.array_equal(s, s_ref)
+
+
+@pytest.mark.parametrize("k,c_in,c_out,t,m,rounding", [(3, 64, 64, 64, 8, 0), (3, 128, 64, 64, 8, 1), (5, 64, 128, 32, 6, 0),
+                                                       (1, 128, 256, 128, 12, 1), (3, 32, 96, 32, 12, 0)])
+def test_backward_data_filter_operand_is_a_regrouping_of_the_forward_weights(hb, k, c_in, c_out, t, m, rounding):
+    """hbfp_conv_dgrad_filters moves bytes and tile exponents only: decoded, the operand is the oracle's view c1
+    with taps reversed and rows regrouped by input map."""
+    taps = k * k
+    w = wl.draw("he_weight", (taps * c_in, c_out), seed=91, fan_in=taps * c_in)
+    w *= np.exp(wl.draw("normal", (taps * c_in, 1), seed=92)).astype(np.float32)
+    fd = dict(mant_bits=m, block=t, tile=t, rounding=rounding, seed=5, stream_id=2)
+    _, c1, _ = hb.quantize_conv_weights(to_dev(w), taps, gfmt(fd))
+    d = hb.conv_dgrad_filters(c1, k, k, c_in, c_out)
+    assert hb.device_status() == 0
+    assert (d.rows, d.k) == (c_in, taps * c_out)
+    q1, s1 = oracle.quantize_conv_weights(w, taps, 1, ofmt(fd))
+    qd, sd = dgrad_filters_view(q1, s1, taps, c_in)
+    gd, ed = decode_packed(d, hb.packed_layout(d.rows, d.k, d.fmt))
+    assert np.array_equal(gd, qd) and np.array_equal(ed, sd)
+
+
+@pytest.mark.parametrize("n,h,w_,c_in,c_out,k,pad", [(2, 32, 32, 64, 64, 3, 1), (3, 16, 16, 128, 128, 3, 1), (2, 16, 16, 128, 64, 3, 1),
+                                                     (1, 8, 16, 128, 128, 5, 2), (2, 4, 64, 64, 64, 1, 0), (1, 16, 32, 256, 64, 3, 1)])
+def test_backward_data_convolution_on_the_packed_gradient_equals_oracle(hb, n, h, w_, c_in, c_out, k, pad):
+    """dX as an implicit GEMM: the packed output gradient (one block per pixel) against the regrouped forward
+    weights, padding k - 1 - pad. Expected: the oracle's GEMM on the oracle's quantised gather of dY and the
+    oracle's tiled weights regrouped the same way, bit for bit in the sequential order."""
+    taps = k * k
+    ho, wo = h + 2 * pad - k + 1, w_ + 2 * pad - k + 1
+    dy = wl.draw("normal", (n * ho * wo, c_out), seed=93).reshape(n, ho, wo, c_out)
+    dy *= np.exp(2 * wl.draw("normal", (n * ho * wo, 1), seed=94)).reshape(n, ho, wo, 1).astype(np.float32) * 1e-3
+    wt = wl.draw("he_weight", (taps * c_in, c_out), seed=95, fan_in=taps * c_in)
+    fg = dict(mant_bits=8, block=c_out, rounding=1, seed=11, stream_id=3)
+    fw = dict(mant_bits=8, block=c_out, tile=c_out, stream_id=1)
+    pg = hb.quantize(to_dev(dy.reshape(n * ho * wo, c_out)), 1, gfmt(fg))
+    _, c1, _ = hb.quantize_conv_weights(to_dev(wt), taps, gfmt(fw))
+    d = hb.conv_dgrad_filters(c1, k, k, c_in, c_out)
+    dX = hb.conv_forward(pg, d, n, ho, wo, c_out, k, k, k - 1 - pad).cpu().numpy()
+    assert hb.device_status() == 0
+    assert hb.last_gemm_kernel() == "conv_fwd_kernel"
+    assert dX.shape == (n * h * w_, c_in)
+    # the oracle's side: every block of the gathered gradient is the pixel's own block (one conversion per pixel,
+    # stochastic draws keyed by the element's index in dY), so gather the canonical arrays of the pixels
+    qp, sp = oracle.quantize(dy.reshape(n * ho * wo, c_out), 1, ofmt(fg))
+    qa = oracle.im2col(qp.reshape(n, ho, wo, c_out), k, k, k - 1 - pad)
+    sa = oracle.im2col(sp.reshape(n, ho, wo, 1), k, k, k - 1 - pad)
+    q1, s1 = oracle.quantize_conv_weights(wt, taps, 1, ofmt(fw))
+    qb, sb = dgrad_filters_view(q1, s1, taps, c_in)
+    ref = oracle.gemm(qa, sa, qb, sb, c_out)
+    err = np.abs(dX.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+    assert np.array_equal(dX, ref["c_seq"])
+
+
+def test_backward_data_filter_operand_says_what_it_does_not_cover(hb):
+    w = wl.draw("he_weight", (9 * 24, 40), seed=96, fan_in=9 * 24)
+    fd = dict(mant_bits=8, block=24, tile=24)
+    _, c1, _ = hb.quantize_conv_weights(to_dev(w), 9, gfmt(fd))
+    with pytest.raises(hb.HbfpError) as e:
+        hb.conv_dgrad_filters(c1, 3, 3, 24, 40)
+    assert e.value.code == hb.ERR_UNSUPPORTED

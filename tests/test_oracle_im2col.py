@@ -5,6 +5,7 @@ import pytest
 
 import oracle
 from oracle import Format
+from tests.helpers import dgrad_filters_view
 
 
 @pytest.mark.parametrize("n,h,w,c,kh,kw,pad,f", [(2, 5, 6, 3, 3, 3, 1, 4), (1, 4, 4, 2, 1, 1, 0, 3), (2, 6, 5, 4, 3, 3, 0, 2),
@@ -89,3 +90,25 @@ def test_im2col_index_names_the_activation_each_entry_copies():
     # every interior activation appears once per tap
     counts = np.bincount(idx[inside], minlength=flat.size).reshape(n, h, w, c)
     assert (counts[:, 1:-1, 1:-1, :] == 9).all()
+
+
+@pytest.mark.parametrize("n,h,w,c,k,pad,f", [(2, 5, 6, 3, 3, 1, 4), (1, 6, 5, 2, 5, 2, 3), (2, 4, 4, 3, 1, 0, 2), (1, 7, 6, 2, 3, 0, 3),
+                                             (1, 6, 6, 2, 3, 2, 2)])
+def test_backward_data_is_the_gather_of_the_gradient_times_the_turned_filters(n, h, w, c, k, pad, f):
+    """The index transform the backward-data convolution rests on: the gradient with respect to the input is the
+    gather of the output gradient with padding k - 1 - pad times the filters with taps reversed and feature-map
+    roles swapped. Checked against the library's own derivative of its convolution, in integers held in float64."""
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(17 * n + h)
+    wt = rng.integers(-3, 4, size=(k * k * c, f)).astype(np.float64)
+    ho, wo = h + 2 * pad - k + 1, w + 2 * pad - k + 1
+    dy = rng.integers(-4, 5, size=(n, ho, wo, f)).astype(np.float64)
+    x = torch.zeros(n, c, h, w, dtype=torch.float64, requires_grad=True)
+    wt_t = torch.from_numpy(wt.reshape(k, k, c, f)).permute(3, 2, 0, 1).contiguous()      # [f][c][kh][kw]
+    y = torch.nn.functional.conv2d(x, wt_t, padding=pad)
+    y.backward(torch.from_numpy(dy).permute(0, 3, 1, 2).contiguous())
+    want = x.grad.permute(0, 2, 3, 1).numpy()                                             # [n][h][w][c]
+    turned, _ = dgrad_filters_view(wt, np.zeros((k * k * c, 1)), k * k, c)                # [c][taps * f]
+    got = oracle.im2col(dy, k, k, k - 1 - pad) @ turned.T
+    assert got.shape == (n * h * w, c)
+    assert np.array_equal(got.reshape(n, h, w, c), want)
