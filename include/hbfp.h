@@ -287,7 +287,7 @@ HBFP_API int hbfp_gemm_q_workspace(int64_t M, int64_t N, int64_t K, const hbfp_o
  * 2^(sA + sB) into two factors and need more: the paired-SM kernel chooses the split per K-block and
  * 128-row tile and fails only when that tile's row exponents span more than 104 within one block
  * (or the products leave binary32); the single-SM kernel's biased path needs sA <= 103 (|A| < 2^110
- * at 8-bit mantissas). A kernel that meets exponents outside its range does not depart silently: it
+ * at 8-bit mantissas; sA <= 96 for 12-bit mantissas). A kernel that meets exponents outside its range does not depart silently: it
  * records a code in the device status word (hbfp_device_status then returns
  * HBFP_ERR_EXPONENT_RANGE) and the values of C it wrote for that call are unspecified;
  * HBFP_GEMM_FORCE_SIMT computes the same product without the restriction. */

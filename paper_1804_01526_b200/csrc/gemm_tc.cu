@@ -24,8 +24,12 @@
 //   t   = fma(v, 2^sA, -1.5*2^23 * 2^sA)   = P * 2^sA          (exact)
 //   acc = fma(t, 2^sB, acc)                = acc + P*2^(sA+sB) (one rounding, as the definition)
 // both as packed two-wide FP32 FMAs; after reading a chunk the warp stores the bias back.
-// Other formats (12-bit planes, longer blocks) clear the accumulator with the first MMA of a
-// block and convert with cvt.rn.f32.s32.
+// 12-bit mantissas with blocks below 256 take the same route with three armed parts per group: one FMA per
+// part removes the bias and applies the part's weight (256, 16, 1) and 2^sA exactly, two additions form
+// float(P) * 2^sA with the single rounding of the definition, one FMA accumulates it times 2^sB.
+// Longer blocks clear the accumulator with the first MMA of a block and convert with cvt.rn.f32.s32.
+// The MMA thread and the rescale warps wait for their barriers with a few looks, then naps of at most 64 ns
+// (a suspended wait of unbounded length wakes late; a spinning one takes issue slots from the rescale warps).
 //
 // Every wait on an mbarrier is bounded: when it expires the CTA records a code in the device
 // status word, raises a shared abort flag, drains its own copies and MMAs (bounded again),
@@ -157,6 +161,22 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
     return done != 0;
 }
 
+__device__ __forceinline__ bool mbar_try_wait_ns(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+// A few looks at the barrier, then naps of at most 64 ns (no issue slots taken from the arithmetic warps), then the
+// bounded wait.
+__device__ __forceinline__ bool mbar_wait_quick(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
+    for (int i = 0; i < 32; ++i)
+        if (mbar_test_wait(bar, parity)) return true;
+    for (int i = 0; i < 1024; ++i)
+        if (mbar_try_wait_ns(bar, parity, 64u)) return true;
+    return mbar_wait(bar, parity, abort_flag, status, code);
+}
+
 // 2^e as binary32 bits (MAGIC) or the exponent shifted into the exponent field, e = signed byte i of
 // a packed word of exponents.
 __device__ __forceinline__ uint32_t exp_to_field(uint32_t packed, int i, int add) {
@@ -197,7 +217,7 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
         int left = w.nblk, sib = 0;
         for (int si = 0; ok && si < nst; ++si, ++it) {
             if (pre_full) pre_full = false;
-            else if (!mbar_wait(a.full_bar + 8 * s, ph, a.abort_flag, p.status, 201)) { ok = false; break; }
+            else if (!mbar_wait_quick(a.full_bar + 8 * s, ph, a.abort_flag, p.status, 201)) { ok = false; break; }
             tc_fence_after();
             const uint32_t ms = a.mant_base + s * C::MANT_STAGE;
             const uint64_t a_hi = smem_desc_sw128(ms), b_hi = smem_desc_sw128(ms + PLANES * C::A_BYTES);
@@ -212,7 +232,7 @@ __device__ __forceinline__ void mma_issue_loop(const Problem& p, const Shape& sh
                     if (first) {
                         // the group was read (and, on the biased path, re-armed) by all rescale warps
                         if (pre_tempty) pre_tempty = false;
-                        else if (!mbar_wait(a.tempty_bar + 8 * g, gph, a.abort_flag, p.status, 202)) { ok = false; break; }
+                        else if (!mbar_wait_quick(a.tempty_bar + 8 * g, gph, a.abort_flag, p.status, 202)) { ok = false; break; }
                         tc_fence_after();
                     }
                     const uint32_t d = a.tmem_base + g * PARTS * N_TILE;
@@ -277,7 +297,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
     using C = Cfg<N_TILE, PLANES, TSTORE>;
     constexpr int STAGES = C::STAGES, GROUPS = C::GROUPS, PARTS = C::PARTS, TSLOTS = C::TABLE_SLOTS;
     constexpr int COLS_PER_WARP = N_TILE / COL_GROUPS;  // warps that share a lane quarter split the columns
-    static_assert(!(MAGIC && PLANES != 1), "the biased-accumulator path is for one-plane operands");
 
     extern __shared__ unsigned char smem_dyn[];
     const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
@@ -404,7 +423,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                         const uint32_t ra = *reinterpret_cast<const uint32_t*>(eA + jb * TILE_M + 4 * lane);
                         // the biased path forms 1.5 * 2^23 * 2^sA: finite up to sA = 103; beyond it the result
                         // would be wrong, which is reported instead
-                        if (MAGIC) out_of_range |= __vmaxs4(ra, 0x67676767u) != 0x67676767u;
+                        // (two planes: 1.5 * 2^31 * 2^sA and 2^29 * 2^sA, finite up to sA = 96)
+                        if (MAGIC) out_of_range |= __vmaxs4(ra, PLANES == 1 ? 0x67676767u : 0x60606060u) != (PLANES == 1 ? 0x67676767u : 0x60606060u);
                         uint32_t cs[CPL];
 #pragma unroll
                         for (int i = 0; i < CPL; ++i) cs[i] = exp_to_field(cw[i >> 2], i & 3, MAGIC ? 127 : 0);
@@ -452,9 +472,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
                 uint32_t bias[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) bias[i] = BIAS_BITS;
-                for (int g = 0; g < GROUPS; ++g)
+                for (int gp = 0; gp < GROUPS * PARTS; ++gp)
 #pragma unroll
-                    for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + g * N_TILE + c8 * 8, bias);
+                    for (int c8 = 0; c8 < COLS_PER_WARP / 8; ++c8) tc_st8(lane_addr + gp * N_TILE + c8 * 8, bias);
                 tc_wait_st();
             }
             // Read the bias back as one sixteen-register tuple: a tuple that is born as such is passed
@@ -479,12 +499,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant_
             for (int c = 0; c < COLS_PER_WARP / 2; ++c) acc2[c] = 0ull;
             for (int kb = w.kb0; kb < w.kb0 + w.nblk; ++kb, ++blk) {
                 // one wait per block: the block sums are complete and the scale table is written
-                if (!mbar_wait_warp(tfull_bar + 8 * g, gph, abort_flag, p.status, 302)) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait_quick(tfull_bar + 8 * g, gph, abort_flag, p.status, 302))) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = lane_addr + g * PARTS * N_TILE;
                 const uint32_t* tab = tables + slot * C::TABLE_SLOT_WORDS + col0;
                 const uint32_t sa_u = tables[slot * C::TABLE_SLOT_WORDS + N_TILE + row];
-                if (MAGIC) {
+                if (MAGIC && PLANES == 2) {
+                    // Two planes, mantissa = 16 hi + lo: the three armed parts read as binary32 are 1.5*2^23 + hi.hi,
+                    // + (hi.lo + lo.hi), + lo.lo. One FMA each removes the bias and applies the part's weight and the
+                    // row scale, all exactly: 256 hi.hi 2^sA, 16 mid 2^sA, lo.lo 2^sA. The two lower parts add up
+                    // exactly (below 2^23 units); adding the upper part is the one rounding of float(P), which a power
+                    // of two does not move; then acc += that * 2^sB. No integer-to-float conversion, no integer
+                    // arithmetic per element.
+                    const float sa_f = __uint_as_float(sa_u);
+                    const float k1 = 16.0f * sa_f, k2 = 256.0f * sa_f;
+                    const float c0 = -12582912.0f * sa_f, c1 = -12582912.0f * k1, c2 = -12582912.0f * k2;
+                    const uint64_t k0_2 = pack2(__float_as_uint(sa_f), __float_as_uint(sa_f)), c0_2 = pack2(__float_as_uint(c0), __float_as_uint(c0));
+                    const uint64_t k1_2 = pack2(__float_as_uint(k1), __float_as_uint(k1)), c1_2 = pack2(__float_as_uint(c1), __float_as_uint(c1));
+                    const uint64_t k2_2 = pack2(__float_as_uint(k2), __float_as_uint(k2)), c2_2 = pack2(__float_as_uint(c2), __float_as_uint(c2));
+                    constexpr int CH = 16;
+                    constexpr int NCHK = COLS_PER_WARP / CH;
+                    uint32_t v[2][3][CH];
+#pragma unroll
+                    for (int part = 0; part < 3; ++part) tc_ld16(taddr + part * N_TILE, v[0][part]);
+#pragma unroll
+                    for (int ch = 0; ch < NCHK; ++ch) {
+                        tc_wait_ld();
+                        if (ch + 1 < NCHK) {
+#pragma unroll
+                            for (int part = 0; part < 3; ++part) tc_ld16(taddr + part * N_TILE + (ch + 1) * CH, v[(ch + 1) & 1][part]);
+                        }
+                        const uint32_t(&xh)[CH] = v[ch & 1][0];
+                        const uint32_t(&xm)[CH] = v[ch & 1][1];
+                        const uint32_t(&xl)[CH] = v[ch & 1][2];
+                        if (DUMP && p.P != nullptr && gi < p.M) {
+#pragma unroll
+                            for (int c = 0; c < CH; ++c) {
+                                const int64_t gj = n0 + col0 + ch * CH + c;
+                                if (gj < p.N)
+                                    p.P[(gi * p.N + gj) * p.nkb + kb] =
+                                        (int32_t)(((xh[c] - BIAS_BITS) << 8) + ((xm[c] - BIAS_BITS) << 4) + (xl[c] - BIAS_BITS));
+                            }
+                        }
+#pragma unroll
+                        for (int q = 0; q < CH; q += 2) {
+                            const uint2 sb = *reinterpret_cast<const uint2*>(tab + ch * CH + q);
+                            const uint64_t h01 = ffma2(pack2(xh[q], xh[q + 1]), k2_2, c2_2);
+                            const uint64_t m01 = ffma2(pack2(xm[q], xm[q + 1]), k1_2, c1_2);
+                            const uint64_t l01 = ffma2(pack2(xl[q], xl[q + 1]), k0_2, c0_2);
+                            const uint64_t p01 = fadd2(h01, fadd2(m01, l01));
+                            acc2[(ch * CH + q) / 2] = ffma2(p01, pack2(sb.x, sb.y), acc2[(ch * CH + q) / 2]);
+                        }
+#pragma unroll
+                        for (int part = 0; part < 3; ++part)
+                            tc_st16(taddr + part * N_TILE + ch * CH, reinterpret_cast<const uint32_t(&)[16]>(bias16));   // re-arm
+                    }
+                    tc_wait_st();
+                } else if (MAGIC) {
                     // the accumulator was armed with 0x4B400000, so a block sum read as binary32 is
                     // v = 1.5*2^23 + P exactly;  t = (v - 1.5*2^23) * 2^sA = P * 2^sA;  acc += t * 2^sB
                     const float sa_f = __uint_as_float(sa_u);
@@ -789,15 +860,16 @@ int launch_gemm_tensor(int64_t M, int64_t N, int64_t K, const Packed& a, const P
     int rc;
     // the biased-accumulator path needs every |P| < 2^22
     const int64_t qa = (1ll << (a.mant_bits - 1)) - 1, qb = (1ll << (b.mant_bits - 1)) - 1;
-    const bool magic = a.L.planes == 1 && qa * qb * a.L.b < (1ll << 22);
+    // (two planes: the largest part, hi.hi, stays below 128 * 128 * b)
+    const bool magic = a.L.planes == 1 ? qa * qb * a.L.b < (1ll << 22) : 128ll * 128ll * a.L.b < (1ll << 22);
     // Short contractions are bound by the write of C: the tile then leaves through shared memory and TMA stores,
     // which the copy engine writes as whole lines while the warps go on with the next tile.
     const bool tstore = p.splits == 1 && !P && a.L.nkb * a.L.bp <= 1024 && (reinterpret_cast<uintptr_t>(Cout) & 15) == 0 && (ldc % 4) == 0;
     if (P) {   // the inspection build of the kernel: 64-column tiles, writes the block sums
         p.tiles_n = (int)((N + 63) / 64);
-        if (a.L.planes == 2) rc = launch_cfg<64, 2, false, true>(p, a, b, st);
+        if (a.L.planes == 2) rc = magic ? launch_cfg<64, 2, true, true>(p, a, b, st) : launch_cfg<64, 2, false, true>(p, a, b, st);
         else rc = magic ? launch_cfg<64, 1, true, true>(p, a, b, st) : launch_cfg<64, 1, false, true>(p, a, b, st);
-    } else if (a.L.planes == 2) rc = launch_cfg<64, 2, false, false>(p, a, b, st);
+    } else if (a.L.planes == 2) rc = magic ? launch_cfg<64, 2, true, false>(p, a, b, st) : launch_cfg<64, 2, false, false>(p, a, b, st);
     else if (magic && tstore && plan.n_tile == 256) rc = launch_cfg<256, 1, true, false, true>(p, a, b, st);
     else if (magic && tstore && plan.n_tile == 128) rc = launch_cfg<128, 1, true, false, true>(p, a, b, st);
     else if (plan.n_tile == 256) rc = magic ? launch_cfg<256, 1, true, false>(p, a, b, st) : launch_cfg<256, 1, false, false>(p, a, b, st);

@@ -311,6 +311,25 @@ def test_large_magnitudes_are_computed_or_reported_never_silently_wrong(hb, kern
     assert rc == hb.OK and np.array_equal(C, ref["c_seq"])
 
 
+def test_large_magnitudes_with_two_plane_mantissas_are_computed_or_reported(hb):
+    """12-bit mantissas take the biased path of the single-SM kernel with a narrower exponent range
+    (the bias is scaled by 256 * 2^sA): inside it the result is the oracle's, outside the status says so."""
+    M, N, K = 384, 320, 256
+    fd = dict(mant_bits=12, block=64)
+    B = wl.draw("normal", (K, N), seed=178)
+    for scale_a, scale_b in ((2.0 ** 60, 1.0), (2.0 ** 100, 2.0 ** -40), (2.0 ** 112, 2.0 ** -60), (1.0, 1.0)):
+        A = (wl.draw("normal", (M, K), seed=179) * np.float32(scale_a)).astype(np.float32)
+        Bs = (B * np.float32(scale_b)).astype(np.float32)
+        ref = oracle.hbfp_gemm(0, 0, A, Bs, ofmt(fd), ofmt(fd, stream_id=1))
+        C = hb.gemm(0, 0, to_dev(A), to_dev(Bs), gfmt(fd), gfmt(fd, stream_id=1), flags=hb.GEMM_FORCE_TENSOR_1SM).cpu().numpy()
+        rc, code = hb.device_status_rc()
+        if rc == hb.OK:
+            assert np.array_equal(C, ref["c_seq"]), (scale_a, scale_b)
+        else:
+            assert scale_a > 2.0 ** 80 and rc == hb.ERR_EXPONENT_RANGE and 900 <= code < 1000
+    assert rc == hb.OK            # the last, ordinary case ran clean
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_leaves_the_library_usable(hb):
     """The wait routine of the GEMM kernels, on a barrier nobody arrives on, with a budget of a few
     thousand cycles: the status word carries the code, the next read is clean, the next GEMM is right."""
