@@ -123,7 +123,18 @@ class _HbfpConv3x3Fn(torch.autograd.Function):
         dy2 = dy.contiguous().view(n * h * w, f)
         dx = dw = None
         if ctx.needs_input_grad[0]:
-            # gradient of the im2col matrix, then its scatter back onto the pixels (an FP32 operation)
+            try:
+                # the convolution of the packed output gradient with the forward weights regrouped (taps turned by
+                # 180 degrees, feature-map roles swapped) yields dX itself
+                pg = hb.quantize(dy2, 1, layer.fmt_pixels(2))
+                turned = hb.conv_dgrad_filters(layer.views[1], 3, 3, c, f)
+                dx = hb.conv_forward(pg, turned, n, h, w, f, 3, 3, 1).view(n, h, w, c)
+            except hb.HbfpError as e:
+                if e.code != hb.ERR_UNSUPPORTED:
+                    raise
+        if ctx.needs_input_grad[0] and dx is None:
+            # shapes that route does not cover: gradient of the im2col matrix, then its scatter back onto the
+            # pixels (an FP32 operation)
             dcols = hb.gemm_q(n * h * w, 9 * c, f, dy2, layer.views[1], fmtA=layer.fmt_pixels(2)).view(n, h, w, 3, 3, c)
             dxp = torch.zeros((n, h + 2, w + 2, c), device=x.device)
             for i in range(3):
@@ -140,7 +151,8 @@ class HbfpConv3x3(torch.nn.Module):
     """3 x 3 convolution, stride 1, one pixel of zero padding, channels-last activations ``[n][h][w][c]``,
     as three BFP GEMMs (Sec. 5.1) without an FP32 im2col matrix: the forward operand is gathered from
     activations converted once per pixel, the backward-weight operand is converted straight from the
-    activations, backward-data is a GEMM followed by the FP32 scatter onto the pixels. The weights
+    activations, backward-data is the same implicit GEMM on the packed output gradient with the regrouped
+    forward weights (a GEMM followed by the FP32 scatter onto the pixels where that does not apply). The weights
     ``[9 c][filters]`` (rows ordered (filter row, filter column, channel)) live in wide storage with
     ``c x c`` tiles, so the K-blocks of weights and activations coincide. Nearest-even rounding."""
 

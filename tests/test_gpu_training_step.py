@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 import oracle
-from tests.helpers import ofmt
+from tests.helpers import dgrad_filters_view, ofmt
 
 pytestmark = pytest.mark.gpu
 
@@ -144,6 +144,13 @@ def test_convolution_layer_products_match_the_oracle_and_fp32(env):
             dxp[:, i:i + hw, j:j + hw, :] += dcols[:, :, :, i, j, :]
     dx_ref = dxp[:, 1:hw + 1, 1:hw + 1, :]
     assert np.allclose(x.grad.cpu().numpy(), dx_ref, rtol=1e-4, atol=1e-6)
+    # ... computed as the convolution of the packed gradient with the regrouped forward weights: bit for bit the
+    # oracle's GEMM on the gathered quantised gradient, taps in that operand's order
+    qa = oracle.im2col(qd.reshape(n, hw, hw, f), 3, 3, 1)
+    sa = oracle.im2col(sd.reshape(n, hw, hw, 1), 3, 3, 1)
+    qb, sb = dgrad_filters_view(qm, sm, 9, c)
+    ref = oracle.gemm(qa, sa, qb, sb, t)
+    assert np.array_equal(x.grad.cpu().numpy().reshape(n * hw * hw, c), ref["c_seq"])
     # and the whole layer stays close to the FP32 convolution it stands for
     w4 = layer.weight.detach().view(3, 3, c, f).permute(3, 2, 0, 1).contiguous()          # [f][c][3][3]
     y32 = torch.nn.functional.conv2d(x.detach().permute(0, 3, 1, 2), w4, padding=1).permute(0, 2, 3, 1)
