@@ -259,11 +259,14 @@ typedef struct hbfp_operand {
     hbfp_format fmt;    /* FP32: format to quantise to. PACKED: format it was quantised with         */
 } hbfp_operand;
 
-#define HBFP_GEMM_AUTO 0u        /* tensor-core kernel when it supports the case, else SIMT */
+#define HBFP_GEMM_AUTO 0u        /* smallest problems: tiled kernel; else a tensor-core kernel when it supports the case, else SIMT */
 #define HBFP_GEMM_FORCE_SIMT 1u  /* plain dp4a kernel (reference path, any format)           */
 #define HBFP_GEMM_FORCE_TENSOR 2u /* tcgen05 kernel or HBFP_ERR_UNSUPPORTED                  */
 #define HBFP_GEMM_FORCE_TENSOR_1SM 3u  /* as FORCE_TENSOR, but never the paired-SM tile kernel */
 #define HBFP_GEMM_FORCE_TENSOR_2SM 4u  /* paired-SM tile kernel or HBFP_ERR_UNSUPPORTED        */
+#define HBFP_GEMM_FORCE_SMALL 5u       /* the tiled kernel that HBFP_GEMM_AUTO takes for the smallest problems (contraction
+                                          of at most 512 bytes, at most 296 tiles of 32 x 32; one launch, no split-K,
+                                          one-plane operands) at any size, or HBFP_ERR_UNSUPPORTED */
 
 /* Host-only: bytes of workspace hbfp_gemm / hbfp_gemm_q need for this problem (packed copies
  * of FP32 operands, split-K partial tiles). Depends only on its arguments. */

@@ -20,7 +20,7 @@ LIB_PATH = os.environ.get("HBFP_LIBRARY") or os.path.join(_HERE, "libhbfp.so")
 (OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT,
  ERR_STATIC_LIMIT, ERR_EXPONENT_RANGE) = range(9)
 STATIC_WORKSPACE_BYTES = 16 << 20
-GEMM_AUTO, GEMM_FORCE_SIMT, GEMM_FORCE_TENSOR, GEMM_FORCE_TENSOR_1SM, GEMM_FORCE_TENSOR_2SM = 0, 1, 2, 3, 4
+GEMM_AUTO, GEMM_FORCE_SIMT, GEMM_FORCE_TENSOR, GEMM_FORCE_TENSOR_1SM, GEMM_FORCE_TENSOR_2SM, GEMM_FORCE_SMALL = 0, 1, 2, 3, 4, 5
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 
 EXPORTS = [

@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhbfp.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm_simt.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_conv.cu", "gemm_static.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm_simt.cu", "gemm_small.cu", "gemm_tc.cu", "gemm_tc2.cu", "gemm_conv.cu", "gemm_static.cu"]
 # (object name, source, extra flags): quantize.cu is compiled a second time for the full-tile kernel of small tiles
 EXTRA_OBJECTS = [("quantize_tiles_small.o", "quantize.cu", ["-DHBFP_QUANT_PART=2", "-Xptxas", "-O1"])]
 # Per-file additions. The paired-SM GEMM is built with ptxas -O1: measured in SM cycles per launch (16384^3, b = 128)

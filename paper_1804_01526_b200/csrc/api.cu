@@ -110,7 +110,7 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
     GemmPlan g;
     int rc = make_plan(M, N, K, a, b, &g);
     if (rc) return rc;
-    if (flags > HBFP_GEMM_FORCE_TENSOR_2SM) return HBFP_ERR_INVALID_ARG;
+    if (flags > HBFP_GEMM_FORCE_SMALL) return HBFP_ERR_INVALID_ARG;
     if (P) {   // the inspection hook never splits K and needs no scratch
         g.total -= align_up(g.tp.partial_bytes, 1024);
         g.tp.partial_bytes = 0;
@@ -129,6 +129,13 @@ int gemm_impl(int64_t M, int64_t N, int64_t K, const hbfp_operand* a, const hbfp
     if (rc) return rc;
     rc = resolve_operand(b, false, N, K, g.lb, ws, g.off_bm, g.off_be, &pb, st);
     if (rc) return rc;
+    // a problem of a few hundred MOPs is over before a tensor-core kernel has filled its pipeline
+    if (!P && (flags == HBFP_GEMM_AUTO || flags == HBFP_GEMM_FORCE_SMALL) &&
+        small_gemm_eligible(M, N, pa, pb, flags == HBFP_GEMM_FORCE_SMALL)) {
+        t_last_gemm_kernel = "gemm_small_kernel";
+        return launch_gemm_small(M, N, pa, pb, C, ldc, st);
+    }
+    if (flags == HBFP_GEMM_FORCE_SMALL) return HBFP_ERR_UNSUPPORTED;
     const bool quad_rows = (reinterpret_cast<uintptr_t>(C) & 15) == 0 && (ldc % 4) == 0;
     const bool want_tensor = flags != HBFP_GEMM_FORCE_SIMT && g.tp.supported &&
                              (reinterpret_cast<uintptr_t>(C) & 3) == 0;

@@ -92,6 +92,10 @@ int launch_dequantize(const Packed& p, float* out, int64_t ld, cudaStream_t st);
 int launch_gemm_simt(int64_t M, int64_t N, int64_t K, const Packed& a, const Packed& b, float* C,
                      int64_t ldc, int32_t* P, cudaStream_t st);
 
+// Tiled dp4a kernel for small problems (gemm_small.cu): one-plane operands, one launch, no split-K.
+bool small_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b, bool any_size);
+int launch_gemm_small(int64_t M, int64_t N, const Packed& a, const Packed& b, float* C, int64_t ldc, cudaStream_t st);
+
 struct TensorPlan {
     int supported;      // 0: this case has no tensor-core kernel
     int n_tile;         // 64, 128 or 256

@@ -73,6 +73,49 @@ def test_transformer_gemms_reduced(hb, flag):
                  expect_seq=(flag == "simt"))
 
 
+SMALL_CASES = [
+    # transA, transB, M, N, K, mantissa bits, block, tile of B, rounding
+    (0, 0, 128, 1024, 784, 8, 24, 24, 1),       # forward GEMM of the MLP configuration
+    (0, 1, 128, 784, 1024, 8, 24, 24, 1),       # its backward-data GEMM (shared tiles read the other way)
+    (1, 0, 784, 1024, 128, 8, 24, 0, 1),        # its backward-weight GEMM
+    (0, 0, 1, 1, 1, 8, 32, 0, 0),
+    (0, 0, 33, 95, 100, 6, 64, 0, 0),           # ragged in every dimension, two 32-byte steps per block
+    (0, 0, 70, 50, 520, 8, 128, 0, 0),
+    (1, 1, 40, 72, 900, 8, 200, 0, 1),          # blocks that span two 128-byte slices
+    (0, 0, 64, 48, 300, 8, 0, 0, 0),            # one exponent per row / column
+    (0, 0, 256, 256, 256, 4, 32, 32, 0),
+]
+
+
+@pytest.mark.parametrize("tA,tB,M,N,K,m,b,t,rounding", SMALL_CASES)
+def test_small_problem_kernel_equals_the_sequential_definition(hb, tA, tB, M, N, K, m, b, t, rounding):
+    """The tiled kernel for the smallest problems never splits K and adds blocks in ascending order: bit-equal to the oracle's c_seq."""
+    A = wl.draw("lognormal", (K, M) if tA else (M, K), seed=31)
+    B = wl.draw("he_weight", (N, K) if tB else (K, N), seed=32, fan_in=K)
+    fa = dict(mant_bits=m, block=b, rounding=rounding, seed=4, stream_id=0)
+    fb = dict(mant_bits=m, block=b, tile=t, rounding=rounding, seed=4, stream_id=1)
+    ref = oracle.hbfp_gemm(tA, tB, A, B, ofmt(fa), ofmt(fb))
+    C = hb.gemm(tA, tB, to_dev(A), to_dev(B), gfmt(fa), gfmt(fb), flags=hb.GEMM_FORCE_SMALL).cpu().numpy()
+    assert hb.device_status() == 0 and hb.last_gemm_kernel() == "gemm_small_kernel"
+    assert np.array_equal(C, ref["c_seq"])
+    err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
+    assert (err <= TOL * ref["a_mag"]).all()
+
+
+def test_small_problem_kernel_is_what_small_problems_get_and_large_ones_do_not(hb):
+    fd = dict(mant_bits=8, block=64)
+    A, B = wl.draw("normal", (256, 512), seed=33), wl.draw("normal", (512, 256), seed=34)
+    hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd, stream_id=1))
+    assert hb.last_gemm_kernel() == "gemm_small_kernel"
+    A, B = wl.draw("normal", (1024, 2048), seed=35), wl.draw("normal", (2048, 1024), seed=36)
+    hb.gemm(0, 0, to_dev(A), to_dev(B), gfmt(fd), gfmt(fd, stream_id=1))
+    assert hb.last_gemm_kernel() == "gemm_tc_kernel"
+    f12 = dict(mant_bits=12, block=64)
+    with pytest.raises(hb.HbfpError) as e:
+        hb.gemm(0, 0, to_dev(A[:64, :128].copy()), to_dev(B[:128, :64].copy()), gfmt(f12), gfmt(f12, stream_id=1), flags=hb.GEMM_FORCE_SMALL)
+    assert e.value.code == hb.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("impl", ["simt", "tensor"])
 @pytest.mark.parametrize("m,b,M,N,K", [(8, 32, 200, 136, 288), (8, 128, 130, 260, 1024), (12, 64, 96, 72, 320),
                                        (8, 24, 50, 40, 100), (8, 0, 64, 64, 700), (8, 64, 128, 256, 512)])
