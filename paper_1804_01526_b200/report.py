@@ -115,11 +115,12 @@ def mlp_step_lines():
 def wide_lines(hbm_gbs):
     """Wide weight storage on the weight matrices of the configurations: first conversion, in-place
     FP32 update (with the narrow views of the new weights) and the narrow views alone."""
-    out = ["", "| weights | format | wide quantise µs | wide update + views µs (GB/s, % HBM) | narrow views only µs | FP32 -> views (`hbfp_quantize_tiles`) µs |",
+    out = ["", "| weights | format | wide quantise µs | wide update + views µs (GB/s, % HBM) | narrow views only µs | FP32 -> views (`hbfp_quantize_tiles`) µs (GB/s, % HBM) |",
            "|---|---|---|---|---|---|"]
     for name, shape, fd in (("c1.l1.W", (1024, 1024), dict(mant_bits=8, block=24, tile=24, rounding=1, seed=1)),
                             ("c3.up.W", (1024, 4096), dict(mant_bits=12, block=64, tile=64, rounding=1, seed=7)),
                             ("8192 x 8192", (8192, 8192), dict(mant_bits=8, block=64, tile=64, rounding=0)),
+                            ("16384 x 16384", (16384, 16384), dict(mant_bits=8, block=64, tile=64, rounding=0)),
                             ("16384 x 16384", (16384, 16384), dict(mant_bits=8, block=128, tile=128, rounding=0))):
         fmt = hb.Format(**fd)
         w = torch.from_numpy(wl.draw("he_weight", shape, seed=3, fan_in=shape[0])).cuda()
@@ -133,9 +134,10 @@ def wide_lines(hbm_gbs):
         n = shape[0] * shape[1]
         bytes_u = n * (2 + 4 + 2 + 2 * planes)          # read wide + delta, write wide + both views
         gbs = bytes_u / (t_u * 1e-3) / 1e9
+        gbs_t = n * (4 + 2 * planes) / (t_t * 1e-3) / 1e9      # read FP32, write both views
         f = f"m{fd['mant_bits']} t{fd['tile']}" + (" SR" if fd["rounding"] else " RNE")
         out.append(f"| {name} {shape[0]}x{shape[1]} | {f} | {t_q*1e3:.1f} | {t_u*1e3:.1f} ({gbs:.0f}, {100*gbs/hbm_gbs:.0f} %) | "
-                   f"{t_n*1e3:.1f} | {t_t*1e3:.1f} |")
+                   f"{t_n*1e3:.1f} | {t_t*1e3:.1f} ({gbs_t:.0f}, {100*gbs_t/hbm_gbs:.0f} %) |")
         del w, dw, wide, views
     torch.cuda.empty_cache()
     return out
