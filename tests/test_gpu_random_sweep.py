@@ -60,6 +60,7 @@ def test_random_gemm_cases(hb, seed):
     import torch
     rng = np.random.default_rng(100 + seed)
     done = 0
+    ran = {}
     for _ in range(45):
         M, N, K = (int(rng.integers(1, 600)) for _ in range(3))
         if rng.random() < 0.3:
@@ -76,10 +77,19 @@ def test_random_gemm_cases(hb, seed):
         fa = dict(mant_bits=m, block=b, rounding=int(rng.integers(0, 2)), seed=int(rng.integers(0, 1000)), stream_id=0)
         fb = dict(fa, stream_id=1)
         ref = oracle.hbfp_gemm(tA, tB, A, B, oracle.Format(**fa), oracle.Format(**fb))
-        for flags in (hb.GEMM_AUTO, hb.GEMM_FORCE_SIMT):
-            C = hb.gemm(tA, tB, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), hb.Format(**fa), hb.Format(**fb),
-                        flags=flags).cpu().numpy()
+        for flags in (hb.GEMM_AUTO, hb.GEMM_FORCE_SIMT, hb.GEMM_FORCE_TENSOR, hb.GEMM_FORCE_SMALL):
+            try:
+                C = hb.gemm(tA, tB, torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), hb.Format(**fa), hb.Format(**fb),
+                            flags=flags).cpu().numpy()
+            except hb.HbfpError as e:
+                # a forced kernel may not cover the format (two-plane operands on the small-problem kernel, ...)
+                assert e.code == hb.ERR_UNSUPPORTED and flags in (hb.GEMM_FORCE_TENSOR, hb.GEMM_FORCE_SMALL), (M, N, K, m, b, flags)
+                continue
             err = np.abs(C.astype(np.float64) - ref["c_ref"].astype(np.float64))
             assert (err <= 1e-6 * ref["a_mag"] + 1e-300).all(), (M, N, K, m, b, tA, tB, flags)
+            if flags in (hb.GEMM_FORCE_SIMT, hb.GEMM_FORCE_SMALL):       # neither splits K: the sequential order
+                assert np.array_equal(C, ref["c_seq"]), (M, N, K, m, b, tA, tB, flags)
+            ran[flags] = ran.get(flags, 0) + 1
         done += 1
     assert hb.device_status() == 0 and done > 30
+    assert ran.get(hb.GEMM_FORCE_TENSOR, 0) > 20 and ran.get(hb.GEMM_FORCE_SMALL, 0) > 15, ran
