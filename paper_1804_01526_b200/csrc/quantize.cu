@@ -832,6 +832,48 @@ __global__ void exps_axis1(const float* __restrict__ x, int64_t rows, int64_t K,
     }
 }
 
+// One exponent per whole row (block = 0, "BFP without tiles", Sec. 6) for rows of 2048 G elements: a CTA per row
+// keeps the row in registers (eight elements per thread and step, G steps) between the maximum and the rounding,
+// so the tensor is read once.
+template <int G, bool SR, int PLANES>
+__global__ void __launch_bounds__(256)
+quant_row_whole(const float* __restrict__ x, int64_t ld, int64_t d1, QParams p, int8_t* __restrict__ mant, int64_t kst,
+                int64_t plane_stride, int8_t* __restrict__ exps) {
+    __shared__ uint32_t part[8];
+    const int tid = threadIdx.x;
+    const int64_t r = blockIdx.x;
+    const float4* src = reinterpret_cast<const float4*>(x + r * ld);
+    float e[G][8];
+    uint32_t am = 0;
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+        const int g = tid + 256 * i;
+        const float4 a = __ldg(src + 2 * g), b = __ldg(src + 2 * g + 1);
+        e[i][0] = a.x; e[i][1] = a.y; e[i][2] = a.z; e[i][3] = a.w;
+        e[i][4] = b.x; e[i][5] = b.y; e[i][6] = b.z; e[i][7] = b.w;
+    }
+#pragma unroll
+    for (int i = 0; i < G; ++i) am = max(am, amax8_bits(e[i]));
+    for (int off = 16; off > 0; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    if ((tid & 31) == 0) part[tid >> 5] = am;
+    __syncthreads();
+    am = part[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) am = max(am, part[i]);
+    const int s = block_exponent(am, p.m, p.exp_mode);
+    if (tid == 0) exps[r] = (int8_t)s;
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+        const int g = tid + 256 * i;
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (SR) w = draws_of_group(p, (uint64_t)(r * d1 + 8 * (int64_t)g) >> 3);
+        uint2 hi, lo;
+        quantize_pack8<SR, PLANES>(e[i], s, p, w, hi, lo);
+        *reinterpret_cast<uint2*>(mant + r * kst + 8 * g) = hi;
+        if (PLANES == 2) *reinterpret_cast<uint2*>(mant + plane_stride + r * kst + 8 * g) = lo;
+    }
+}
+
 // Pass 1b, blocks down columns: one thread per (block, line); neighbouring threads read
 // neighbouring addresses.
 __global__ void exps_axis0(const float* __restrict__ x, int64_t rows, int64_t K, int64_t ld, int64_t b,
@@ -1575,6 +1617,19 @@ int launch_quantize(const float* x, int64_t d0, int64_t d1, int64_t ld, int axis
     // then the fast kernel with the exponents given
     if (f->tile == 0 && axis == 1 && aligned && d1 % 8 == 0 && L.nkb == 1 && L.b == K && K > 256) {
         if (L.rs != rows) HBFP_CUDA_OK(cudaMemsetAsync(exps, 0, (size_t)L.exp_bytes, st));
+        // rows of 2048, 4096, 8192 or 16384 elements stay in a CTA's registers: one pass
+        if ((K == 2048 || K == 4096 || K == 8192 || K == 16384) && L.kst == K && rows < (1ll << 31)) {
+#define HBFP_QROW_WHOLE2(GV, SRV, PL) quant_row_whole<GV, SRV, PL><<<(unsigned)rows, 256, 0, st>>>(x, ld, d1, p, mant, L.kst, L.plane_stride, exps)
+#define HBFP_QROW_WHOLE(GV)                                                                          \
+    do {                                                                                             \
+        if (p.rounding == 1) { if (L.planes == 1) HBFP_QROW_WHOLE2(GV, true, 1); else HBFP_QROW_WHOLE2(GV, true, 2); }   \
+        else { if (L.planes == 1) HBFP_QROW_WHOLE2(GV, false, 1); else HBFP_QROW_WHOLE2(GV, false, 2); }                 \
+    } while (0)
+            if (K == 2048) HBFP_QROW_WHOLE(1); else if (K == 4096) HBFP_QROW_WHOLE(2); else if (K == 8192) HBFP_QROW_WHOLE(4); else HBFP_QROW_WHOLE(8);
+#undef HBFP_QROW_WHOLE
+#undef HBFP_QROW_WHOLE2
+            return launch_status();
+        }
         const int64_t want = (rows * 32 + 255) / 256;
         exps_axis1<<<(unsigned)(want < 148 * 16 ? want : 148 * 16), 256, 0, st>>>(x, rows, K, ld, L.b, L.nkb, p, exps, L.rs);
         if (launch_status()) return HBFP_ERR_CUDA;

@@ -130,6 +130,10 @@ ROW_WHOLE_AXIS_CASES = [
     ((1000, 2048), "outliers", F(8, 0, exp_mode=1)),
     ((72, 384), "grad", F(12, 0, rounding=1, seed=2)),                      # two planes
     ((33, 264), "normal", F(4, 0)),                                         # ragged last row tile
+    ((37, 4096), "lognormal", F(8, 0, rounding=1, seed=9, sid=1)),          # rows kept in registers: one pass
+    ((5, 8192), "outliers", F(6, 0)),
+    ((3, 16384), "lognormal", F(8, 0, rounding=1, seed=4)),
+    ((64, 1536), "normal", F(8, 0)),                                        # not a multiple of 2048: two passes
 ]
 
 
