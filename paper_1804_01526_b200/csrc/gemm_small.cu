@@ -147,7 +147,14 @@ bool small_gemm_eligible(int64_t M, int64_t N, const Packed& a, const Packed& b,
 int launch_gemm_small(int64_t M, int64_t N, const Packed& a, const Packed& b, float* C, int64_t ldc, cudaStream_t st) {
     const int nkb = (int)a.L.nkb;
     const size_t smem = 2 * SM_BUF + 2 * (size_t)nkb * SM_TILE;          // at most 132 KB
-    HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * SM_BUF + 2 * SM_MAX_NKB * SM_TILE));
+    // the attribute belongs to the device: set once per device (same value from any thread)
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HBFP_ERR_CUDA;
+    if (!attr_set[dev]) {
+        HBFP_CUDA_OK(cudaFuncSetAttribute(gemm_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * SM_BUF + 2 * SM_MAX_NKB * SM_TILE));
+        attr_set[dev] = true;
+    }
     const dim3 grid((unsigned)((N + SM_TILE - 1) / SM_TILE), (unsigned)((M + SM_TILE - 1) / SM_TILE));
     gemm_small_kernel<<<grid, 256, smem, st>>>(M, N, nkb, (int)a.L.bp, a.mant, a.L.kst, a.exps, a.L.rs, b.mant, b.L.kst,
                                                b.exps, b.L.rs, C, ldc);
