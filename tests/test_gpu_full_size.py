@@ -116,3 +116,69 @@ def test_transformer_full_size_tiled_weights_sampled(hb):
         Cs = C[ri][:, ci].cpu().numpy()
         err = np.abs(Cs.astype(np.float64) - ref["c_ref"].astype(np.float64))
         assert (err <= TOL * ref["a_mag"]).all(), sp.name
+
+
+def _gathered_rows(hw, ids_q, q_rows, s_rows, pix, c):
+    """im2col rows (3 x 3, one pixel of padding) of the sampled pixels `pix` from the canonical rows of the pixels
+    they touch: ids_q maps a pixel id to its line in q_rows / s_rows. Pure index movement."""
+    qa = np.zeros((len(pix), 9 * c), dtype=np.int16)
+    sa = np.zeros((len(pix), 9), dtype=np.int8)
+    for r, p in enumerate(pix):
+        img, rem = divmod(int(p), hw * hw)
+        y, x = divmod(rem, hw)
+        for tap in range(9):
+            yy, xx = y + tap // 3 - 1, x + tap % 3 - 1
+            if 0 <= yy < hw and 0 <= xx < hw:
+                k = ids_q[img * hw * hw + yy * hw + xx]
+                qa[r, tap * c:(tap + 1) * c] = q_rows[k]
+                sa[r, tap] = s_rows[k, 0]
+    return qa, sa
+
+
+@pytest.mark.parametrize("hw,c", [(32, 64), (16, 128)])
+def test_convolutions_full_batch_sampled(hb, hw, c):
+    """The two 3 x 3 convolutions of the ResNet configuration at batch 128 through the implicit-GEMM kernel,
+    forward and backward-data, on sampled pixels (image corners and edges among them): bit-equal to the
+    oracle's sequential GEMM on the gathered rows of oracle-quantised pixels."""
+    from tests.helpers import dgrad_filters_view
+    n, f = 128, c
+    rows = n * hw * hw
+    rng = np.random.default_rng(hw)
+    pix = np.unique(np.concatenate([[0, hw - 1, hw * hw - 1, rows - 1, rows - hw, 5 * hw * hw + 7 * hw],
+                                    rng.choice(rows, size=40, replace=False)]))
+    need = sorted({int(p) // (hw * hw) * hw * hw + yy * hw + xx
+                   for p in pix for yy in range(int(p) % (hw * hw) // hw - 1, int(p) % (hw * hw) // hw + 2)
+                   for xx in range(int(p) % hw - 1, int(p) % hw + 2) if 0 <= yy < hw and 0 <= xx < hw})
+    ids_q = {p: k for k, p in enumerate(need)}
+    wt = wl.draw("he_weight", (9 * c, f), seed=52, fan_in=9 * c)
+    fw = dict(mant_bits=8, block=c, tile=c, stream_id=1)
+    c0, c1, _ = hb.quantize_conv_weights(to_dev(wt), 9, gfmt(fw))
+    # forward
+    x = wl.draw("half_normal", (rows, c), seed=51)
+    fx = dict(mant_bits=8, block=c)
+    px = hb.quantize(to_dev(x), 1, gfmt(fx))
+    Y = hb.conv_forward(px, c0, n, hw, hw, c, 3, 3, 1)
+    assert hb.device_status() == 0 and hb.last_gemm_kernel() == "conv_fwd_kernel"
+    q_rows, s_rows = _lines(x, True, need, fx)
+    qa, sa = _gathered_rows(hw, ids_q, q_rows, s_rows, pix, c)
+    qb, sb = oracle.quantize_conv_weights(wt, 9, 0, ofmt(fw))
+    ref = oracle.gemm(qa, sa, qb, sb, c)
+    assert np.array_equal(Y[torch_index(pix)].cpu().numpy(), ref["c_seq"])
+    # backward-data: the packed output gradient (stochastic rounding, draws keyed by its own index) against the
+    # regrouped forward weights
+    dy = (wl.draw("normal", (rows, f), seed=53) * np.float32(0.03)).astype(np.float32)
+    fg = dict(mant_bits=8, block=f, rounding=1, seed=13, stream_id=2)
+    pg = hb.quantize(to_dev(dy), 1, gfmt(fg))
+    dX = hb.conv_forward(pg, hb.conv_dgrad_filters(c1, 3, 3, c, f), n, hw, hw, f, 3, 3, 1)
+    assert hb.device_status() == 0
+    q_rows, s_rows = _lines(dy, True, need, fg)
+    qa, sa = _gathered_rows(hw, ids_q, q_rows, s_rows, pix, f)
+    q1, s1 = oracle.quantize_conv_weights(wt, 9, 1, ofmt(fw))
+    qb, sb = dgrad_filters_view(q1, s1, 9, c)
+    ref = oracle.gemm(qa, sa, qb, sb, f)
+    assert np.array_equal(dX[torch_index(pix)].cpu().numpy(), ref["c_seq"])
+
+
+def torch_index(ids):
+    import torch
+    return torch.as_tensor(np.asarray(ids, dtype=np.int64), device="cuda")
