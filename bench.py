@@ -474,7 +474,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quantize-line", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the few-second back-to-back GEMM loop")
-    ap.add_argument("--e2e-panels", type=int, default=8, help="row panels of A in the end-to-end leg")
+    ap.add_argument("--e2e-panels", type=int, default=16, help="row panels of A in the end-to-end leg (16: 2 % faster than 8, as fast as 32)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
